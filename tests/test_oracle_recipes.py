@@ -1,0 +1,323 @@
+"""Pins for the oracle's recipes: an independent exact-rational evaluation on tiny blocks, closed
+forms and special cases, and the orderings and symmetries the method implies."""
+from fractions import Fraction as F
+
+import ml_dtypes
+import numpy as np
+import pytest
+import torch
+
+import exact_ref as ex
+from oracle import mxq_oracle as orc
+from paper_2605_08565_b200 import inputs
+
+f32 = np.float32
+FMTS = [orc.UE8M0, orc.UE4M3, orc.UE5M3]
+RECIPES = [orc.ABSMAX, orc.ABSMAX_PZ, orc.R4O6, orc.R4O6_PZ, orc.BRUTE, orc.BRUTE_PZ]
+
+
+def _unpack(codes):
+    codes = np.asarray(codes, dtype=np.uint8)
+    out = np.empty(codes.size * 2, dtype=np.uint8)
+    out[0::2] = codes & 15
+    out[1::2] = codes >> 4
+    return out
+
+
+def _tiny_blocks(seed, n_blocks, B):
+    """Small mix: normals at several magnitudes, short-mantissa (tie-prone) values, zeros."""
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal(n_blocks * B).astype(f32) * np.repeat(np.exp2(rng.integers(-12, 6, n_blocks)).astype(f32), B)
+    adv = inputs.adversarial(n_blocks * B, seed).numpy()
+    pick = np.repeat(rng.random(n_blocks) < 0.4, B)
+    big = np.abs(adv) > 1e6
+    return np.where(pick & ~big, adv, x).astype(f32)
+
+
+# ------------------------------------------------------------------------------------------------
+# Independent exact evaluation (every float op = exact rational + one rounding)
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("recipe", [orc.ABSMAX, orc.ABSMAX_PZ, orc.R4O6, orc.R4O6_PZ])
+@pytest.mark.parametrize("g", [1.0, 0.0123])
+def test_fast_recipes_equal_exact_reference(fmt, recipe, g):
+    B, nb = 8, 24
+    x = _tiny_blocks(100 + fmt * 10 + recipe, nb, B)
+    codes, scales, sse = orc.quantize(x, B, fmt, recipe, g)
+    c4 = _unpack(codes)
+    for b in range(nb):
+        v = x[b * B:(b + 1) * B]
+        code, s = ex.choose_exact(v, fmt, recipe, g)
+        assert int(scales[b]) == code, (b, v)
+        s2, cc = ex.eval_block_exact(v, fmt, code, g)
+        assert list(c4[b * B:(b + 1) * B]) == cc
+        assert f32(sse[b]).tobytes() == f32(s).tobytes() == f32(s2).tobytes()
+
+
+@pytest.mark.parametrize("fmt,g", [(orc.UE4M3, 1.0), (orc.UE4M3, 0.0371), (orc.UE5M3, 1.0), (orc.UE8M0, 0.0371)])
+@pytest.mark.parametrize("recipe", [orc.BRUTE, orc.BRUTE_PZ])
+def test_brute_force_equals_exact_reference(fmt, g, recipe):
+    B, nb = 4, 3
+    x = _tiny_blocks(200 + fmt, nb, B)
+    x[:B] = 0  # an all-zero block: every code ties at SSE 0, smallest admissible code wins
+    codes, scales, sse = orc.quantize(x, B, fmt, recipe, g)
+    for b in range(nb):
+        v = x[b * B:(b + 1) * B]
+        code, s = ex.choose_exact(v, fmt, recipe, g)
+        assert int(scales[b]) == code
+        assert f32(sse[b]).tobytes() == f32(s).tobytes()
+    assert int(scales[0]) == (1 if (recipe == orc.BRUTE_PZ and fmt != orc.UE8M0) else 0)
+
+
+def test_element_rounding_is_nearest_point_for_unit_global_scale():
+    # g = 1: the chosen code is the grid point nearest to v/S in exact arithmetic (ties -> even)
+    grid = ex.e2m1_magnitudes()
+    x = _tiny_blocks(300, 64, 16)
+    for fmt in (orc.UE4M3, orc.UE5M3):
+        codes, scales, _ = orc.quantize(x, 16, fmt, orc.ABSMAX)
+        c4 = _unpack(codes)
+        for b in range(64):
+            S = ex.TABLES[fmt]()[int(scales[b])]
+            for i in range(16):
+                v = x[b * 16 + i]
+                idx = int(c4[b * 16 + i]) & 7
+                assert (int(c4[b * 16 + i]) >> 3) == int(np.signbit(v))
+                if S == 0:
+                    assert idx == 0
+                    continue
+                q = abs(ex.frac(v)) / ex.frac(S)
+                assert idx == (7 if q >= 6 else ex.nearest_even_index(q, grid)), (v, S)
+
+
+# ------------------------------------------------------------------------------------------------
+# Special cases with a closed form
+# ------------------------------------------------------------------------------------------------
+def test_zero_scale_sets_everything_to_zero():
+    # "all values are set to zero": magnitudes 0, signs kept, SSE = sum v^2 in element order
+    x = np.array([1e-3, -2e-3, 3e-4, -0.0, 5e-3, -4e-3, 1e-5, 2e-3], dtype=f32)
+    codes, scales, sse = orc.quantize(x, 8, orc.UE4M3, orc.ABSMAX)
+    assert scales[0] == 0
+    assert list(_unpack(codes)) == [0, 8, 0, 8, 0, 8, 0, 0]
+    s = f32(0)
+    for v in x:
+        s = ex.f32_fma(v, v, s)
+    assert f32(sse[0]).tobytes() == s.tobytes()
+    # prevent-zero (Eq. 3) lifts the scale to the smallest nonzero value
+    codes, scales, sse_pz = orc.quantize(x, 8, orc.UE4M3, orc.ABSMAX_PZ)
+    assert scales[0] == 1 and sse_pz[0] < sse[0]
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_exact_reconstruction_of_on_grid_blocks(fmt):
+    rng = np.random.default_rng(5)
+    ncode = orc.num_codes(fmt)
+    for _ in range(40):
+        c = int(rng.integers(1 if fmt != orc.UE8M0 else 60, min(ncode, 200)))
+        S = f32(orc.scale_value(fmt, c))
+        mags = np.array([orc.e2m1_value(int(k)) for k in rng.integers(0, 16, 16)], dtype=f32)
+        mags[3] = 6.0  # the block maximum sits on the top grid point
+        x = (mags * S).astype(f32)
+        codes, scales, sse = orc.quantize(x, 16, fmt, orc.ABSMAX)
+        assert scales[0] == c and sse[0] == 0
+        xh = orc.dequantize(codes, scales, 16, 16, fmt)
+        assert np.array_equal(xh, x)
+
+
+def test_all_zero_tensor():
+    x = np.zeros(64, dtype=f32)
+    for fmt in FMTS:
+        for r in RECIPES:
+            codes, scales, sse = orc.quantize(x, 16, fmt, r)
+            want = 1 if (r in (orc.ABSMAX_PZ, orc.R4O6_PZ, orc.BRUTE_PZ) and fmt != orc.UE8M0) else 0
+            assert np.all(scales == want) and np.all(codes == 0) and np.all(sse == 0)
+
+
+def test_saturating_block_under_hierarchical_scale():
+    # the block holding the tensor maximum: amax/g = 2688 -> scale 448 (top code); the M = 4
+    # candidate also clips to 448, ties, and M = 6 is kept
+    x = inputs.normal(256, 3).numpy().copy()
+    x[17] = 9.5
+    g = orc.global_scale_from_amax(orc.tensor_amax(x))
+    _, sc_a, sse_a = orc.quantize(x, 16, orc.UE4M3, orc.ABSMAX, g)
+    _, sc_4, sse_4 = orc.quantize(x, 16, orc.UE4M3, orc.R4O6, g)
+    assert sc_a[1] == 0x7E and sc_4[1] == 0x7E and sse_a[1] == sse_4[1]
+
+
+# ------------------------------------------------------------------------------------------------
+# Orderings the method implies (bitwise, per block)
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("g", [1.0, 0.004])
+def test_brute_le_four_over_six_le_absmax(fmt, g):
+    x = _tiny_blocks(400 + fmt, 96, 8)
+    for pz in (0, 1):
+        _, _, s_abs = orc.quantize(x, 8, fmt, orc.ABSMAX + pz, g)
+        _, _, s_46 = orc.quantize(x, 8, fmt, orc.R4O6 + pz, g)
+        _, _, s_bf = orc.quantize(x, 8, fmt, orc.BRUTE + pz, g)
+        assert np.all(s_bf <= s_46) and np.all(s_46 <= s_abs)
+    assert np.any(s_bf < s_46) and np.any(s_46 < s_abs)
+
+
+@pytest.mark.parametrize("fmt", [orc.UE4M3, orc.UE5M3])
+def test_prevent_zero_never_hurts_and_only_touches_zero_scales(fmt):
+    x = _tiny_blocks(500 + fmt, 256, 4) * f32(2.0 ** -8 if fmt == orc.UE4M3 else 2.0 ** -16)
+    for base in (orc.ABSMAX, orc.R4O6, orc.BRUTE):
+        c0, s0, e0 = orc.quantize(x, 4, fmt, base)
+        c1, s1, e1 = orc.quantize(x, 4, fmt, base + 1)
+        assert np.all(e1 <= e0)
+        if base != orc.BRUTE:
+            touched = s0 != s1
+            assert np.any(touched) and np.all(s0[touched] == 0) and np.all(s1[touched] == 1)
+            # for 4-over-6 a clamp can change which candidate wins; abs-max blocks are untouched
+            if base == orc.ABSMAX:
+                assert np.array_equal(e0[~touched], e1[~touched])
+                assert np.array_equal(c0.reshape(-1, 2)[~touched], c1.reshape(-1, 2)[~touched])
+    _, s8, _ = orc.quantize(x, 4, orc.UE8M0, orc.ABSMAX)
+    _, s8p, _ = orc.quantize(x, 4, orc.UE8M0, orc.ABSMAX_PZ)
+    assert np.array_equal(s8, s8p)  # every UE8M0 code is nonzero: the clamp is a no-op
+
+
+def test_finer_is_better_for_the_brute_force_optimum():
+    # Children may reuse the parent's scale, so the optimum cannot get worse when a block is split
+    # (Results: "the optimal MSE monotonically increases with larger block sizes").
+    for seed, sigma in ((1, 0.004), (2, 0.02), (3, 1.0)):
+        x = inputs.normal(2048, seed, sigma).numpy()
+        prev = None
+        for B in (2, 4, 8, 16, 32, 64):
+            _, _, sse = orc.quantize(x, B, orc.UE4M3, orc.BRUTE)
+            if prev is not None:
+                parent = sse.astype(np.float64)
+                kids = prev.astype(np.float64).reshape(-1, 2).sum(1)
+                assert np.all(kids <= parent * (1 + 1e-6) + 1e-30)
+            prev = sse
+    # the same statement is allowed to fail for plain abs-max: that is the paradox being studied
+    x = inputs.normal(1 << 14, 7, 0.0035).numpy()
+    mse = {B: orc.tensor_mse(orc.quantize(x, B, orc.UE4M3, orc.ABSMAX)[2], x.size) for B in (4, 32)}
+    assert mse[4] > mse[32]
+
+
+def test_wider_scale_format_is_never_worse_for_brute_force():
+    x = _tiny_blocks(600, 64, 8)
+    _, _, s4 = orc.quantize(x, 8, orc.UE4M3, orc.BRUTE)
+    _, _, s5 = orc.quantize(x, 8, orc.UE5M3, orc.BRUTE)
+    assert np.all(s5 <= s4)
+
+
+def test_tiny_sigma_collapses_to_zero_scale():
+    # Region A: sigma = 0.0005, block 4, E4M3 abs-max -> scale 0 nearly always -> MSE ~ E[v^2]
+    x = inputs.normal(4 * 50000, 9, 0.0005).numpy()
+    _, scales, sse = orc.quantize(x, 4, orc.UE4M3, orc.ABSMAX)
+    zero = scales == 0
+    assert zero.mean() > 0.99
+    assert np.allclose(sse[zero], (x.reshape(-1, 4)[zero].astype(np.float64) ** 2).sum(1), rtol=1e-5)
+    assert abs(orc.tensor_mse(sse, x.size) / np.mean(x.astype(np.float64) ** 2) - 1) < 0.02
+
+
+# ------------------------------------------------------------------------------------------------
+# Symmetries
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("recipe", RECIPES)
+def test_sign_flip_only_flips_sign_bits(recipe):
+    x = _tiny_blocks(700, 48, 8)
+    c0, s0, e0 = orc.quantize(x, 8, orc.UE4M3, recipe)
+    c1, s1, e1 = orc.quantize(-x, 8, orc.UE4M3, recipe)
+    assert np.array_equal(s0, s1) and np.array_equal(e0, e1) and np.array_equal(c0 ^ 0x88, c1)
+
+
+@pytest.mark.parametrize("recipe", [orc.ABSMAX, orc.R4O6, orc.BRUTE])
+def test_power_of_two_input_scaling_shifts_scale_codes(recipe):
+    x = inputs.normal(512, 21).numpy()          # block scales well inside the normal range
+    k = 3
+    c0, s0, e0 = orc.quantize(x, 16, orc.UE4M3, recipe)
+    c1, s1, e1 = orc.quantize(x * f32(2.0 ** k), 16, orc.UE4M3, recipe)
+    assert s0.min() >= 8 and s1.max() < 0x7E
+    if recipe == orc.BRUTE:   # candidates below/above the shifted window exist on one side only
+        same = (s0 > 16) & (s1 < 0x70)
+    else:
+        same = np.ones_like(s0, dtype=bool)
+    assert same.mean() > 0.9
+    assert np.array_equal(s1[same], s0[same] + 8 * k)
+    assert np.array_equal(c1.reshape(-1, 8)[same], c0.reshape(-1, 8)[same])
+    assert np.array_equal(e1[same], e0[same] * f32(4.0 ** k))
+    # the tensor scale g plays the same role: scaling x and g together changes nothing
+    c2, s2, e2 = orc.quantize(x * f32(2.0 ** k), 16, orc.UE4M3, recipe, g=2.0 ** k)
+    assert np.array_equal(s2, s0) and np.array_equal(c2, c0)
+
+
+# ------------------------------------------------------------------------------------------------
+# Whole-tensor plumbing
+# ------------------------------------------------------------------------------------------------
+def test_tensor_mse_is_exact_sum_over_n():
+    rng = np.random.default_rng(8)
+    sse = (rng.random(1000) * np.exp2(rng.integers(-20, 5, 1000))).astype(f32)
+    exact = sum((ex.frac(s) for s in sse), F(0)) / 16000
+    assert abs(F(orc.tensor_mse(sse, 16000)) / exact - 1) < F(1, 10 ** 12)
+
+
+def test_tensor_amax_and_global_scale():
+    x = inputs.normal(4096, 1).numpy()
+    assert orc.tensor_amax(x) == np.abs(x).max()
+    assert orc.tensor_amax(-x) == np.abs(x).max()
+    assert orc.global_scale_from_amax(f32(2688.0)) == 1.0
+    assert orc.global_scale_from_amax(f32(0)) == 1.0
+
+
+def test_bf16_input_equals_widened_fp32_input():
+    xb = inputs.student_t(2048, 5, 0.02, 2)
+    bits = inputs.to_numpy_bits(xb)
+    wide = xb.to(torch.float32).numpy()
+    assert np.array_equal(bits.view(ml_dtypes.bfloat16).astype(f32), wide)  # widening is exact
+    for r in (orc.ABSMAX, orc.R4O6_PZ, orc.BRUTE):
+        a = orc.quantize(bits, 16, orc.UE4M3, r)
+        b = orc.quantize(wide, 16, orc.UE4M3, r)
+        assert all(np.array_equal(p, q) for p, q in zip(a, b))
+
+
+def test_threads_do_not_change_results():
+    x = _tiny_blocks(800, 333, 8)
+    for r in (orc.ABSMAX_PZ, orc.R4O6, orc.BRUTE):
+        a = orc.quantize(x, 8, orc.UE5M3, r, 0.5)
+        b = orc.quantize(x, 8, orc.UE5M3, r, 0.5, threads=5)
+        assert all(np.array_equal(p, q) for p, q in zip(a, b))
+
+
+@pytest.mark.parametrize("fmt,g", [(orc.UE4M3, 1.0), (orc.UE5M3, 0.37), (orc.UE8M0, 1.0)])
+def test_dequantize_multiplies_by_the_decode_scale(fmt, g):
+    x = _tiny_blocks(900 + fmt, 32, 16)
+    codes, scales, _ = orc.quantize(x, 16, fmt, orc.ABSMAX, g)
+    xh = orc.dequantize(codes, scales, x.size, 16, fmt, g)
+    c4 = _unpack(codes)
+    grid = ex.e2m1_magnitudes()
+    tab = ex.TABLES[fmt]()
+    for i in range(x.size):
+        D = ex.f32_mul(f32(tab[int(scales[i // 16])]), f32(g))
+        q = grid[c4[i] & 7] * (-1 if c4[i] & 8 else 1)
+        assert xh[i] == ex.f32_mul(f32(q), D)
+    xb = orc.dequantize(codes, scales, x.size, 16, fmt, g, orc.BF16)
+    assert np.array_equal(xb, xh.astype(ml_dtypes.bfloat16).view(np.uint16))
+
+
+def test_bad_arguments_are_rejected():
+    x = np.zeros(32, dtype=f32)
+    for kw in (dict(block_size=3), dict(block_size=128), dict(fmt=9), dict(recipe=9), dict(g=0.0), dict(g=float("inf"))):
+        a = dict(block_size=16, fmt=orc.UE4M3, recipe=orc.ABSMAX, g=1.0)
+        a.update(kw)
+        with pytest.raises(ValueError):
+            orc.quantize(x, a["block_size"], a["fmt"], a["recipe"], a["g"])
+    with pytest.raises(ValueError):
+        orc.quantize(np.zeros(30, dtype=f32), 16, orc.UE4M3, orc.ABSMAX)
+
+
+def test_values_exactly_on_a_midpoint_use_a_correctly_rounded_quotient():
+    # v = midpoint * S is exact in float32 for 4-bit-mantissa scales, so v / S must come out as the
+    # midpoint itself and tie to the even index.  Multiplying by a rounded reciprocal of S instead
+    # of dividing misses many of these.
+    mids = {0.25: 0, 0.75: 2, 1.25: 2, 1.75: 4, 2.5: 4, 3.5: 6, 5.0: 6}
+    for fmt, codes in ((orc.UE4M3, range(1, 0x7F)), (orc.UE5M3, range(1, 0xFF, 3))):
+        for c in codes:
+            S = f32(orc.scale_value(fmt, c))
+            v = np.array([f32(m) * S for m in mids] + [-f32(m) * S for m in mids], dtype=f32)
+            assert all(abs(ex.frac(x)) == F(m) * ex.frac(S) for x, m in zip(v, list(mids) * 2))
+            _, c4 = orc.block_sse(v, fmt, c)
+            assert list(c4 & 7) == list(mids.values()) * 2, (fmt, c)
+            assert list(c4 >> 3) == [0] * 7 + [1] * 7
