@@ -1,0 +1,152 @@
+/*
+ * mxq.h -- C-ABI of libmxq: block-wise microscaled FP4 (E2M1) quantization of whole tensors with
+ * per-block scale selection, scored by per-block SSE and per-tensor MSE, on one NVIDIA B200
+ * (sm_100a).  Implements the quantization recipes studied in "Finer is Better (with the Right
+ * Scaling)": MX power-of-two scales (Eq. 1), abs-max rounded to an FP8 scale format (Eq. 2), the
+ * prevent-zero clamp (Eq. 3), 4-over-6 (Eq. 4), hierarchical tensor + block scaling and the
+ * brute-force search over every scale code (Experimental Setup).
+ *
+ * Conventions for every entry point
+ *   - Pointers named d_* or documented "device" are DEVICE pointers owned by the caller.  The
+ *     library never allocates, frees or keeps them.  All device buffers must be 16-byte aligned.
+ *   - Calls validate their arguments on the host, enqueue kernels on `cuda_stream` (a
+ *     cudaStream_t passed as void*; NULL = the default stream) and return without synchronising.
+ *     Nothing is launched when validation fails.
+ *   - Return value: MXQ_OK (0) or a positive mxq_status.  Nothing throws, aborts or prints.
+ *   - Results are deterministic from run to run (no floating-point atomics).
+ *   - Inputs must be finite.  NaN or Inf elements give unspecified (but memory-safe) outputs.
+ *
+ * Data layout
+ *   x            n elements, contiguous; a block is B consecutive elements of the flat array
+ *                (a row-major matrix whose row length is a multiple of B is blocked along rows).
+ *   out_codes    n/2 bytes; byte j holds element 2j in bits 0..3 and element 2j+1 in bits 4..7;
+ *                a 4-bit code is sign<<3 | index into {0, 0.5, 1, 1.5, 2, 3, 4, 6}
+ *                (Experimental Setup, FP4 value set); the sign bit is the sign bit of the input.
+ *   out_scales   n/B bytes, one scale code per block in the chosen scale format.
+ *   out_block_sse n/B floats: sum over the block of (x - dequantized x)^2, accumulated in
+ *                binary32 in element order with fused multiply-adds; may be NULL.
+ */
+#ifndef MXQ_H_
+#define MXQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MXQ_OK = 0,
+    MXQ_ERR_NULL = 1,      /* a required pointer is NULL */
+    MXQ_ERR_BAD_ENUM = 2,  /* dtype, scale_fmt or recipe out of range */
+    MXQ_ERR_BAD_SHAPE = 3, /* n == 0, n not a multiple of block_size, block_size not in {2,4,8,16,32,64},
+                              or n so small that n/2 is not an integer */
+    MXQ_ERR_ALIGN = 4,     /* a device pointer is not 16-byte aligned */
+    MXQ_ERR_BAD_SCALE = 5, /* global_scale is not finite or is <= 0 */
+    MXQ_ERR_WORKSPACE = 6, /* workspace NULL or smaller than required */
+    MXQ_ERR_CUDA = 7       /* a CUDA call failed; see mxq_last_cuda_error() */
+} mxq_status;
+
+typedef enum { MXQ_F32 = 0, MXQ_BF16 = 1 } mxq_dtype;
+
+/* Block-scale formats (Background).  UE8M0: 2^(code-127), codes 0..254.  UE4M3: E4M3 with the
+ * sign bit unused, bias 7, subnormals, smallest nonzero 2^-9, largest 448, codes 0..0x7E.
+ * UE5M3: 5 exponent + 3 mantissa bits, bias 15, subnormals, smallest nonzero 2^-17, largest
+ * 1.75*2^16, codes 0..0xFE (the paper names this format without defining it; this is the
+ * library's definition). */
+typedef enum { MXQ_SF_UE8M0 = 0, MXQ_SF_UE4M3 = 1, MXQ_SF_UE5M3 = 2 } mxq_scale_fmt;
+
+/* Scale-selection recipes (Experimental Setup).
+ *   ABSMAX     Eq. 2 with M = 6: code = Round_SF(amax / g / 6), round-to-nearest-even, clipped to
+ *              the largest finite code.  With MXQ_SF_UE8M0 the rule is Eq. 1 instead: the
+ *              largest power of two <= amax / g / 6.
+ *   *_PZ       Eq. 3: a scale that rounds to zero is replaced by the smallest nonzero scale
+ *              (code 1).  No effect for UE8M0, whose codes are all nonzero.
+ *   4O6        Eq. 4: candidates Round_SF(amax/g/6) and Round_SF(amax/g/4); the block is
+ *              quantized with both and the one with the smaller SSE is kept (tie: M = 6).
+ *   BRUTE      every finite scale code is tried (BRUTE_PZ: every code with a nonzero value);
+ *              smallest SSE wins, equal SSE keeps the smaller code.  A code whose decode scale
+ *              S*g is not a finite float is skipped.
+ * Hierarchical scaling is any recipe called with global_scale != 1. */
+typedef enum {
+    MXQ_ABSMAX = 0, MXQ_ABSMAX_PZ = 1, MXQ_4O6 = 2, MXQ_4O6_PZ = 3, MXQ_BRUTE = 4, MXQ_BRUTE_PZ = 5
+} mxq_recipe;
+
+/*
+ * mxq_quantize -- quantize a float32 tensor on the default stream (Experimental Setup: Eq. 2-4,
+ * "quant(v_i / S)", hierarchical scaling, brute-force search).
+ *   x             device, n floats.
+ *   n             element count, a positive multiple of block_size.
+ *   block_size    2, 4, 8, 16, 32 or 64.
+ *   scale_fmt     mxq_scale_fmt.         recipe   mxq_recipe.
+ *   global_scale  g > 0, finite: the per-tensor decode scale of hierarchical scaling; 1 = none.
+ *                 Block targets are found from amax/g; elements are divided by D = fl32(S*g).
+ *   out_codes, out_scales, out_block_sse   device outputs as described above (sse may be NULL).
+ * Per element: t = fl32(x / D), code = sign | RNE_E2M1(min(|t|, 6)); D = 0 gives magnitude 0.
+ */
+int mxq_quantize(const float* x, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,
+                 uint8_t* out_codes, uint8_t* out_scales, float* out_block_sse);
+
+/*
+ * mxq_quantize_ex -- as mxq_quantize, with an input dtype, an optional device-resident global
+ * scale and a stream.
+ *   x               device, n elements of `dtype` (MXQ_F32 or MXQ_BF16; bf16 is widened exactly).
+ *   d_global_scale  device pointer to one float holding g, or NULL.  When non-NULL it overrides
+ *                   `global_scale` and is read by the kernel at run time (no host
+ *                   synchronisation); it must hold a finite positive value when the kernel runs.
+ */
+int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe,
+                    float global_scale, const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales,
+                    float* out_block_sse, void* cuda_stream);
+
+/*
+ * mxq_tensor_amax -- first stage of hierarchical scaling (Experimental Setup, "a per-tensor scale
+ * is first identified using the abs-max across the entire tensor").
+ *   d_out_amax  device, one float: max_i |x_i| (0 for an all-zero tensor).
+ *   d_out_global_scale  device, one float, or NULL: receives g = amax / (6*448) computed in
+ *               binary32 (1 if amax == 0), ready to be passed as d_global_scale.
+ */
+int mxq_tensor_amax(const void* x, int dtype, size_t n, float* d_out_amax, float* d_out_global_scale,
+                    void* cuda_stream);
+
+/* Host helper: the same g = amax / 2688 in binary32 (1 if amax is 0 or not finite). */
+float mxq_global_scale_from_amax(float amax);
+
+/*
+ * mxq_tensor_mse -- tensor MSE = (sum of the block SSEs) / n (Eq. 4 text, "MSE(v, S)"; Results,
+ * numerical study), as a fixed-shape two-level tree in binary64: the same inputs always give the
+ * same bits.
+ *   d_block_sse     device, n_blocks floats.
+ *   n               element count the SSEs cover (the divisor).
+ *   d_out_mse       device, one double.
+ *   d_workspace     device scratch of at least mxq_tensor_mse_workspace_bytes(n_blocks) bytes;
+ *                   contents are overwritten; no need to clear it.
+ */
+size_t mxq_tensor_mse_workspace_bytes(size_t n_blocks);
+int mxq_tensor_mse(const float* d_block_sse, size_t n_blocks, size_t n, double* d_out_mse, void* d_workspace,
+                   size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * mxq_dequantize -- "de-quantization simply multiplies by S" (Experimental Setup):
+ * out_i = fl32(grid(code_i) * D_b), D_b = fl32(S_b * g); MXQ_BF16 output rounds that to bf16 (RNE).
+ *   d_codes  n/2 bytes;  d_scales  n/block_size bytes;  d_out  n elements of out_dtype.
+ * A scale byte that is not a finite code of the format decodes as NaN.
+ */
+int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
+                   float global_scale, void* d_out, int out_dtype, void* cuda_stream);
+
+/* Number of kernels the library has launched in this process (all entry points), for
+ * accounting in benchmarks. */
+unsigned long long mxq_launch_count(void);
+
+const char* mxq_status_string(int status);
+/* The cudaError_t (as int) behind the most recent MXQ_ERR_CUDA on this thread, else 0. */
+int mxq_last_cuda_error(void);
+/* major*10000 + minor*100 + patch */
+int mxq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXQ_H_ */

@@ -1,0 +1,163 @@
+// C-ABI entry points of libmxq: host-side argument validation and kernel dispatch.
+#include <atomic>
+#include <cmath>
+
+#include "../../include/mxq.h"
+#include "mxq_device.cuh"
+#include "mxq_internal.h"
+
+namespace mxq {
+
+static std::atomic<unsigned long long> g_launches{0};
+static thread_local int tl_cuda_error = 0;
+
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+int sm_count(int device) {
+    static int cached[kMaxDevices] = {0};
+    if (device < 0 || device >= kMaxDevices) return 1;
+    if (cached[device] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = 1;
+        cached[device] = n;
+    }
+    return cached[device];
+}
+
+static int cuda_fail(cudaError_t e) {
+    tl_cuda_error = (int)e;
+    return MXQ_ERR_CUDA;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool valid_block(int b) { return b == 2 || b == 4 || b == 8 || b == 16 || b == 32 || b == 64; }
+
+}  // namespace mxq
+
+using namespace mxq;
+
+extern "C" {
+
+int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,
+                    const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales, float* out_block_sse,
+                    void* cuda_stream) {
+    if (!x || !out_codes || !out_scales) return MXQ_ERR_NULL;
+    if (dtype != MXQ_F32 && dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
+    if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
+    if (recipe < MXQ_ABSMAX || recipe > MXQ_BRUTE_PZ) return MXQ_ERR_BAD_ENUM;
+    if (!valid_block(block_size) || n == 0 || n % (size_t)block_size != 0) return MXQ_ERR_BAD_SHAPE;
+    if (!d_global_scale && !(global_scale > 0.0f && std::isfinite(global_scale))) return MXQ_ERR_BAD_SCALE;
+    if (!aligned16(x) || !aligned16(out_codes) || !aligned16(out_scales) || !aligned16(out_block_sse) ||
+        (d_global_scale && (reinterpret_cast<uintptr_t>(d_global_scale) & 3u)))
+        return MXQ_ERR_ALIGN;
+
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    QuantArgs a;
+    a.x = x;
+    a.first_item = 0;
+    a.global_scale = d_global_scale ? 1.0f : global_scale;
+    a.d_global_scale = d_global_scale;
+    a.codes = out_codes;
+    a.scales = out_scales;
+    a.block_sse = out_block_sse;
+    a.prevent_zero = (recipe == MXQ_ABSMAX_PZ || recipe == MXQ_4O6_PZ || recipe == MXQ_BRUTE_PZ) ? 1 : 0;
+
+    cudaError_t err;
+    if (recipe == MXQ_BRUTE || recipe == MXQ_BRUTE_PZ) {
+        a.n_items = n / (size_t)block_size;
+        err = (dtype == MXQ_F32) ? launch_brute_f32(a, block_size, scale_fmt, s)
+                                 : launch_brute_bf16(a, block_size, scale_fmt, s);
+        return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+    }
+    const bool dual = (recipe == MXQ_4O6 || recipe == MXQ_4O6_PZ);
+    const size_t chunk = block_size < 8 ? 8 : (size_t)block_size;
+    a.n_items = n / chunk;
+    if (a.n_items > 0) {
+        err = (dtype == MXQ_F32) ? launch_quantize_f32(a, block_size, scale_fmt, dual, s)
+                                 : launch_quantize_bf16(a, block_size, scale_fmt, dual, s);
+        if (err != cudaSuccess) return cuda_fail(err);
+    }
+    const size_t rest = n - a.n_items * chunk;  // < 8 elements, block sizes 2 and 4 only
+    if (rest > 0) {
+        a.first_item = a.n_items * chunk / (size_t)block_size;
+        a.n_items = rest / (size_t)block_size;
+        err = launch_quantize_tail(a, dtype, block_size, scale_fmt, dual, s);
+        if (err != cudaSuccess) return cuda_fail(err);
+    }
+    return MXQ_OK;
+}
+
+int mxq_quantize(const float* x, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,
+                 uint8_t* out_codes, uint8_t* out_scales, float* out_block_sse) {
+    return mxq_quantize_ex(x, MXQ_F32, n, block_size, scale_fmt, recipe, global_scale, nullptr, out_codes, out_scales,
+                           out_block_sse, nullptr);
+}
+
+int mxq_tensor_amax(const void* x, int dtype, size_t n, float* d_out_amax, float* d_out_global_scale,
+                    void* cuda_stream) {
+    if (!x || !d_out_amax) return MXQ_ERR_NULL;
+    if (dtype != MXQ_F32 && dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
+    if (n == 0) return MXQ_ERR_BAD_SHAPE;
+    if (!aligned16(x) || (reinterpret_cast<uintptr_t>(d_out_amax) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_out_global_scale) & 3u))
+        return MXQ_ERR_ALIGN;
+    cudaError_t err = launch_tensor_amax(x, dtype, n, d_out_amax, d_out_global_scale, static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+float mxq_global_scale_from_amax(float amax) {
+    return (amax > 0.0f && std::isfinite(amax)) ? amax / 2688.0f : 1.0f;
+}
+
+size_t mxq_tensor_mse_workspace_bytes(size_t n_blocks) {
+    (void)n_blocks;
+    return (size_t)kMsePartials * sizeof(double);
+}
+
+int mxq_tensor_mse(const float* d_block_sse, size_t n_blocks, size_t n, double* d_out_mse, void* d_workspace,
+                   size_t workspace_bytes, void* cuda_stream) {
+    if (!d_block_sse || !d_out_mse) return MXQ_ERR_NULL;
+    if (n_blocks == 0 || n == 0) return MXQ_ERR_BAD_SHAPE;
+    if (!d_workspace || workspace_bytes < mxq_tensor_mse_workspace_bytes(n_blocks)) return MXQ_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(d_block_sse) & 3u) || (reinterpret_cast<uintptr_t>(d_out_mse) & 7u) ||
+        (reinterpret_cast<uintptr_t>(d_workspace) & 7u))
+        return MXQ_ERR_ALIGN;
+    cudaError_t err = launch_tensor_mse(d_block_sse, n_blocks, n, d_out_mse, static_cast<double*>(d_workspace),
+                                        static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
+                   float global_scale, void* d_out, int out_dtype, void* cuda_stream) {
+    if (!d_codes || !d_scales || !d_out) return MXQ_ERR_NULL;
+    if (out_dtype != MXQ_F32 && out_dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
+    if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
+    if (!valid_block(block_size) || n == 0 || n % (size_t)block_size != 0) return MXQ_ERR_BAD_SHAPE;
+    if (!(global_scale > 0.0f && std::isfinite(global_scale))) return MXQ_ERR_BAD_SCALE;
+    if (!aligned16(d_codes) || !aligned16(d_out)) return MXQ_ERR_ALIGN;
+    cudaError_t err = launch_dequantize(d_codes, d_scales, n, block_size, scale_fmt, global_scale, d_out, out_dtype,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+unsigned long long mxq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* mxq_status_string(int status) {
+    switch (status) {
+    case MXQ_OK: return "ok";
+    case MXQ_ERR_NULL: return "a required pointer is NULL";
+    case MXQ_ERR_BAD_ENUM: return "dtype, scale format or recipe out of range";
+    case MXQ_ERR_BAD_SHAPE: return "n must be a positive multiple of block_size, block_size in {2,4,8,16,32,64}";
+    case MXQ_ERR_ALIGN: return "device pointer not sufficiently aligned";
+    case MXQ_ERR_BAD_SCALE: return "global_scale must be finite and > 0";
+    case MXQ_ERR_WORKSPACE: return "workspace missing or too small";
+    case MXQ_ERR_CUDA: return "CUDA call failed (see mxq_last_cuda_error)";
+    default: return "unknown status";
+    }
+}
+
+int mxq_last_cuda_error(void) { return tl_cuda_error; }
+
+int mxq_version(void) { return 100; /* 0.1.0 */ }
+
+}  // extern "C"

@@ -1,0 +1,44 @@
+// Host-side declarations shared by the translation units of libmxq (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace mxq {
+
+constexpr int kMaxDevices = 64;
+
+// Arguments of the quantization kernels.  n_items counts what one thread owns per loop trip:
+// chunks of max(B, 8) elements for the one-pass kernels, blocks for the search and tail kernels.
+struct QuantArgs {
+    const void* x;
+    size_t n_items;
+    size_t first_item;            // tail kernel only: index of the first block it handles
+    float global_scale;
+    const float* d_global_scale;  // overrides global_scale when non-NULL
+    uint8_t* codes;
+    uint8_t* scales;
+    float* block_sse;             // may be NULL
+    int prevent_zero;
+};
+
+int sm_count(int device);
+void count_launch();
+
+cudaError_t launch_quantize_f32(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
+cudaError_t launch_quantize_bf16(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
+cudaError_t launch_brute_f32(const QuantArgs& a, int B, int fmt, cudaStream_t s);
+cudaError_t launch_brute_bf16(const QuantArgs& a, int B, int fmt, cudaStream_t s);
+// Scalar kernel for the few blocks that do not fill a whole chunk (abs-max and 4-over-6 only).
+cudaError_t launch_quantize_tail(const QuantArgs& a, int dtype, int B, int fmt, bool dual, cudaStream_t s);
+
+cudaError_t launch_tensor_amax(const void* x, int dtype, size_t n, float* d_amax, float* d_g, cudaStream_t s);
+cudaError_t launch_tensor_mse(const float* d_sse, size_t n_blocks, size_t n, double* d_out, double* d_partials,
+                              cudaStream_t s);
+cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n, int B, int fmt, float g, void* out,
+                              int out_dtype, cudaStream_t s);
+
+constexpr int kMsePartials = 1024;  // fixed first-level width of the MSE tree
+
+}  // namespace mxq

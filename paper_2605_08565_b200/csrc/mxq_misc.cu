@@ -1,0 +1,279 @@
+// Small kernels around the quantization pass: per-tensor abs-max (first stage of hierarchical
+// scaling), deterministic tensor MSE, de-quantization, and a scalar kernel for the few blocks
+// that do not fill a whole per-thread chunk.
+#include <cuda_bf16.h>
+
+#include "mxq_device.cuh"
+#include "mxq_internal.h"
+
+namespace mxq {
+
+// ------------------------------------------------------------------------------------------------
+// Tensor abs-max: max is exact and order-independent, so the cross-CTA step is an integer
+// atomicMax on the bit pattern of the non-negative result (deterministic).
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_max(float m) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    return m;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) k_tensor_amax(const void* x, size_t n, uint32_t* out_bits) {
+    constexpr int VEC = 16 / elem_bytes(DT);
+    const size_t n_vec = n / VEC;
+    const size_t stride = (size_t)gridDim.x * kThreads;
+    const uint4* p = static_cast<const uint4*>(x);
+    float m = 0.0f;
+    if constexpr (DT == kF32) {
+        float m0 = 0.f, m1 = 0.f, m2 = 0.f, m3 = 0.f;
+        for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec; i += stride) {
+            const uint4 w = __ldcs(p + i);
+            m0 = fmaxf(m0, fabsf(__uint_as_float(w.x)));
+            m1 = fmaxf(m1, fabsf(__uint_as_float(w.y)));
+            m2 = fmaxf(m2, fabsf(__uint_as_float(w.z)));
+            m3 = fmaxf(m3, fabsf(__uint_as_float(w.w)));
+        }
+        m = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+    } else {
+        // magnitudes of bf16 order like their 15-bit patterns: packed unsigned 16-bit max
+        uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+        for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec; i += stride) {
+            const uint4 w = __ldcs(p + i);
+            a0 = __vmaxu2(a0, w.x & 0x7FFF7FFFu);
+            a1 = __vmaxu2(a1, w.y & 0x7FFF7FFFu);
+            a2 = __vmaxu2(a2, w.z & 0x7FFF7FFFu);
+            a3 = __vmaxu2(a3, w.w & 0x7FFF7FFFu);
+        }
+        const uint32_t a = __vmaxu2(__vmaxu2(a0, a1), __vmaxu2(a2, a3));
+        m = fmaxf(__uint_as_float(a << 16), __uint_as_float(a & 0xFFFF0000u));
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)(n - n_vec * VEC)) {  // ragged end, scalar
+        const size_t i = n_vec * VEC + threadIdx.x;
+        float v;
+        if constexpr (DT == kF32) v = static_cast<const float*>(x)[i];
+        else v = __uint_as_float((uint32_t) static_cast<const uint16_t*>(x)[i] << 16);
+        m = fmaxf(m, fabsf(v));
+    }
+    __shared__ float warp_m[kThreads / 32];
+    m = warp_max(m);
+    if ((threadIdx.x & 31) == 0) warp_m[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        m = threadIdx.x < kThreads / 32 ? warp_m[threadIdx.x] : 0.0f;
+        m = warp_max(m);
+        if (threadIdx.x == 0) atomicMax(out_bits, __float_as_uint(m));
+    }
+}
+
+// g = amax / (6 * 448): the tensor maximum maps to the top of FP4 times the top of E4M3.
+__global__ void k_global_scale(const float* amax, float* g) {
+    const float a = *amax;
+    *g = (a > 0.0f && a <= 3.402823466e38f) ? __fdiv_rn(a, 2688.0f) : 1.0f;
+}
+
+cudaError_t launch_tensor_amax(const void* x, int dtype, size_t n, float* d_amax, float* d_g, cudaStream_t s) {
+    cudaError_t err = cudaMemsetAsync(d_amax, 0, sizeof(float), s);
+    if (err != cudaSuccess) return err;
+    int dev = 0;
+    err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    const size_t n_vec = n / (16 / elem_bytes(dtype));
+    size_t want = (n_vec + kThreads - 1) / kThreads;
+    if (want == 0) want = 1;
+    const size_t cap = (size_t)sm_count(dev) * 8;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    if (dtype == kF32) k_tensor_amax<kF32><<<grid, kThreads, 0, s>>>(x, n, reinterpret_cast<uint32_t*>(d_amax));
+    else k_tensor_amax<kBF16><<<grid, kThreads, 0, s>>>(x, n, reinterpret_cast<uint32_t*>(d_amax));
+    count_launch();
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    if (d_g) {
+        k_global_scale<<<1, 1, 0, s>>>(d_amax, d_g);
+        count_launch();
+        err = cudaGetLastError();
+    }
+    return err;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Tensor MSE: two-level tree of fixed shape in binary64.  Level 1: P = min(1024, ceil(nb/256))
+// CTAs, CTA p sums the contiguous slice [p*L, (p+1)*L), L = ceil(nb/P): thread t adds elements
+// t, t+256, ... in order, then a shared-memory halving tree.  Level 2: one CTA, halving tree over
+// the P partials, divided by n.
+// ------------------------------------------------------------------------------------------------
+template <int T>
+__device__ __forceinline__ double cta_tree_sum(double v, double* sh) {
+    sh[threadIdx.x] = v;
+    __syncthreads();
+#pragma unroll
+    for (int w = T / 2; w > 0; w >>= 1) {
+        if (threadIdx.x < w) sh[threadIdx.x] = __dadd_rn(sh[threadIdx.x], sh[threadIdx.x + w]);
+        __syncthreads();
+    }
+    return sh[0];
+}
+
+__global__ void __launch_bounds__(kThreads) k_mse_partial(const float* sse, size_t nb, size_t slice, double* partials) {
+    __shared__ double sh[kThreads];
+    const size_t lo = (size_t)blockIdx.x * slice;
+    const size_t hi = (lo + slice < nb) ? lo + slice : nb;
+    double acc = 0.0;
+    for (size_t i = lo + threadIdx.x; i < hi; i += kThreads) acc = __dadd_rn(acc, (double)__ldcs(sse + i));
+    const double total = cta_tree_sum<kThreads>(acc, sh);
+    if (threadIdx.x == 0) partials[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(kMsePartials) k_mse_final(const double* partials, int n_partials, double n, double* out) {
+    __shared__ double sh[kMsePartials];
+    const double v = (int)threadIdx.x < n_partials ? partials[threadIdx.x] : 0.0;
+    const double total = cta_tree_sum<kMsePartials>(v, sh);
+    if (threadIdx.x == 0) *out = __ddiv_rn(total, n);
+}
+
+cudaError_t launch_tensor_mse(const float* d_sse, size_t n_blocks, size_t n, double* d_out, double* d_partials,
+                              cudaStream_t s) {
+    size_t P = (n_blocks + kThreads - 1) / kThreads;
+    if (P > (size_t)kMsePartials) P = kMsePartials;
+    const size_t slice = (n_blocks + P - 1) / P;
+    k_mse_partial<<<(unsigned)P, kThreads, 0, s>>>(d_sse, n_blocks, slice, d_partials);
+    count_launch();
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    k_mse_final<<<1, kMsePartials, 0, s>>>(d_partials, (int)P, (double)n, d_out);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// De-quantization: x_hat = fl32(grid(code) * D), D = fl32(S * g).  One thread per 8 elements.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float decode_scale(int fmt, int c, float g) {
+    if (c >= num_codes(fmt)) return __uint_as_float(0x7FC00000u);
+    return __fmul_rn(scale_value(fmt, c), g);
+}
+
+template <int ODT>
+__global__ void __launch_bounds__(kThreads) k_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n,
+                                                         int log2B, int fmt, float g, void* out) {
+    const size_t n8 = n >> 3;
+    const size_t stride = (size_t)gridDim.x * kThreads;
+    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n8; i += stride) {
+        const uint32_t w = __ldcs(reinterpret_cast<const uint32_t*>(codes) + i);
+        float q[8];
+        unpack_e2m1x8(w, q);
+        float xh[8];
+        if (log2B >= 3) {
+            const float D = decode_scale(fmt, scales[(i << 3) >> log2B], g);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) xh[k] = __fmul_rn(q[k], D);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) xh[k] = __fmul_rn(q[k], decode_scale(fmt, scales[((i << 3) + k) >> log2B], g));
+        }
+        if constexpr (ODT == kF32) {
+            float4* o = static_cast<float4*>(out) + 2 * i;
+            __stcs(o, make_float4(xh[0], xh[1], xh[2], xh[3]));
+            __stcs(o + 1, make_float4(xh[4], xh[5], xh[6], xh[7]));
+        } else {
+            uint32_t h[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const __nv_bfloat162 b = __floats2bfloat162_rn(xh[2 * k], xh[2 * k + 1]);
+                h[k] = *reinterpret_cast<const uint32_t*>(&b);
+            }
+            __stcs(static_cast<uint4*>(out) + i, make_uint4(h[0], h[1], h[2], h[3]));
+        }
+    }
+    // ragged end (n not a multiple of 8; only possible for block sizes 2 and 4)
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)(n - (n8 << 3))) {
+        const size_t e = (n8 << 3) + threadIdx.x;
+        const uint32_t c4 = (codes[e >> 1] >> ((e & 1) ? 4 : 0)) & 15u;
+        float q[8];
+        unpack_e2m1x8(c4, q);
+        const float xh = __fmul_rn(q[0], decode_scale(fmt, scales[e >> log2B], g));
+        if constexpr (ODT == kF32) static_cast<float*>(out)[e] = xh;
+        else static_cast<__nv_bfloat16*>(out)[e] = __float2bfloat16_rn(xh);
+    }
+}
+
+cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n, int B, int fmt, float g, void* out,
+                              int out_dtype, cudaStream_t s) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    int log2B = 0;
+    while ((1 << log2B) < B) ++log2B;
+    size_t want = ((n >> 3) + kThreads - 1) / kThreads;
+    if (want == 0) want = 1;
+    const size_t cap = (size_t)sm_count(dev) * 8;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    if (out_dtype == kF32) k_dequantize<kF32><<<grid, kThreads, 0, s>>>(codes, scales, n, log2B, fmt, g, out);
+    else k_dequantize<kBF16><<<grid, kThreads, 0, s>>>(codes, scales, n, log2B, fmt, g, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Scalar abs-max / 4-over-6 for the blocks past the last whole chunk (at most three blocks).
+// Same arithmetic as the one-pass kernels, general quotient only.
+// ------------------------------------------------------------------------------------------------
+template <int FMT>
+__device__ float tail_eval(const float* v, int B, int c, float g, uint8_t* codes_out) {
+    const float D = __fmul_rn(scale_value(FMT, c), g);
+    float s = 0.0f;
+    for (int i = 0; i < B; i += 2) {
+        const float t0 = quotient_general(v[i], D), t1 = quotient_general(v[i + 1], D);
+        if (codes_out) codes_out[i >> 1] = (uint8_t)pack_e2m1x2(t0, t1);
+        const float2 q = round_e2m1x2(t0, t1);
+        const float e0 = __fmaf_rn(-q.x, D, v[i]);
+        s = __fmaf_rn(e0, e0, s);
+        const float e1 = __fmaf_rn(-q.y, D, v[i + 1]);
+        s = __fmaf_rn(e1, e1, s);
+    }
+    return s;
+}
+
+template <int FMT>
+__global__ void k_quantize_tail(QuantArgs p, int dtype, int B, int dual) {
+    const size_t b = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= p.n_items) return;
+    const size_t blk = p.first_item + b;
+    const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
+    float v[8];
+    float amax = 0.0f;
+    for (int i = 0; i < B; ++i) {
+        const size_t e = blk * B + i;
+        v[i] = dtype == kF32 ? static_cast<const float*>(p.x)[e]
+                             : __uint_as_float((uint32_t) static_cast<const uint16_t*>(p.x)[e] << 16);
+        amax = fmaxf(amax, fabsf(v[i]));
+    }
+    const bool pz = p.prevent_zero && FMT != kUE8M0;
+    const float u = __fdiv_rn(amax, g);
+    int c = round_scale<FMT>(__fdiv_rn(u, 6.0f));
+    if (pz) c = max(c, 1);
+    float s = tail_eval<FMT>(v, B, c, g, nullptr);
+    if (dual) {
+        int c4 = round_scale<FMT>(__fdiv_rn(u, 4.0f));
+        if (pz) c4 = max(c4, 1);
+        const float s4 = tail_eval<FMT>(v, B, c4, g, nullptr);
+        if (s4 < s) { s = s4; c = c4; }
+    }
+    tail_eval<FMT>(v, B, c, g, p.codes + blk * (B / 2));
+    p.scales[blk] = (uint8_t)c;
+    if (p.block_sse) p.block_sse[blk] = s;
+}
+
+cudaError_t launch_quantize_tail(const QuantArgs& a, int dtype, int B, int fmt, bool dual, cudaStream_t s) {
+    if (B > 8) return cudaErrorInvalidValue;
+    const unsigned grid = (unsigned)((a.n_items + 31) / 32);
+    switch (fmt) {
+    case kUE8M0: k_quantize_tail<kUE8M0><<<grid, 32, 0, s>>>(a, dtype, B, dual ? 1 : 0); break;
+    case kUE4M3: k_quantize_tail<kUE4M3><<<grid, 32, 0, s>>>(a, dtype, B, dual ? 1 : 0); break;
+    default: k_quantize_tail<kUE5M3><<<grid, 32, 0, s>>>(a, dtype, B, dual ? 1 : 0); break;
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace mxq

@@ -1,0 +1,208 @@
+"""GPU parity: the CUDA library, called through its C-ABI binding, against the CPU oracle on the
+same seeded inputs.  Codes, scale bytes and block SSE must be bit-identical; tensor MSE within 1e-6
+relative (binary64 sums in a different order)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mxq_oracle as orc
+from paper_2605_08565_b200 import binding as mxq
+from paper_2605_08565_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+FMTS = [mxq.MXQ_SF_UE8M0, mxq.MXQ_SF_UE4M3, mxq.MXQ_SF_UE5M3]
+RECIPES = [mxq.MXQ_ABSMAX, mxq.MXQ_ABSMAX_PZ, mxq.MXQ_4O6, mxq.MXQ_4O6_PZ, mxq.MXQ_BRUTE, mxq.MXQ_BRUTE_PZ]
+BLOCKS = [2, 4, 8, 16, 32, 64]
+MSE_RTOL = 1e-6
+
+
+def _mixed(n, seed, dtype):
+    """Normals at several magnitudes interleaved with tie-prone / zero / denormal / huge runs."""
+    a = inputs.adversarial(n, seed, torch.float32)
+    b = inputs.normal(n, seed + 1, 1.0, torch.float32) * torch.exp2(torch.randint(-14, 8, (n // 64 + 1,), generator=torch.Generator().manual_seed(seed)).float()).repeat_interleave(64)[:n]
+    pick = (torch.arange(n) // 64) % 3 == 0
+    return torch.where(pick, a, b).to(dtype).contiguous()
+
+
+def gpu_quantize(x_cpu, B, fmt, recipe, g=1.0, device_g=False):
+    x = x_cpu.cuda()
+    dg = torch.tensor([g], dtype=torch.float32, device="cuda") if device_g else None
+    codes, scales, sse = mxq.quantize(x, B, fmt, recipe, 1.0 if device_g else g, dg)
+    mse = mxq.tensor_mse(sse, x.numel())
+    torch.cuda.synchronize()
+    return codes.cpu().numpy(), scales.cpu().numpy(), sse.cpu().numpy(), float(mse.cpu()[0])
+
+
+def check_parity(x_cpu, B, fmt, recipe, g=1.0, device_g=False):
+    gc, gs, ge, gm = gpu_quantize(x_cpu, B, fmt, recipe, g, device_g)
+    oc, os_, oe = orc.quantize(inputs.to_numpy_bits(x_cpu), B, fmt, recipe, g, threads=8)
+    bad = np.flatnonzero(gs != os_)
+    assert bad.size == 0, f"scale bytes differ at blocks {bad[:8]} gpu={gs[bad[:8]]} oracle={os_[bad[:8]]}"
+    bad = np.flatnonzero(gc != oc)
+    assert bad.size == 0, f"code bytes differ at {bad[:8]} gpu={gc[bad[:8]]} oracle={oc[bad[:8]]}"
+    bad = np.flatnonzero(ge.view(np.uint32) != oe.view(np.uint32))
+    assert bad.size == 0, f"block SSE differs at {bad[:8]} gpu={ge[bad[:8]]} oracle={oe[bad[:8]]}"
+    om = orc.tensor_mse(oe, x_cpu.numel())
+    assert abs(gm - om) <= MSE_RTOL * abs(om) + 1e-300, (gm, om)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", BLOCKS)
+@pytest.mark.parametrize("fmt", FMTS)
+def test_one_pass_recipes_bit_exact(dtype, B, fmt):
+    # several CTAs' worth of chunks plus a ragged end (not a multiple of 8 for the small blocks)
+    n = 3 * 256 * max(B, 8) + 5 * 64 + (B if B < 8 else 0)
+    x = _mixed(n, 10 + B + fmt, dtype)
+    for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_ABSMAX_PZ, mxq.MXQ_4O6, mxq.MXQ_4O6_PZ):
+        check_parity(x, B, fmt, recipe, 1.0)
+        check_parity(x, B, fmt, recipe, 0.0131)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", BLOCKS)
+@pytest.mark.parametrize("fmt", FMTS)
+def test_brute_force_bit_exact(dtype, B, fmt):
+    n = 2 * 256 * B + 7 * B
+    x = _mixed(n, 40 + B + fmt, dtype)
+    check_parity(x, B, fmt, mxq.MXQ_BRUTE, 1.0)
+    check_parity(x, B, fmt, mxq.MXQ_BRUTE_PZ, 0.0131)
+
+
+@pytest.mark.parametrize("recipe", RECIPES)
+def test_extreme_global_scales(recipe):
+    x = _mixed(4096, 77, torch.float32)
+    for g in (2.0 ** -30, 2.0 ** 20, 3.0e-37, 1.0e30):
+        check_parity(x, 16, mxq.MXQ_SF_UE4M3, recipe, g)
+    check_parity(x, 8, mxq.MXQ_SF_UE8M0, recipe, 2.0 ** -100)
+    check_parity(x, 8, mxq.MXQ_SF_UE8M0, recipe, 2.0 ** 100)
+    check_parity(x, 8, mxq.MXQ_SF_UE5M3, recipe, 5.0e-33)
+
+
+def test_device_resident_global_scale_matches_host_scale():
+    x = _mixed(8192, 5, torch.bfloat16)
+    for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_4O6, mxq.MXQ_BRUTE):
+        check_parity(x, 16, mxq.MXQ_SF_UE4M3, recipe, 0.0421, device_g=True)
+
+
+def test_all_zero_and_single_block_tensors():
+    for B in BLOCKS:
+        z = torch.zeros(B, dtype=torch.float32)
+        for fmt in FMTS:
+            for recipe in RECIPES:
+                check_parity(z, B, fmt, recipe)
+        one = inputs.normal(B, B, 0.3)
+        check_parity(one, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6)
+        check_parity(one, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_BRUTE)
+
+
+def test_fp4_rounding_boundaries_through_the_kernel():
+    # a block whose maximum is 6*S makes the block scale exactly S, so every other element v
+    # is divided by S: sweep v across all seven rounding midpoints and one float either side
+    S = 0.40625  # 1.625 * 2^-2, a UE4M3 value
+    mids = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0], dtype=np.float32) * np.float32(S)
+    pts = np.concatenate([np.nextafter(mids, 0), mids, np.nextafter(mids, np.float32(10))]).astype(np.float32)
+    pts = np.concatenate([pts, -pts, [0.0, -0.0, 1e-30, -1e-30, 1e-45, -1e-45]]).astype(np.float32)
+    blocks = []
+    for i in range(0, len(pts), 15):
+        chunk = list(pts[i:i + 15])
+        chunk += [0.0] * (15 - len(chunk))
+        blocks.append(chunk + [6 * S])
+    x = torch.tensor(np.array(blocks, dtype=np.float32).reshape(-1))
+    check_parity(x, 16, mxq.MXQ_SF_UE4M3, mxq.MXQ_ABSMAX)
+    check_parity(x, 16, mxq.MXQ_SF_UE5M3, mxq.MXQ_ABSMAX)
+
+
+# ------------------------------------------------------------------------------------------------
+# Workload-shaped cases (small versions of the benchmark configurations)
+# ------------------------------------------------------------------------------------------------
+def test_config_normal_1024x1024_fp32_hierarchical():
+    x = inputs.normal(1024 * 1024, 1, 1.0, torch.float32)
+    xg = x.cuda()
+    amax = torch.empty(1, dtype=torch.float32, device="cuda")
+    dg = torch.empty(1, dtype=torch.float32, device="cuda")
+    mxq.mxq_tensor_amax(xg, xg.numel(), amax, dg)
+    torch.cuda.synchronize()
+    o_amax = orc.tensor_amax(x.numpy())
+    assert float(amax.cpu()[0]) == float(o_amax)
+    g = float(orc.global_scale_from_amax(o_amax))
+    assert float(dg.cpu()[0]) == g == mxq.mxq_global_scale_from_amax(float(o_amax))
+    for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_4O6, mxq.MXQ_BRUTE):
+        check_parity(x, 16, mxq.MXQ_SF_UE4M3, recipe, g, device_g=True)
+
+
+@pytest.mark.parametrize("B", BLOCKS)
+def test_config_weight_student_t_bf16(B):
+    x = inputs.student_t(512 * 1024, 5, 0.02, 2, torch.bfloat16)
+    for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_ABSMAX_PZ):
+        check_parity(x, B, mxq.MXQ_SF_UE4M3, recipe)
+    check_parity(x[: 64 * 1024], B, mxq.MXQ_SF_UE4M3, mxq.MXQ_BRUTE)
+
+
+def test_config_activation_outlier_columns_bf16():
+    x = inputs.outlier_columns(256, 4096, 3, dtype=torch.bfloat16)
+    g = float(orc.global_scale_from_amax(orc.tensor_amax(inputs.to_numpy_bits(x))))
+    for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_4O6):
+        check_parity(x, 16, mxq.MXQ_SF_UE4M3, recipe, g)
+        check_parity(x, 16, mxq.MXQ_SF_UE5M3, recipe, 1.0)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_config_laplace_fp32_brute_force_with_tensor_scale(fmt):
+    x = inputs.laplace(96 * 1024, 5, torch.float32)
+    g = float(orc.global_scale_from_amax(orc.tensor_amax(x.numpy())))
+    for B in (2, 4, 8, 16, 32):
+        check_parity(x[: 1024 * B], B, fmt, mxq.MXQ_BRUTE, g)
+
+
+# ------------------------------------------------------------------------------------------------
+# The smaller entry points
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_tensor_amax(dtype):
+    for n in (1, 7, 8, 1000, 256 * 1024 + 3):
+        x = _mixed(max(n, 64), n, dtype)[:n].contiguous()
+        xg = x.cuda()
+        out = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+        mxq.mxq_tensor_amax(xg, n, out)
+        torch.cuda.synchronize()
+        assert float(out.cpu()[0]) == float(orc.tensor_amax(inputs.to_numpy_bits(x)))
+
+
+def test_tensor_mse_is_deterministic_and_accurate():
+    rng = np.random.default_rng(3)
+    for nb in (1, 255, 256, 257, 100_000, 1024 * 256 + 17):
+        sse = (rng.random(nb) * np.exp2(rng.integers(-30, 4, nb))).astype(np.float32)
+        d = torch.from_numpy(sse).cuda()
+        a = float(mxq.tensor_mse(d, nb * 16).cpu()[0])
+        b = float(mxq.tensor_mse(d, nb * 16).cpu()[0])
+        want = orc.tensor_mse(sse, nb * 16)
+        assert a == b
+        assert abs(a - want) <= 1e-12 * want
+
+
+@pytest.mark.parametrize("fmt,g", [(mxq.MXQ_SF_UE4M3, 1.0), (mxq.MXQ_SF_UE5M3, 0.37), (mxq.MXQ_SF_UE8M0, 1.0)])
+@pytest.mark.parametrize("B", [2, 4, 16, 64])
+def test_dequantize(fmt, g, B):
+    n = 256 * 64 * 2 + (B if B < 8 else 0)
+    x = _mixed(n, 90 + B, torch.float32)
+    codes, scales, _ = orc.quantize(x.numpy(), B, fmt, mxq.MXQ_ABSMAX, g)
+    dc, ds = torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda()
+    for odt, oid in ((torch.float32, orc.F32), (torch.bfloat16, orc.BF16)):
+        out = torch.empty(n, dtype=odt, device="cuda")
+        mxq.mxq_dequantize(dc, ds, n, B, fmt, g, out)
+        torch.cuda.synchronize()
+        want = orc.dequantize(codes, scales, n, B, fmt, g, oid)
+        got = inputs.to_numpy_bits(out)
+        assert np.array_equal(got.view(np.uint32 if odt == torch.float32 else np.uint16),
+                              want.view(np.uint32 if odt == torch.float32 else np.uint16))
+
+
+def test_sse_output_is_optional_and_launches_are_counted():
+    x = inputs.normal(4096, 1).cuda()
+    before = mxq.mxq_launch_count()
+    codes, scales, sse = mxq.quantize(x, 16, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6)
+    c2, s2, none = mxq.quantize(x, 16, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6, with_sse=False)
+    torch.cuda.synchronize()
+    assert none is None and torch.equal(codes, c2) and torch.equal(scales, s2)
+    assert mxq.mxq_launch_count() == before + 2
