@@ -47,10 +47,8 @@ __device__ __forceinline__ void encode_chunk(const float (&v)[C], const float (&
     float q[C];
 #pragma unroll
     for (int k = 0; k < C / 8; ++k) {
-        packed[k] = pack_e2m1x8(t[8 * k], t[8 * k + 1], t[8 * k + 2], t[8 * k + 3], t[8 * k + 4], t[8 * k + 5],
-                                t[8 * k + 6], t[8 * k + 7]);
         float q8[8];
-        unpack_e2m1x8(packed[k], q8);
+        packed[k] = quantize_e2m1x8(&t[8 * k], q8);
 #pragma unroll
         for (int i = 0; i < 8; ++i) q[8 * k + i] = q8[i];
     }
