@@ -356,13 +356,79 @@ def run_gpu(args) -> None:
     dist.shutdown()
 
 
+def run_single_kernel(args) -> None:
+    """Time one kernel alone (`--kernel`): used for sweeps and as the small case for ncu captures."""
+    import torch
+    from paper_2605_08565_b200 import binding as mxq
+    from paper_2605_08565_b200 import inputs
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    n = args.elems - args.elems % 64
+    dtype = torch.bfloat16 if args.dtype == "bf16" else torch.float32
+    fmt = {"ue8m0": 0, "ue4m3": 1, "ue5m3": 2}[args.fmt]
+    x = inputs.student_t(n, 5, 0.02, 2, dtype, dev) if args.dtype == "bf16" else inputs.laplace(n, 5, dtype, dev)
+    B = args.block
+    codes, scales, sse = mxq.alloc_outputs(n, B, dev)
+    g = args.global_scale
+    recipe = {"absmax": 0, "absmax_pz": 1, "4o6": 2, "4o6_pz": 3, "brute": 4, "brute_pz": 5}.get(args.kernel)
+    out = torch.empty(n, dtype=dtype, device=dev)
+    amax = torch.empty(1, dtype=torch.float32, device=dev)
+    mse = torch.empty(1, dtype=torch.float64, device=dev)
+    ws = torch.empty(mxq.mxq_tensor_mse_workspace_bytes(n // B) // 8, dtype=torch.float64, device=dev)
+    eb = x.element_size()
+    if recipe is not None:
+        fn = lambda: mxq.mxq_quantize_ex(x, n, B, fmt, recipe, g, None, codes, scales, sse)
+        nbytes = algorithmic_bytes(n, eb, B)
+    elif args.kernel == "amax":
+        fn = lambda: mxq.mxq_tensor_amax(x, n, amax)
+        nbytes = n * eb
+    elif args.kernel == "mse":
+        fn = lambda: mxq.mxq_tensor_mse(sse, n // B, n, mse, ws)
+        nbytes = 4.0 * n / B
+    elif args.kernel == "dequant":
+        mxq.mxq_quantize_ex(x, n, B, fmt, 0, g, None, codes, scales, sse)
+        fn = lambda: mxq.mxq_dequantize(codes, scales, n, B, fmt, g, out)
+        nbytes = n * (eb + 0.5 + 1.0 / B)
+    else:
+        raise SystemExit(f"unknown --kernel {args.kernel}")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if n * eb < (256 << 20) else None
+    for _ in range(3):
+        fn()
+    times = []
+    for _ in range(args.iters):
+        if flush is not None:
+            flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = statistics.median(times)
+    res = {"kernel": args.kernel, "block": B, "dtype": args.dtype, "fmt": args.fmt, "elems": n, "ms": ms,
+           "gelem_s": n / ms / 1e6, "algorithmic_gb_s": nbytes / ms / 1e6,
+           "l2": "flushed between iterations" if flush is not None else "input larger than L2"}
+    if recipe in (4, 5):
+        ncodes = 127 if fmt == 1 else 255
+        res["tlaneop_s"] = n * ncodes * 4.0 / (ms * 1e-3) / 1e12
+    print(json.dumps(res))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
+    ap.add_argument("--kernel", default=None, help="time one kernel alone: absmax|absmax_pz|4o6|4o6_pz|brute|brute_pz|amax|mse|dequant")
+    ap.add_argument("--block", type=int, default=16)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--fmt", default="ue4m3", choices=["ue8m0", "ue4m3", "ue5m3"])
+    ap.add_argument("--elems", type=int, default=1 << 27)
+    ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--global-scale", type=float, default=1.0)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="mxq", choices=["mxq", "reference"])
     args = ap.parse_args()
+    if args.kernel:
+        run_single_kernel(args)
+        return
     if args.warmup < 3 and args.impl == "mxq":
         args.warmup = 3
     if args.impl == "reference":
