@@ -45,7 +45,8 @@ typedef enum {
     MXQ_ERR_ALIGN = 4,     /* a device pointer is not 16-byte aligned */
     MXQ_ERR_BAD_SCALE = 5, /* global_scale is not finite or is <= 0 */
     MXQ_ERR_WORKSPACE = 6, /* workspace NULL or smaller than required */
-    MXQ_ERR_CUDA = 7       /* a CUDA call failed; see mxq_last_cuda_error() */
+    MXQ_ERR_CUDA = 7,      /* a CUDA call failed; see mxq_last_cuda_error() */
+    MXQ_ERR_TOO_LARGE = 8  /* the size exceeds the fixed capacity of an entry point that owns its scratch */
 } mxq_status;
 
 typedef enum { MXQ_F32 = 0, MXQ_BF16 = 1 } mxq_dtype;
@@ -126,6 +127,29 @@ float mxq_global_scale_from_amax(float amax);
 size_t mxq_tensor_mse_workspace_bytes(size_t n_blocks);
 int mxq_tensor_mse(const float* d_block_sse, size_t n_blocks, size_t n, double* d_out_mse, void* d_workspace,
                    size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * mxq_tensor_mse_static -- mxq_tensor_mse for callers that have no device memory to lend as a
+ * workspace and must not allocate any: for example a plug-in or operator that a serving runtime
+ * hands nothing but its input and output buffers, while the runtime's own pool has already
+ * reserved the rest of the GPU (a raw cudaMalloc there fails, or stalls the device while it
+ * synchronises), or a latency-bound loop in which an allocation is not acceptable.  The paper has
+ * no counterpart of this call; it computes exactly what mxq_tensor_mse computes (same kernels,
+ * same tree, same bits) and differs only in where the 1024 first-level partial sums live: in an
+ * 8 KiB array that is part of the library image, present on every GPU that loads the library
+ * until the process exits.  The call allocates nothing and frees nothing.
+ *   d_block_sse, n_blocks, n, d_out_mse, cuda_stream   as for mxq_tensor_mse (caller-owned).
+ *   n_blocks    at most MXQ_TENSOR_MSE_STATIC_MAX_BLOCKS; a larger count returns
+ *               MXQ_ERR_TOO_LARGE and launches nothing (use mxq_tensor_mse with a workspace).
+ * The first call on each device looks up the array's device address (the device must be current,
+ * as for every call); make that first call outside any stream capture.  All calls on a device
+ * share the one array and each overwrites what the previous one left; nothing needs clearing
+ * between calls.  Two calls whose kernels can overlap on the GPU (different streams, no ordering
+ * between them) race on the array and give undefined results: keep such calls on one stream or
+ * order them with events.
+ */
+#define MXQ_TENSOR_MSE_STATIC_MAX_BLOCKS ((size_t)1 << 31)
+int mxq_tensor_mse_static(const float* d_block_sse, size_t n_blocks, size_t n, double* d_out_mse, void* cuda_stream);
 
 /*
  * mxq_dequantize -- "de-quantization simply multiplies by S" (Experimental Setup):

@@ -20,7 +20,7 @@ MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ = range(
 
 EXPORTS = (
     "mxq_quantize", "mxq_quantize_ex", "mxq_tensor_amax", "mxq_global_scale_from_amax",
-    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_dequantize", "mxq_launch_count",
+    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_launch_count",
     "mxq_status_string", "mxq_last_cuda_error", "mxq_version",
 )
 
@@ -55,6 +55,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_tensor_mse_workspace_bytes.argtypes = [sz]
     L.mxq_tensor_mse.restype = i32
     L.mxq_tensor_mse.argtypes = [vp, sz, sz, vp, vp, sz, vp]
+    L.mxq_tensor_mse_static.restype = i32
+    L.mxq_tensor_mse_static.argtypes = [vp, sz, sz, vp, vp]
     L.mxq_dequantize.restype = i32
     L.mxq_dequantize.argtypes = [vp, vp, sz, i32, i32, f32, vp, i32, vp]
     L.mxq_launch_count.restype = c.c_ulonglong
@@ -134,6 +136,11 @@ def mxq_tensor_mse(d_block_sse, n_blocks, n, d_out_mse, d_workspace, stream=None
     ws_bytes = d_workspace.numel() * d_workspace.element_size() if d_workspace is not None else 0
     _check(load_library().mxq_tensor_mse(_ptr(d_block_sse), n_blocks, n, _ptr(d_out_mse), _ptr(d_workspace),
                                          ws_bytes, _stream(stream)))
+
+
+def mxq_tensor_mse_static(d_block_sse, n_blocks, n, d_out_mse, stream=None) -> None:
+    """Tensor MSE with the library's built-in scratch array: no workspace argument, nothing allocated."""
+    _check(load_library().mxq_tensor_mse_static(_ptr(d_block_sse), n_blocks, n, _ptr(d_out_mse), _stream(stream)))
 
 
 def mxq_dequantize(d_codes, d_scales, n, block_size, scale_fmt, global_scale, d_out, stream=None) -> None:

@@ -127,6 +127,17 @@ int mxq_tensor_mse(const float* d_block_sse, size_t n_blocks, size_t n, double* 
     return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
 }
 
+int mxq_tensor_mse_static(const float* d_block_sse, size_t n_blocks, size_t n, double* d_out_mse, void* cuda_stream) {
+    if (!d_block_sse || !d_out_mse) return MXQ_ERR_NULL;
+    if (n_blocks == 0 || n == 0) return MXQ_ERR_BAD_SHAPE;
+    if (n_blocks > MXQ_TENSOR_MSE_STATIC_MAX_BLOCKS) return MXQ_ERR_TOO_LARGE;
+    if ((reinterpret_cast<uintptr_t>(d_block_sse) & 3u) || (reinterpret_cast<uintptr_t>(d_out_mse) & 7u))
+        return MXQ_ERR_ALIGN;
+    cudaError_t err =
+        launch_tensor_mse_static(d_block_sse, n_blocks, n, d_out_mse, static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
 int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
                    float global_scale, void* d_out, int out_dtype, void* cuda_stream) {
     if (!d_codes || !d_scales || !d_out) return MXQ_ERR_NULL;
@@ -152,6 +163,7 @@ const char* mxq_status_string(int status) {
     case MXQ_ERR_BAD_SCALE: return "global_scale must be finite and > 0";
     case MXQ_ERR_WORKSPACE: return "workspace missing or too small";
     case MXQ_ERR_CUDA: return "CUDA call failed (see mxq_last_cuda_error)";
+    case MXQ_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this entry point (use the workspace variant)";
     default: return "unknown status";
     }
 }

@@ -3,6 +3,8 @@
 // that do not fill a whole per-thread chunk.
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "mxq_device.cuh"
 #include "mxq_internal.h"
 
@@ -274,6 +276,43 @@ cudaError_t launch_quantize_tail(const QuantArgs& a, int dtype, int B, int fmt, 
     }
     count_launch();
     return cudaGetLastError();
+}
+
+}  // namespace mxq
+
+// ------------------------------------------------------------------------------------------------
+// Tensor MSE for callers that cannot provide scratch memory: the first-level partial sums live in
+// a file-scope device array instead of a caller workspace.  Every GPU that loads the library
+// carries these 8 KiB until the process exits.  In host code the array's name is only a handle
+// for the runtime, so its device address is looked up once per device (with that device current)
+// and handed to the same two kernels as the workspace variant.  Nothing in the array has to start
+// at zero: the first kernel writes every partial the second one reads.
+// ------------------------------------------------------------------------------------------------
+namespace mxq {
+
+static __device__ __align__(256) double g_mse_static_partials[kMsePartials];
+
+cudaError_t launch_tensor_mse_static(const float* d_sse, size_t n_blocks, size_t n, double* d_out, cudaStream_t s) {
+    static std::mutex mu;
+    static double* scratch_of_device[kMaxDevices] = {nullptr};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    double* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        scratch = scratch_of_device[dev];
+        if (scratch == nullptr) {  // first call on this device: resolve the symbol to a device address
+            void* p = nullptr;
+            err = cudaGetSymbolAddress(&p, g_mse_static_partials);
+            if (err != cudaSuccess) return err;
+            if (p == nullptr) return cudaErrorInvalidSymbol;
+            scratch = static_cast<double*>(p);
+            scratch_of_device[dev] = scratch;
+        }
+    }
+    return launch_tensor_mse(d_sse, n_blocks, n, d_out, scratch, s);
 }
 
 }  // namespace mxq
