@@ -2,11 +2,31 @@
 // factors to minimize the MSE"): every finite scale code of the format is tried on every block and
 // the code with the smallest SSE is kept (equal SSE: the smaller code).
 //
-// One thread owns one block of B elements in registers.  The candidate loop is uniform across the
-// CTA, so the candidate's decode scale D and its reciprocal come from the shared-memory tables as
-// broadcast reads.  Per candidate and element: exact quotient, round onto the FP4 grid, residual
-// FMA, square-accumulate FMA -- in element order, so the SSE has the same bits as in the one-pass
-// kernels and in the final encode.
+// Work layout.  A thread keeps its elements in registers as float pairs and runs every step of a
+// candidate on both halves of the pair at once with the packed binary32 instructions of sm_100
+// (fma.rn.f32x2 / mul.rn.f32x2), so one issue slot serves two elements:
+//   B <= 16   the thread owns 32 consecutive elements; pair i = (element i, element 16 + i), i.e.
+//             the two halves of a pair belong to different blocks and their SSE chains are
+//             independent.
+//   B >= 32   the thread owns one block; pair i = (element i, element B/2 + i).  The SSE of a
+//             block is one sequential chain, so the second half runs one candidate behind the
+//             first and starts from the first half's sum of the previous step.
+// The candidate loop is uniform across the CTA: decode scales come from shared memory as
+// broadcasts.
+//
+// One exact quotient per mantissa, not per candidate.  The decode scale of code c is
+// D_c = fl(S_c * g).  All codes whose S_c share a mantissa (eight classes for the FP8 scale
+// formats, one for the power-of-two format) have decode scales that differ by exact powers of two,
+// D_c = Dref * 2^k, as long as D_c is a normal number.  Hence fl(v / D_c) = fl(v / Dref) * 2^-k
+// exactly: the correctly rounded quotient is formed once per class and element, and a candidate
+// costs one multiply by a power of two, the FP4 rounding, and the two FMAs of the SSE.  Codes
+// whose decode scale is zero, subnormal, not finite or above 2^126, and threads holding a magnitude
+// above 2^60 or a nonzero one below 2^-62, take the general path (IEEE division), candidate by
+// candidate.
+//
+// Inside a class the members are visited in ascending code order and the smallest SSE bit pattern
+// is kept with a strict compare (SSE >= 0, so integer order is float order and the first of equals
+// is the smaller code); class winners are merged as 64-bit keys (SSE bits << 32 | code).
 #pragma once
 
 #include "mxq_device.cuh"
@@ -14,84 +34,393 @@
 
 namespace mxq {
 
-template <int B, bool FAST>
-__device__ __forceinline__ float candidate_sse(const float (&v)[B], float D, float R) {
+constexpr int kMaxMembers = 36;  // codes per mantissa class, FP8 formats (31 normal + 3 subnormal at most)
+
+// Mantissa class of a scale code: index of the 3-bit mantissa of its value.
+template <int FMT>
+__device__ __forceinline__ int code_class(int c) {
+    if constexpr (FMT == kUE8M0) return 0;
+    if (c >= 8) return c & 7;
+    // subnormal codes m * 2^(1-bias-3): 1, 2, 4 -> 1.0; 3, 6 -> 1.5; 5 -> 1.25; 7 -> 1.75
+    return (int)((0x64204000u >> (4 * c)) & 7u);
+}
+
+// Per-CTA tables of the search.  A code is "paired" when its decode scale is a normal number with
+// a biased exponent of at most 253, so that D = Dref * 2^k and 2^-k are both representable.
+struct BruteTables {
+    float D[256];          // decode scale of the code; NaN for codes that do not exist
+    float R[256];          // RN(1 / D) when 2^-60 <= D <= 2^60, else 0 (used by the final encode)
+    float4 cand[288];      // per class, paired members in ascending code order: (-D, -D, 2^-k, 2^-k)
+    uint8_t member[288];   // the code of each slot of cand[]
+    uint8_t paired[256];   // 1 when the code is in cand[]
+    float clsD[8];         // Dref of the class, in [1, 2)
+    float clsR[8];         // RN(1 / Dref)
+    int cnt[8];            // members per class
+    uint32_t warp_mask[8];
+    int n_unpaired;        // codes with a finite decode scale that are not in cand[]
+    uint8_t unpaired[256]; // ... in ascending order
+};
+
+template <int FMT>
+__device__ __forceinline__ int members_base(int cls) {
+    return FMT == kUE8M0 ? 0 : cls * kMaxMembers;
+}
+
+template <int FMT>
+__device__ __forceinline__ void build_brute_tables(BruteTables& T, float g) {
+    static_assert(kThreads == 256, "one thread per table entry");
+    build_scale_tables<FMT>(T.D, T.R, g);
+    const int c = threadIdx.x;
+    const uint32_t b = __float_as_uint(T.D[c]);
+    const uint32_t e = (b >> 23) & 0xFFu;
+    const bool is_paired = c < num_codes(FMT) && (b >> 31) == 0 && e >= 1 && e <= 253;
+    T.paired[c] = is_paired ? 1 : 0;
+    if (c < 8) T.cnt[c] = 0;
+    const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, is_paired);
+    if ((c & 31) == 0) T.warp_mask[c >> 5] = ballot;
+    // codes left to the general path: finite decode scale (zero and subnormal included), not paired
+    const bool is_unpaired = c < num_codes(FMT) && !is_paired && (b & 0x7FFFFFFFu) < 0x7F800000u;
+    const uint32_t ballot_u = __ballot_sync(0xFFFFFFFFu, is_unpaired);
+    __shared__ uint32_t unpaired_mask[8];
+    if ((c & 31) == 0) unpaired_mask[c >> 5] = ballot_u;
+    __syncthreads();
+    if (is_unpaired) {
+        int rank = __popc(ballot_u & ((1u << (c & 31)) - 1u));
+        for (int w = 0; w < (c >> 5); ++w) rank += __popc(unpaired_mask[w]);
+        T.unpaired[rank] = (uint8_t)c;
+    }
+    if (c == 0) {
+        int n = 0;
+        for (int w = 0; w < 8; ++w) n += __popc(unpaired_mask[w]);
+        T.n_unpaired = n;
+    }
+    if (is_paired) {
+        const int cls = code_class<FMT>(c);
+        int rank = 0;
+        if constexpr (FMT == kUE8M0) {
+            for (int w = 0; w < (c >> 5); ++w) rank += __popc(T.warp_mask[w]);
+            rank += __popc(ballot & ((1u << (c & 31)) - 1u));
+        } else {
+            for (int o = 1; o < 8 && o < c; ++o) rank += (T.paired[o] && code_class<FMT>(o) == cls) ? 1 : 0;
+            for (int o = 8 + cls; o < c; o += 8) rank += T.paired[o];
+        }
+        const float P = __uint_as_float((254u - e) << 23);
+        const float D = T.D[c];
+        const int slot = members_base<FMT>(cls) + rank;
+        T.cand[slot] = make_float4(-D, -D, P, P);
+        T.member[slot] = (uint8_t)c;
+        atomicAdd(&T.cnt[cls], 1);
+        if (rank == 0) {
+            const float Dref = __uint_as_float((b & 0x007FFFFFu) | 0x3F800000u);
+            T.clsD[cls] = Dref;
+            T.clsR[cls] = __frcp_rn(Dref);
+        }
+    }
+    __syncthreads();
+    // the search takes two members per trip: an odd class repeats its last member once
+    if (c < 8 && (T.cnt[c] & 1)) {
+        const int last = members_base<FMT>(c) + T.cnt[c] - 1;
+        T.cand[last + 1] = T.cand[last];
+        T.member[last + 1] = T.member[last];
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------------
+// packed helpers
+// ------------------------------------------------------------------------------------------------
+// Both halves of t rounded onto the FP4 grid (round-to-nearest-even, saturating at +-6), returned
+// as floats.
+__device__ __forceinline__ float2 round_e2m1_pair(float2 t) {
+    uint32_t h;
+    asm("{\n"
+        " .reg .b8 b0;\n"
+        " cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n"
+        " cvt.rn.f16x2.e2m1x2 %0, b0;\n"
+        "}"
+        : "=r"(h)
+        : "f"(t.x), "f"(t.y));
+    return __half22float2(*reinterpret_cast<__half2*>(&h));
+}
+
+// fl32(v / Dref) for both halves; nD = -Dref, R = RN(1 / Dref), Dref in [1, 2), |v| <= 2^60.
+// Same value as quotient_corrected() except for the sign of a zero quotient, which the search
+// does not use.
+__device__ __forceinline__ float2 quotient_pair(float2 v, float2 nD, float2 R) {
+    float2 q = __fmul2_rn(v, R);
+    float2 r = __ffma2_rn(q, nD, v);
+    q = __ffma2_rn(r, R, q);
+    r = __ffma2_rn(q, nD, v);
+    q = __ffma2_rn(r, R, q);
+    return q;
+}
+
+__device__ __forceinline__ unsigned long long sse_key(float s, int c) {
+    return ((unsigned long long)__float_as_uint(s) << 32) | (unsigned long long)(unsigned)c;
+}
+
+// General path for one block held in `lane` (0 = .x, 1 = .y) of pairs first .. first + B - 1.
+template <int B, int NP>
+__device__ __forceinline__ float general_sse(const float2 (&v2)[NP], int first, int lane, float D) {
     float s = 0.0f;
 #pragma unroll
     for (int i = 0; i < B; i += 2) {
-        float t0, t1;
-        if constexpr (FAST) {
-            t0 = quotient_corrected(v[i], D, R);
-            t1 = quotient_corrected(v[i + 1], D, R);
-        } else {
-            t0 = quotient_general(v[i], D);
-            t1 = quotient_general(v[i + 1], D);
-        }
-        const float2 q = round_e2m1x2(t0, t1);
-        const float e0 = __fmaf_rn(-q.x, D, v[i]);
+        const float a = lane ? v2[first + i].y : v2[first + i].x;
+        const float b = lane ? v2[first + i + 1].y : v2[first + i + 1].x;
+        const float2 q = round_e2m1x2(quotient_general(a, D), quotient_general(b, D));
+        const float e0 = __fmaf_rn(-q.x, D, a);
         s = __fmaf_rn(e0, e0, s);
-        const float e1 = __fmaf_rn(-q.y, D, v[i + 1]);
+        const float e1 = __fmaf_rn(-q.y, D, b);
         s = __fmaf_rn(e1, e1, s);
     }
     return s;
 }
 
+// ------------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------------
+// Fold the winner of one class (smallest SSE bits; first, i.e. smallest, code among equals) into
+// the running (SSE, code) key.
+__device__ __forceinline__ void merge_class_winner(unsigned long long& best, uint32_t bits, int code) {
+    const unsigned long long k = ((unsigned long long)bits << 32) | (unsigned long long)(unsigned)code;
+    if (k < best) best = k;
+}
+
+// Strict "smaller SSE bits wins", without a branch.
+__device__ __forceinline__ void keep_smaller(uint32_t& best_bits, int& best_slot, uint32_t bits, int slot) {
+    best_slot = bits < best_bits ? slot : best_slot;
+    best_bits = min(best_bits, bits);
+}
+
 template <int DT, int B, int FMT>
 __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
-    __shared__ float tabD[256];
-    __shared__ float tabR[256];
+    constexpr bool SKEW = (B >= 32);          // the pair's halves are the two halves of one block
+    constexpr int G = SKEW ? B : 32;          // elements per thread
+    constexpr int NP = G / 2;                 // pairs per thread
+    constexpr int BL = SKEW ? NP : B;         // elements of one block inside one half
+    constexpr int NBL = NP / BL;              // blocks per half (1 when SKEW)
+    constexpr int NBT = SKEW ? 1 : 2 * NBL;   // blocks per thread
+    constexpr int NCLS = (FMT == kUE8M0) ? 1 : 8;
+    constexpr float kTiny = 2.168404344971009e-19f;  // 2^-62
+
+    __shared__ BruteTables T;
     const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    build_scale_tables<FMT>(tabD, tabR, g);
+    build_brute_tables<FMT>(T, g);
     const int first = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
 
     const size_t stride = (size_t)gridDim.x * kThreads;
-    for (size_t blk = (size_t)blockIdx.x * kThreads + threadIdx.x; blk < p.n_items; blk += stride) {
-        float v[B];
-        load_elems<DT, B>(p.x, blk * B, v);
+    for (size_t grp = (size_t)blockIdx.x * kThreads + threadIdx.x; grp < p.n_items; grp += stride) {
+        float2 v2[NP];
         float amax = 0.0f;
+        bool tiny = false;   // a nonzero magnitude below 2^-62: its quotient by Dref may be inexact
+        {
+            float v[G];
+            load_elems<DT, G>(p.x, grp * G, v);
 #pragma unroll
-        for (int i = 0; i < B; ++i) amax = fmaxf(amax, fabsf(v[i]));
-        const bool fast_ok = amax <= kFastMax;
+            for (int i = 0; i < NP; ++i) {
+                v2[i] = make_float2(v[i], v[NP + i]);
+                const float a0 = fabsf(v[i]), a1 = fabsf(v[NP + i]);
+                amax = fmaxf(amax, fmaxf(a0, a1));
+                tiny |= (a0 < kTiny && a0 != 0.0f) || (a1 < kTiny && a1 != 0.0f);
+            }
+        }
+        const bool fast_ok = (amax <= kFastMax) && !tiny;
 
-        uint32_t best_bits = 0xFFFFFFFFu;
-        int best = first;
-        for (int c = first; c < num_codes(FMT); ++c) {
-            const float D = tabD[c];
-            const float R = tabR[c];
-            if (!(fabsf(D) <= 3.402823466e38f)) continue;  // decode scale overflowed: not usable
-            float s;
-            if (R != 0.0f && fast_ok) s = candidate_sse<B, true>(v, D, R);
-            else s = candidate_sse<B, false>(v, D, R);
-            const uint32_t bits = __float_as_uint(s);  // s >= 0: integer order equals float order
-            if (bits < best_bits) {
-                best_bits = bits;
-                best = c;
+        // best[k]: k < NBL -> block k of the low half, else block k - NBL of the high half
+        unsigned long long best[NBT];
+#pragma unroll
+        for (int k = 0; k < NBT; ++k) best[k] = sse_key(__uint_as_float(0xFFFFFFFFu), first);
+
+        if (fast_ok) {
+            for (int cls = 0; cls < NCLS; ++cls) {
+                const int cnt = T.cnt[cls];
+                if (cnt == 0) continue;
+                const float Dr = T.clsD[cls], Rr = T.clsR[cls];
+                const float2 nDr2 = make_float2(-Dr, -Dr), Rr2 = make_float2(Rr, Rr);
+                float2 tb[NP];
+#pragma unroll
+                for (int i = 0; i < NP; ++i) tb[i] = quotient_pair(v2[i], nDr2, Rr2);
+                const int base = members_base<FMT>(cls);
+                const float4* cand = T.cand + base;
+
+                uint32_t cbest[NBT];
+                int cslot[NBT];
+#pragma unroll
+                for (int k = 0; k < NBT; ++k) { cbest[k] = 0xFFFFFFFFu; cslot[k] = 0; }
+
+                if constexpr (!SKEW) {
+                    // two members per trip: two independent SSE chains keep the FMA pipe fed
+                    for (int m = 0; m < cnt; m += 2) {
+                        const float4 dpA = cand[m], dpB = cand[m + 1];
+                        const float2 nDA = make_float2(dpA.x, dpA.y), PA = make_float2(dpA.z, dpA.w);
+                        const float2 nDB = make_float2(dpB.x, dpB.y), PB = make_float2(dpB.z, dpB.w);
+                        float2 sA[NBL], sB[NBL];
+#pragma unroll
+                        for (int k = 0; k < NBL; ++k) sA[k] = sB[k] = make_float2(0.0f, 0.0f);
+#pragma unroll
+                        for (int i = 0; i < NP; ++i) {
+                            const float2 qA = round_e2m1_pair(__fmul2_rn(tb[i], PA));
+                            const float2 qB = round_e2m1_pair(__fmul2_rn(tb[i], PB));
+                            const float2 eA = __ffma2_rn(qA, nDA, v2[i]);
+                            const float2 eB = __ffma2_rn(qB, nDB, v2[i]);
+                            sA[i / BL] = __ffma2_rn(eA, eA, sA[i / BL]);
+                            sB[i / BL] = __ffma2_rn(eB, eB, sB[i / BL]);
+                        }
+#pragma unroll
+                        for (int k = 0; k < NBL; ++k) {
+                            keep_smaller(cbest[k], cslot[k], __float_as_uint(sA[k].x), m);
+                            keep_smaller(cbest[NBL + k], cslot[NBL + k], __float_as_uint(sA[k].y), m);
+                            keep_smaller(cbest[k], cslot[k], __float_as_uint(sB[k].x), m + 1);
+                            keep_smaller(cbest[NBL + k], cslot[NBL + k], __float_as_uint(sB[k].y), m + 1);
+                        }
+                    }
+                } else {
+                    // trip m: the low half evaluates members m and m + 1, the high half finishes
+                    // members m - 2 and m - 1 from the low-half sums of the previous trip
+                    float nDA_prev = cand[0].x, PA_prev = cand[0].z, nDB_prev = nDA_prev, PB_prev = PA_prev;
+                    float carryA = 0.0f, carryB = 0.0f;
+                    for (int m = 0; m < cnt + 2; m += 2) {
+                        const int mm = m < cnt ? m : 0;         // past the end: repeat a trip, low-half result unused
+                        const float4 dpA = cand[mm], dpB = cand[mm + 1];
+                        const float2 nDA = make_float2(dpA.x, nDA_prev), PA = make_float2(dpA.z, PA_prev);
+                        const float2 nDB = make_float2(dpB.x, nDB_prev), PB = make_float2(dpB.z, PB_prev);
+                        float2 sA = make_float2(0.0f, carryA), sB = make_float2(0.0f, carryB);
+#pragma unroll
+                        for (int i = 0; i < NP; ++i) {
+                            const float2 qA = round_e2m1_pair(__fmul2_rn(tb[i], PA));
+                            const float2 qB = round_e2m1_pair(__fmul2_rn(tb[i], PB));
+                            const float2 eA = __ffma2_rn(qA, nDA, v2[i]);
+                            const float2 eB = __ffma2_rn(qB, nDB, v2[i]);
+                            sA = __ffma2_rn(eA, eA, sA);
+                            sB = __ffma2_rn(eB, eB, sB);
+                        }
+                        if (m > 0) {
+                            keep_smaller(cbest[0], cslot[0], __float_as_uint(sA.y), m - 2);
+                            keep_smaller(cbest[0], cslot[0], __float_as_uint(sB.y), m - 1);
+                        }
+                        carryA = sA.x; carryB = sB.x;
+                        nDA_prev = dpA.x; PA_prev = dpA.z; nDB_prev = dpB.x; PB_prev = dpB.z;
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < NBT; ++k)
+                    if (cbest[k] != 0xFFFFFFFFu) merge_class_winner(best[k], cbest[k], T.member[base + cslot[k]]);
             }
         }
 
-        // final encode with the winner
-        const float D = tabD[best];
-        const float R = tabR[best];
-        const bool fast = (R != 0.0f) && fast_ok;
-        float t[B];
+        // candidates on the general path (decode scale zero, subnormal or huge; all candidates when
+        // the thread holds a magnitude above 2^60 or a nonzero one below 2^-62)
+        const int n_general = fast_ok ? T.n_unpaired : num_codes(FMT);
+        for (int j = 0; j < n_general; ++j) {
+            const int c = fast_ok ? (int)T.unpaired[j] : j;
+            if (c < first) continue;
+            const float D = T.D[c];
+            if (!(fabsf(D) <= 3.402823466e38f)) continue;  // decode scale overflowed: not usable
+            if constexpr (!SKEW) {
 #pragma unroll
-        for (int i = 0; i < B; ++i) t[i] = fast ? quotient_corrected(v[i], D, R) : quotient_general(v[i], D);
-        if constexpr (B >= 8) {
-            uint32_t packed[B / 8];
+                for (int k = 0; k < NBL; ++k) {
+                    const unsigned long long k0 = sse_key(general_sse<B, NP>(v2, k * BL, 0, D), c);
+                    const unsigned long long k1 = sse_key(general_sse<B, NP>(v2, k * BL, 1, D), c);
+                    if (k0 < best[k]) best[k] = k0;
+                    if (k1 < best[NBL + k]) best[NBL + k] = k1;
+                }
+            } else {
+                float s = 0.0f;
 #pragma unroll
-            for (int k = 0; k < B / 8; ++k)
-                packed[k] = pack_e2m1x8(t[8 * k], t[8 * k + 1], t[8 * k + 2], t[8 * k + 3], t[8 * k + 4],
-                                        t[8 * k + 5], t[8 * k + 6], t[8 * k + 7]);
-            store_bytes<B / 2>(p.codes + blk * (B / 2), packed);
-        } else {
-            uint32_t packed = 0;
+                for (int h = 0; h < 2; ++h) {
 #pragma unroll
-            for (int k = 0; k < B / 2; ++k) packed |= pack_e2m1x2(t[2 * k], t[2 * k + 1]) << (8 * k);
-            store_bytes<B / 2>(p.codes + blk * (B / 2), &packed);
+                    for (int i = 0; i < NP; i += 2) {
+                        const float a = h ? v2[i].y : v2[i].x;
+                        const float b = h ? v2[i + 1].y : v2[i + 1].x;
+                        const float2 q = round_e2m1x2(quotient_general(a, D), quotient_general(b, D));
+                        const float e0 = __fmaf_rn(-q.x, D, a);
+                        s = __fmaf_rn(e0, e0, s);
+                        const float e1 = __fmaf_rn(-q.y, D, b);
+                        s = __fmaf_rn(e1, e1, s);
+                    }
+                }
+                const unsigned long long k0 = sse_key(s, c);
+                if (k0 < best[0]) best[0] = k0;
+            }
         }
-        p.scales[blk] = (uint8_t)best;
-        if (p.block_sse) p.block_sse[blk] = __uint_as_float(best_bits);
+
+        // final encode with the winners
+        uint32_t packed[G / 8];
+        uint32_t sc[(NBT + 3) / 4];
+        uint32_t sw[NBT];
+#pragma unroll
+        for (int k = 0; k < (NBT + 3) / 4; ++k) sc[k] = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float t[NP];
+#pragma unroll
+            for (int k = 0; k < NBL; ++k) {
+                const int kb = SKEW ? 0 : h * NBL + k;   // block index inside the thread
+                const int code = (int)(best[kb] & 0xFFu);
+                const float D = T.D[code];
+                const float R = T.R[code];
+                const bool fast = (R != 0.0f) && (amax <= kFastMax);
+#pragma unroll
+                for (int i = 0; i < BL; ++i) {
+                    const float a = h ? v2[k * BL + i].y : v2[k * BL + i].x;
+                    t[k * BL + i] = fast ? quotient_corrected(a, D, R) : quotient_general(a, D);
+                }
+                if (!SKEW || h == 0) {
+                    sc[kb / 4] |= (uint32_t)code << (8 * (kb % 4));
+                    sw[kb] = (uint32_t)(best[kb] >> 32);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < NP / 8; ++k)
+                packed[h * (NP / 8) + k] = pack_e2m1x8(t[8 * k], t[8 * k + 1], t[8 * k + 2], t[8 * k + 3], t[8 * k + 4],
+                                                       t[8 * k + 5], t[8 * k + 6], t[8 * k + 7]);
+        }
+        store_bytes<G / 2>(p.codes + grp * (G / 2), packed);
+        store_bytes<NBT>(p.scales + grp * NBT, sc);
+        if (p.block_sse) store_bytes<4 * NBT>(p.block_sse + grp * NBT, sw);
     }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The blocks past the last whole 32-element group (block sizes up to 16 only): one block per
+// thread, general path.
+// ------------------------------------------------------------------------------------------------
+template <int DT, int B, int FMT>
+__global__ void k_brute_tail(QuantArgs p) {
+    const size_t b = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= p.n_items) return;
+    const size_t blk = p.first_item + b;
+    const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
+    const int first = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
+    float v[B];
+    load_elems<DT, B>(p.x, blk * B, v);
+    unsigned long long best = sse_key(__uint_as_float(0xFFFFFFFFu), first);
+    for (int c = first; c < num_codes(FMT); ++c) {
+        const float D = __fmul_rn(scale_value(FMT, c), g);
+        if (!(fabsf(D) <= 3.402823466e38f)) continue;
+        float s = 0.0f;
+#pragma unroll
+        for (int i = 0; i < B; i += 2) {
+            const float2 q = round_e2m1x2(quotient_general(v[i], D), quotient_general(v[i + 1], D));
+            const float e0 = __fmaf_rn(-q.x, D, v[i]);
+            s = __fmaf_rn(e0, e0, s);
+            const float e1 = __fmaf_rn(-q.y, D, v[i + 1]);
+            s = __fmaf_rn(e1, e1, s);
+        }
+        const unsigned long long k = sse_key(s, c);
+        if (k < best) best = k;
+    }
+    const int code = (int)(best & 0xFFu);
+    const float D = __fmul_rn(scale_value(FMT, code), g);
+    uint32_t packed[(B + 7) / 8];
+#pragma unroll
+    for (int k = 0; k < (B + 7) / 8; ++k) packed[k] = 0;
+#pragma unroll
+    for (int k = 0; k < B / 2; ++k)
+        packed[k / 4] |= pack_e2m1x2(quotient_general(v[2 * k], D), quotient_general(v[2 * k + 1], D)) << (8 * (k % 4));
+    store_bytes<B / 2>(p.codes + blk * (B / 2), packed);
+    p.scales[blk] = (uint8_t)code;
+    if (p.block_sse) p.block_sse[blk] = __uint_as_float((uint32_t)(best >> 32));
 }
 
 template <int DT, int B, int FMT>
@@ -107,12 +436,32 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
         if (err != cudaSuccess) return err;
         ctas_per_sm[dev] = n > 0 ? n : 1;
     }
-    const size_t want = (a.n_items + kThreads - 1) / kThreads;
-    const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
-    const unsigned grid = (unsigned)(want < cap ? want : cap);
-    k_brute<DT, B, FMT><<<grid, kThreads, 0, stream>>>(a);
-    count_launch();
-    return cudaGetLastError();
+    constexpr size_t G = (B >= 32) ? B : 32;      // elements per thread of k_brute
+    const size_t n_blocks = a.n_items;
+    const size_t n_groups = n_blocks * B / G;
+    if (n_groups > 0) {
+        QuantArgs m = a;
+        m.n_items = n_groups;
+        const size_t want = (n_groups + kThreads - 1) / kThreads;
+        const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
+        const unsigned grid = (unsigned)(want < cap ? want : cap);
+        k_brute<DT, B, FMT><<<grid, kThreads, 0, stream>>>(m);
+        count_launch();
+        err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+    }
+    if constexpr (B < 32) {
+        const size_t done = n_groups * G / B;
+        if (done < n_blocks) {
+            QuantArgs t = a;
+            t.first_item = done;
+            t.n_items = n_blocks - done;
+            k_brute_tail<DT, B, FMT><<<1, 32, 0, stream>>>(t);
+            count_launch();
+            err = cudaGetLastError();
+        }
+    }
+    return err;
 }
 
 template <int DT, int B>
