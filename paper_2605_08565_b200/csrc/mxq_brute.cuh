@@ -46,24 +46,30 @@ __device__ __forceinline__ int code_class(int c) {
 }
 
 // Per-CTA tables of the search.  A code is "paired" when its decode scale is a normal number with
-// a biased exponent of at most 253, so that D = Dref * 2^k and 2^-k are both representable.
+// a biased exponent of at most 253, so that D = Dref * 2^k and 2^-k are both representable.  The
+// paired codes of a mantissa class form two lists: kind 1 holds the codes whose -D is exactly
+// representable in f16 (their residual is one mixed-precision FMA from the unpacked f16 grid
+// value), kind 0 the others (f16 -> f32 convert, then an FFMA).  List index = 2 * class + kind.
+constexpr int kLists = 16;
 struct BruteTables {
-    float D[256];          // decode scale of the code; NaN for codes that do not exist
-    float R[256];          // RN(1 / D) when 2^-60 <= D <= 2^60, else 0 (used by the final encode)
-    float4 cand[288];      // per class, paired members in ascending code order: (-D, -D, 2^-k, 2^-k)
-    uint8_t member[288];   // the code of each slot of cand[]
-    uint8_t paired[256];   // 1 when the code is in cand[]
-    float clsD[8];         // Dref of the class, in [1, 2)
-    float clsR[8];         // RN(1 / Dref)
-    int cnt[8];            // members per class
-    uint32_t warp_mask[8];
-    int n_unpaired;        // codes with a finite decode scale that are not in cand[]
-    uint8_t unpaired[256]; // ... in ascending order
+    float D[256];            // decode scale of the code; NaN for codes that do not exist
+    float R[256];            // RN(1 / D) when 2^-60 <= D <= 2^60, else 0 (used by the final encode)
+    float4 cand[kLists * kMaxMembers];    // per list, ascending code order: (-D, 2^-k, f16(-D) twice as bits, 0)
+    uint8_t member[kLists * kMaxMembers]; // the code of each slot of cand[]
+    uint8_t kind[256];       // 0, 1 as above; 2 = not paired
+    float clsD[8];           // Dref of the class, in [1, 2)
+    float clsR[8];           // RN(1 / Dref)
+    int cnt[kLists];         // members per list
+    uint32_t kind_mask[2][8];
+    uint32_t unpaired_mask[8];
+    int n_unpaired;          // codes with a finite decode scale that are not paired
+    uint8_t unpaired[256];   // ... in ascending order
 };
 
 template <int FMT>
-__device__ __forceinline__ int members_base(int cls) {
-    return FMT == kUE8M0 ? 0 : cls * kMaxMembers;
+__device__ __forceinline__ int members_base(int list) {
+    // the power-of-two format has one class: its two lists get half of the array each
+    return FMT == kUE8M0 ? list * (kLists * kMaxMembers / 2) : list * kMaxMembers;
 }
 
 template <int FMT>
@@ -71,54 +77,62 @@ __device__ __forceinline__ void build_brute_tables(BruteTables& T, float g) {
     static_assert(kThreads == 256, "one thread per table entry");
     build_scale_tables<FMT>(T.D, T.R, g);
     const int c = threadIdx.x;
-    const uint32_t b = __float_as_uint(T.D[c]);
+    const float D = T.D[c];
+    const uint32_t b = __float_as_uint(D);
     const uint32_t e = (b >> 23) & 0xFFu;
     const bool is_paired = c < num_codes(FMT) && (b >> 31) == 0 && e >= 1 && e <= 253;
-    T.paired[c] = is_paired ? 1 : 0;
-    if (c < 8) T.cnt[c] = 0;
-    const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, is_paired);
-    if ((c & 31) == 0) T.warp_mask[c >> 5] = ballot;
+    const __half hD = __float2half_rn(-D);
+    const int kind = !is_paired ? 2 : (__half2float(hD) == -D ? 1 : 0);
+    T.kind[c] = (uint8_t)kind;
+    if (c < kLists) T.cnt[c] = 0;
+    const uint32_t ballot0 = __ballot_sync(0xFFFFFFFFu, kind == 0);
+    const uint32_t ballot1 = __ballot_sync(0xFFFFFFFFu, kind == 1);
     // codes left to the general path: finite decode scale (zero and subnormal included), not paired
     const bool is_unpaired = c < num_codes(FMT) && !is_paired && (b & 0x7FFFFFFFu) < 0x7F800000u;
     const uint32_t ballot_u = __ballot_sync(0xFFFFFFFFu, is_unpaired);
-    __shared__ uint32_t unpaired_mask[8];
-    if ((c & 31) == 0) unpaired_mask[c >> 5] = ballot_u;
+    if ((c & 31) == 0) {
+        T.kind_mask[0][c >> 5] = ballot0;
+        T.kind_mask[1][c >> 5] = ballot1;
+        T.unpaired_mask[c >> 5] = ballot_u;
+    }
     __syncthreads();
+    const uint32_t below = (1u << (c & 31)) - 1u;
     if (is_unpaired) {
-        int rank = __popc(ballot_u & ((1u << (c & 31)) - 1u));
-        for (int w = 0; w < (c >> 5); ++w) rank += __popc(unpaired_mask[w]);
+        int rank = __popc(ballot_u & below);
+        for (int w = 0; w < (c >> 5); ++w) rank += __popc(T.unpaired_mask[w]);
         T.unpaired[rank] = (uint8_t)c;
     }
     if (c == 0) {
         int n = 0;
-        for (int w = 0; w < 8; ++w) n += __popc(unpaired_mask[w]);
+        for (int w = 0; w < 8; ++w) n += __popc(T.unpaired_mask[w]);
         T.n_unpaired = n;
     }
     if (is_paired) {
         const int cls = code_class<FMT>(c);
         int rank = 0;
         if constexpr (FMT == kUE8M0) {
-            for (int w = 0; w < (c >> 5); ++w) rank += __popc(T.warp_mask[w]);
-            rank += __popc(ballot & ((1u << (c & 31)) - 1u));
+            for (int w = 0; w < (c >> 5); ++w) rank += __popc(T.kind_mask[kind][w]);
+            rank += __popc((kind ? ballot1 : ballot0) & below);
         } else {
-            for (int o = 1; o < 8 && o < c; ++o) rank += (T.paired[o] && code_class<FMT>(o) == cls) ? 1 : 0;
-            for (int o = 8 + cls; o < c; o += 8) rank += T.paired[o];
+            for (int o = 1; o < 8 && o < c; ++o) rank += (T.kind[o] == kind && code_class<FMT>(o) == cls) ? 1 : 0;
+            for (int o = 8 + cls; o < c; o += 8) rank += (T.kind[o] == kind) ? 1 : 0;
         }
         const float P = __uint_as_float((254u - e) << 23);
-        const float D = T.D[c];
-        const int slot = members_base<FMT>(cls) + rank;
-        T.cand[slot] = make_float4(-D, -D, P, P);
+        const uint32_t h16 = (uint32_t)__half_as_ushort(hD);
+        const int list = 2 * cls + kind;
+        const int slot = members_base<FMT>(list) + rank;
+        T.cand[slot] = make_float4(-D, P, __uint_as_float(h16 | (h16 << 16)), 0.0f);
         T.member[slot] = (uint8_t)c;
-        atomicAdd(&T.cnt[cls], 1);
-        if (rank == 0) {
+        atomicAdd(&T.cnt[list], 1);
+        if (rank == 0) {   // both kinds of a class write the same values
             const float Dref = __uint_as_float((b & 0x007FFFFFu) | 0x3F800000u);
             T.clsD[cls] = Dref;
             T.clsR[cls] = __frcp_rn(Dref);
         }
     }
     __syncthreads();
-    // the search takes two members per trip: an odd class repeats its last member once
-    if (c < 8 && (T.cnt[c] & 1)) {
+    // the search takes two members per trip: an odd list repeats its last member once
+    if (c < kLists && (T.cnt[c] & 1)) {
         const int last = members_base<FMT>(c) + T.cnt[c] - 1;
         T.cand[last + 1] = T.cand[last];
         T.member[last + 1] = T.member[last];
@@ -129,9 +143,13 @@ __device__ __forceinline__ void build_brute_tables(BruteTables& T, float g) {
 // ------------------------------------------------------------------------------------------------
 // packed helpers
 // ------------------------------------------------------------------------------------------------
-// Both halves of t rounded onto the FP4 grid (round-to-nearest-even, saturating at +-6), returned
-// as floats.
-__device__ __forceinline__ float2 round_e2m1_pair(float2 t) {
+// Residuals of one pair for one candidate: t = tb * 2^-k, q = t rounded onto the FP4 grid
+// (round-to-nearest-even, saturating at +-6), e = fma(q, -D, v).  HALF: -D is given in f16
+// (low half of nD16 for .x, high half for .y) and the FMA takes q straight from the unpacked f16
+// pair (fma.rn.f32.f16: exact product, one rounding to binary32); otherwise q is widened first.
+template <bool HALF>
+__device__ __forceinline__ float2 residual_pair(float2 tb, float2 P2, float2 v, float2 nD2, uint32_t nD16) {
+    const float2 t = __fmul2_rn(tb, P2);
     uint32_t h;
     asm("{\n"
         " .reg .b8 b0;\n"
@@ -140,7 +158,21 @@ __device__ __forceinline__ float2 round_e2m1_pair(float2 t) {
         "}"
         : "=r"(h)
         : "f"(t.x), "f"(t.y));
-    return __half22float2(*reinterpret_cast<__half2*>(&h));
+    if constexpr (HALF) {
+        float2 e;
+        asm("{\n"
+            " .reg .b16 qlo, qhi, dlo, dhi;\n"
+            " mov.b32 {qlo, qhi}, %2;\n"
+            " mov.b32 {dlo, dhi}, %3;\n"
+            " fma.rn.f32.f16 %0, qlo, dlo, %4;\n"
+            " fma.rn.f32.f16 %1, qhi, dhi, %5;\n"
+            "}"
+            : "=f"(e.x), "=f"(e.y)
+            : "r"(h), "r"(nD16), "f"(v.x), "f"(v.y));
+        return e;
+    } else {
+        return __ffma2_rn(__half22float2(*reinterpret_cast<__half2*>(&h)), nD2, v);
+    }
 }
 
 // fl32(v / Dref) for both halves; nD = -Dref, R = RN(1 / Dref), Dref in [1, 2), |v| <= 2^60.
@@ -192,6 +224,83 @@ __device__ __forceinline__ void keep_smaller(uint32_t& best_bits, int& best_slot
     best_bits = min(best_bits, bits);
 }
 
+// All members of one list (one mantissa class, one residual kind) against the thread's elements;
+// the list winner of every block is folded into best[].
+template <int B, int FMT, bool HALF, int NP, int NBT>
+__device__ __forceinline__ void search_list(const BruteTables& T, int list, const float2 (&v2)[NP],
+                                            const float2 (&tb)[NP], unsigned long long (&best)[NBT]) {
+    constexpr bool SKEW = (B >= 32);
+    constexpr int BL = SKEW ? NP : B;
+    constexpr int NBL = NP / BL;
+    const int cnt = T.cnt[list];
+    if (cnt == 0) return;
+    const int base = members_base<FMT>(list);
+    const float4* cand = T.cand + base;
+    uint32_t cbest[NBT];
+    int cslot[NBT];
+#pragma unroll
+    for (int k = 0; k < NBT; ++k) { cbest[k] = 0xFFFFFFFFu; cslot[k] = 0; }
+
+    if constexpr (!SKEW) {
+        // two members per trip: two independent SSE chains keep the FMA pipe fed
+        for (int m = 0; m < cnt; m += 2) {
+            const float4 dpA = cand[m], dpB = cand[m + 1];
+            const float2 nDA = make_float2(dpA.x, dpA.x), PA = make_float2(dpA.y, dpA.y);
+            const float2 nDB = make_float2(dpB.x, dpB.x), PB = make_float2(dpB.y, dpB.y);
+            const uint32_t hA = __float_as_uint(dpA.z), hB = __float_as_uint(dpB.z);
+            float2 sA[NBL], sB[NBL];
+#pragma unroll
+            for (int k = 0; k < NBL; ++k) sA[k] = sB[k] = make_float2(0.0f, 0.0f);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const float2 eA = residual_pair<HALF>(tb[i], PA, v2[i], nDA, hA);
+                const float2 eB = residual_pair<HALF>(tb[i], PB, v2[i], nDB, hB);
+                sA[i / BL] = __ffma2_rn(eA, eA, sA[i / BL]);
+                sB[i / BL] = __ffma2_rn(eB, eB, sB[i / BL]);
+            }
+#pragma unroll
+            for (int k = 0; k < NBL; ++k) {
+                keep_smaller(cbest[k], cslot[k], __float_as_uint(sA[k].x), m);
+                keep_smaller(cbest[NBL + k], cslot[NBL + k], __float_as_uint(sA[k].y), m);
+                keep_smaller(cbest[k], cslot[k], __float_as_uint(sB[k].x), m + 1);
+                keep_smaller(cbest[NBL + k], cslot[NBL + k], __float_as_uint(sB[k].y), m + 1);
+            }
+        }
+    } else {
+        // trip m: the low half evaluates members m and m + 1, the high half finishes members
+        // m - 2 and m - 1 from the low-half sums of the previous trip
+        float nDA_prev = cand[0].x, PA_prev = cand[0].y, nDB_prev = nDA_prev, PB_prev = PA_prev;
+        uint32_t hA_prev = __float_as_uint(cand[0].z), hB_prev = hA_prev;
+        float carryA = 0.0f, carryB = 0.0f;
+        for (int m = 0; m < cnt + 2; m += 2) {
+            const int mm = m < cnt ? m : 0;   // past the end: repeat a trip, low-half result unused
+            const float4 dpA = cand[mm], dpB = cand[mm + 1];
+            const float2 nDA = make_float2(dpA.x, nDA_prev), PA = make_float2(dpA.y, PA_prev);
+            const float2 nDB = make_float2(dpB.x, nDB_prev), PB = make_float2(dpB.y, PB_prev);
+            const uint32_t hA = (__float_as_uint(dpA.z) & 0xFFFFu) | (hA_prev & 0xFFFF0000u);
+            const uint32_t hB = (__float_as_uint(dpB.z) & 0xFFFFu) | (hB_prev & 0xFFFF0000u);
+            float2 sA = make_float2(0.0f, carryA), sB = make_float2(0.0f, carryB);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const float2 eA = residual_pair<HALF>(tb[i], PA, v2[i], nDA, hA);
+                const float2 eB = residual_pair<HALF>(tb[i], PB, v2[i], nDB, hB);
+                sA = __ffma2_rn(eA, eA, sA);
+                sB = __ffma2_rn(eB, eB, sB);
+            }
+            if (m > 0) {
+                keep_smaller(cbest[0], cslot[0], __float_as_uint(sA.y), m - 2);
+                keep_smaller(cbest[0], cslot[0], __float_as_uint(sB.y), m - 1);
+            }
+            carryA = sA.x; carryB = sB.x;
+            nDA_prev = dpA.x; PA_prev = dpA.y; nDB_prev = dpB.x; PB_prev = dpB.y;
+            hA_prev = __float_as_uint(dpA.z); hB_prev = __float_as_uint(dpB.z);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < NBT; ++k)
+        if (cbest[k] != 0xFFFFFFFFu) merge_class_winner(best[k], cbest[k], T.member[base + cslot[k]]);
+}
+
 template <int DT, int B, int FMT>
 __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
     constexpr bool SKEW = (B >= 32);          // the pair's halves are the two halves of one block
@@ -233,78 +342,14 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
 
         if (fast_ok) {
             for (int cls = 0; cls < NCLS; ++cls) {
-                const int cnt = T.cnt[cls];
-                if (cnt == 0) continue;
+                if (T.cnt[2 * cls] + T.cnt[2 * cls + 1] == 0) continue;
                 const float Dr = T.clsD[cls], Rr = T.clsR[cls];
                 const float2 nDr2 = make_float2(-Dr, -Dr), Rr2 = make_float2(Rr, Rr);
                 float2 tb[NP];
 #pragma unroll
                 for (int i = 0; i < NP; ++i) tb[i] = quotient_pair(v2[i], nDr2, Rr2);
-                const int base = members_base<FMT>(cls);
-                const float4* cand = T.cand + base;
-
-                uint32_t cbest[NBT];
-                int cslot[NBT];
-#pragma unroll
-                for (int k = 0; k < NBT; ++k) { cbest[k] = 0xFFFFFFFFu; cslot[k] = 0; }
-
-                if constexpr (!SKEW) {
-                    // two members per trip: two independent SSE chains keep the FMA pipe fed
-                    for (int m = 0; m < cnt; m += 2) {
-                        const float4 dpA = cand[m], dpB = cand[m + 1];
-                        const float2 nDA = make_float2(dpA.x, dpA.y), PA = make_float2(dpA.z, dpA.w);
-                        const float2 nDB = make_float2(dpB.x, dpB.y), PB = make_float2(dpB.z, dpB.w);
-                        float2 sA[NBL], sB[NBL];
-#pragma unroll
-                        for (int k = 0; k < NBL; ++k) sA[k] = sB[k] = make_float2(0.0f, 0.0f);
-#pragma unroll
-                        for (int i = 0; i < NP; ++i) {
-                            const float2 qA = round_e2m1_pair(__fmul2_rn(tb[i], PA));
-                            const float2 qB = round_e2m1_pair(__fmul2_rn(tb[i], PB));
-                            const float2 eA = __ffma2_rn(qA, nDA, v2[i]);
-                            const float2 eB = __ffma2_rn(qB, nDB, v2[i]);
-                            sA[i / BL] = __ffma2_rn(eA, eA, sA[i / BL]);
-                            sB[i / BL] = __ffma2_rn(eB, eB, sB[i / BL]);
-                        }
-#pragma unroll
-                        for (int k = 0; k < NBL; ++k) {
-                            keep_smaller(cbest[k], cslot[k], __float_as_uint(sA[k].x), m);
-                            keep_smaller(cbest[NBL + k], cslot[NBL + k], __float_as_uint(sA[k].y), m);
-                            keep_smaller(cbest[k], cslot[k], __float_as_uint(sB[k].x), m + 1);
-                            keep_smaller(cbest[NBL + k], cslot[NBL + k], __float_as_uint(sB[k].y), m + 1);
-                        }
-                    }
-                } else {
-                    // trip m: the low half evaluates members m and m + 1, the high half finishes
-                    // members m - 2 and m - 1 from the low-half sums of the previous trip
-                    float nDA_prev = cand[0].x, PA_prev = cand[0].z, nDB_prev = nDA_prev, PB_prev = PA_prev;
-                    float carryA = 0.0f, carryB = 0.0f;
-                    for (int m = 0; m < cnt + 2; m += 2) {
-                        const int mm = m < cnt ? m : 0;         // past the end: repeat a trip, low-half result unused
-                        const float4 dpA = cand[mm], dpB = cand[mm + 1];
-                        const float2 nDA = make_float2(dpA.x, nDA_prev), PA = make_float2(dpA.z, PA_prev);
-                        const float2 nDB = make_float2(dpB.x, nDB_prev), PB = make_float2(dpB.z, PB_prev);
-                        float2 sA = make_float2(0.0f, carryA), sB = make_float2(0.0f, carryB);
-#pragma unroll
-                        for (int i = 0; i < NP; ++i) {
-                            const float2 qA = round_e2m1_pair(__fmul2_rn(tb[i], PA));
-                            const float2 qB = round_e2m1_pair(__fmul2_rn(tb[i], PB));
-                            const float2 eA = __ffma2_rn(qA, nDA, v2[i]);
-                            const float2 eB = __ffma2_rn(qB, nDB, v2[i]);
-                            sA = __ffma2_rn(eA, eA, sA);
-                            sB = __ffma2_rn(eB, eB, sB);
-                        }
-                        if (m > 0) {
-                            keep_smaller(cbest[0], cslot[0], __float_as_uint(sA.y), m - 2);
-                            keep_smaller(cbest[0], cslot[0], __float_as_uint(sB.y), m - 1);
-                        }
-                        carryA = sA.x; carryB = sB.x;
-                        nDA_prev = dpA.x; PA_prev = dpA.z; nDB_prev = dpB.x; PB_prev = dpB.z;
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < NBT; ++k)
-                    if (cbest[k] != 0xFFFFFFFFu) merge_class_winner(best[k], cbest[k], T.member[base + cslot[k]]);
+                search_list<B, FMT, false>(T, 2 * cls, v2, tb, best);
+                search_list<B, FMT, true>(T, 2 * cls + 1, v2, tb, best);
             }
         }
 
