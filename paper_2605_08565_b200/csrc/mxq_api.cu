@@ -70,21 +70,10 @@ int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scal
         return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
     }
     const bool dual = (recipe == MXQ_4O6 || recipe == MXQ_4O6_PZ);
-    const size_t chunk = block_size < 8 ? 8 : (size_t)block_size;
-    a.n_items = n / chunk;
-    if (a.n_items > 0) {
-        err = (dtype == MXQ_F32) ? launch_quantize_f32(a, block_size, scale_fmt, dual, s)
-                                 : launch_quantize_bf16(a, block_size, scale_fmt, dual, s);
-        if (err != cudaSuccess) return cuda_fail(err);
-    }
-    const size_t rest = n - a.n_items * chunk;  // < 8 elements, block sizes 2 and 4 only
-    if (rest > 0) {
-        a.first_item = a.n_items * chunk / (size_t)block_size;
-        a.n_items = rest / (size_t)block_size;
-        err = launch_quantize_tail(a, dtype, block_size, scale_fmt, dual, s);
-        if (err != cudaSuccess) return cuda_fail(err);
-    }
-    return MXQ_OK;
+    a.n_items = n / (size_t)block_size;
+    err = (dtype == MXQ_F32) ? launch_quantize_f32(a, block_size, scale_fmt, dual, s)
+                             : launch_quantize_bf16(a, block_size, scale_fmt, dual, s);
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
 }
 
 int mxq_quantize(const float* x, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,

@@ -9,8 +9,8 @@ namespace mxq {
 
 constexpr int kMaxDevices = 64;
 
-// Arguments of the quantization kernels.  n_items counts what one thread owns per loop trip:
-// chunks of max(B, 8) elements for the one-pass kernels, blocks for the search and tail kernels.
+// Arguments of the quantization kernels.  The launchers receive n_items = number of blocks and
+// hand their kernels n_items = what one thread owns per loop trip (chunks of blocks, or blocks).
 struct QuantArgs {
     const void* x;
     size_t n_items;

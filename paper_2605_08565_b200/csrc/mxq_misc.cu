@@ -217,7 +217,8 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Scalar abs-max / 4-over-6 for the blocks past the last whole chunk (at most three blocks).
+// Scalar abs-max / 4-over-6 for the blocks past the last whole per-thread chunk (block sizes up to
+// 16, fewer than 16 blocks).
 // Same arithmetic as the one-pass kernels, general quotient only.
 // ------------------------------------------------------------------------------------------------
 template <int FMT>
@@ -242,7 +243,7 @@ __global__ void k_quantize_tail(QuantArgs p, int dtype, int B, int dual) {
     if (b >= p.n_items) return;
     const size_t blk = p.first_item + b;
     const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    float v[8];
+    float v[16];
     float amax = 0.0f;
     for (int i = 0; i < B; ++i) {
         const size_t e = blk * B + i;
@@ -267,7 +268,7 @@ __global__ void k_quantize_tail(QuantArgs p, int dtype, int B, int dual) {
 }
 
 cudaError_t launch_quantize_tail(const QuantArgs& a, int dtype, int B, int fmt, bool dual, cudaStream_t s) {
-    if (B > 8) return cudaErrorInvalidValue;
+    if (B > 16) return cudaErrorInvalidValue;
     const unsigned grid = (unsigned)((a.n_items + 31) / 32);
     switch (fmt) {
     case kUE8M0: k_quantize_tail<kUE8M0><<<grid, 32, 0, s>>>(a, dtype, B, dual ? 1 : 0); break;

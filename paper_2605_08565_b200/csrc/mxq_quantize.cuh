@@ -1,170 +1,465 @@
 // Fused one-pass quantization kernels: block amax -> scale code -> FP4 codes -> block SSE.
-//   kind SINGLE  abs-max (Eq. 2; Eq. 1 for UE8M0), optional prevent-zero clamp (Eq. 3)
-//   kind DUAL    4-over-6 (Eq. 4): candidates for M = 6 and M = 4, keep the smaller SSE
-// One thread owns a chunk of C = max(B, 8) consecutive elements (one block, or 8/B small
+//   SINGLE  abs-max (Eq. 2; Eq. 1 for UE8M0), optional prevent-zero clamp (Eq. 3)
+//   DUAL    4-over-6 (Eq. 4): candidates for M = 6 and M = 4, keep the smaller SSE
+//
+// Work layout.  One thread owns a chunk of consecutive elements (at least 64 bytes of input and
+// at least one block) and walks it in groups of max(B, 8) elements (one block, or 8/B small
 // blocks), so every per-block quantity lives in registers and the SSE is accumulated in element
-// order.  CTAs are persistent (grid = SMs x resident CTAs) and build the per-code decode-scale
-// tables once in shared memory.
+// order.  CTAs are persistent (grid = SMs x resident CTAs) and build the per-code table once.
+//
+// Input staging.  Every thread copies ITS OWN next chunk into ITS OWN slot of a two-slot
+// shared-memory ring with asynchronous 16-byte copies (cp.async.ca: the 128-byte line that the
+// first piece brings into L1 also serves the thread's other pieces and its neighbour) and waits
+// for it with cp.async.wait_group.  The data never crosses threads, so no barrier of any kind is
+// involved and nothing can wait forever.  One chunk (>= 64 bytes) per thread is in flight while
+// the current one is processed, independent of how many registers the arithmetic needs; a third
+// slot was measured and loses (the extra shared memory leaves too little L1 for fp32 input).
+// Slot layout: piece k of thread t sits at ((slot * PIECES + k) * 256 + t) * 16, so both the
+// asynchronous writes and the later 128-bit reads of a warp are contiguous (no bank conflict).
+//
+// Arithmetic per element (the instruction mix that the issue slots of an SM sub-partition bound):
+// bf16 -> binary32 by a mixed-precision add of -0 (FMA pipe), the exact quotient by the decode
+// scale (reciprocal multiply + one residual correction when every decode scale of the table has a
+// short significand, two corrections otherwise), half an FP4 pack, half an FP4 unpack, and the two
+// FMAs of the SSE -- the first being fma.rn.f32.f16 straight from the unpacked f16 grid value
+// whenever the decode scales of the group are exactly representable in f16 (always, for UE4M3
+// without a tensor scale), else an f16->f32 convert plus an FFMA.  Blocks whose numbers fall
+// outside the ranges these shortcuts need are redone with IEEE divisions (general path).
 #pragma once
+
+#include <cuda_fp16.h>
 
 #include "mxq_device.cuh"
 #include "mxq_internal.h"
 
 namespace mxq {
 
-template <int B, int N>
-__device__ __forceinline__ void block_amax(const float (&v)[N], float (&a)[N / B]) {
+// Per-code table entry, one 128-bit shared-memory read per block and candidate:
+//   x  D = fl32(value(c) * g); NaN for codes that do not exist
+//   y  R = RN(1 / D) when 2^-60 <= D <= 2^60, else 0
+//   z  bits: f16(-D) in the low half
+//   w  0: general path only; 1: shortcuts valid; 2: shortcuts valid and -D exact in f16.
+//      D = 0 counts as valid with R = 0: every quotient comes out as a zero with the sign of v.
+struct QuantTables {
+    float4 E[256];
+    int all_short;   // every entry with w != 0 has a significand of at most 19 bits
+};
+
+template <int FMT>
+__device__ __forceinline__ void build_quant_tables(QuantTables& T, float g) {
+    if (threadIdx.x == 0) T.all_short = 1;
+    __syncthreads();
+    for (int c = threadIdx.x; c < 256; c += blockDim.x) {
+        float D = __uint_as_float(0x7FC00000u), R = 0.0f, w = 0.0f;
+        uint32_t h16 = 0;
+        if (c < num_codes(FMT)) {
+            D = __fmul_rn(scale_value(FMT, c), g);
+            const bool in_range = (D >= kFastMin && D <= kFastMax);
+            if (in_range || D == 0.0f) {
+                if (in_range) R = __frcp_rn(D);
+                const __half hD = __float2half_rn(-D);
+                h16 = (uint32_t)__half_as_ushort(hD);
+                w = (__half2float(hD) == -D) ? 2.0f : 1.0f;
+                if (__float_as_uint(D) & 0x1Fu) T.all_short = 0;   // benign race: every writer stores 0
+            }
+        }
+        T.E[c] = make_float4(D, R, __uint_as_float(h16), w);
+    }
+    __syncthreads();
+}
+
+// fl32(v / D) when the significand of D has at most 19 bits: reciprocal multiply and ONE residual
+// correction.  q0 = RN(v * R) is within 1.5 ulp of v / D, the residual q0 * D - v is then exactly
+// representable, and q0 - r * R differs from v / D by at most 1.5 * 2^-24 ulp before its final
+// rounding; v / D itself stays at least 2^-20 ulp away from every rounding boundary because D has
+// few bits, so that rounding is the correct one.  Range conditions as for quotient_corrected().
+__device__ __forceinline__ float quotient_short(float v, float D, float R) {
+    const float q = __fmul_rn(v, R);
+    const float r = __fmaf_rn(q, D, -v);
+    return __fmaf_rn(-r, R, q);
+}
+
+// fl32(u / 6) by a reciprocal multiply with one correction: exact for this divisor (checked on the
+// host for every binary32 u in [1e-30, 1e30]; 0 maps to 0).  Below that range the residual can
+// underflow and the result may be one ulp off.
+__device__ __forceinline__ float div6_fast(float u) {
+    const float R6 = 0.16666667163372039794921875f;   // RN(1/6)
+    const float q = __fmul_rn(u, R6);
+    const float r = __fmaf_rn(q, -6.0f, u);
+    return __fmaf_rn(r, R6, q);
+}
+
+// Eight quotients -> one word of eight FP4 codes (element 0 in bits 0..3) and the four f16x2
+// words holding the grid values they stand for (element 2k in the low half of h[k]).
+__device__ __forceinline__ uint32_t quantize_e2m1x8_h(const float* t, uint32_t* h) {
+    uint32_t out;
+    asm("{\n"
+        " .reg .b8 b0, b1, b2, b3;\n"
+        " cvt.rn.satfinite.e2m1x2.f32 b0, %6, %5;\n"
+        " cvt.rn.satfinite.e2m1x2.f32 b1, %8, %7;\n"
+        " cvt.rn.satfinite.e2m1x2.f32 b2, %10, %9;\n"
+        " cvt.rn.satfinite.e2m1x2.f32 b3, %12, %11;\n"
+        " cvt.rn.f16x2.e2m1x2 %1, b0;\n"
+        " cvt.rn.f16x2.e2m1x2 %2, b1;\n"
+        " cvt.rn.f16x2.e2m1x2 %3, b2;\n"
+        " cvt.rn.f16x2.e2m1x2 %4, b3;\n"
+        " mov.b32 %0, {b0, b1, b2, b3};\n"
+        "}"
+        : "=r"(out), "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3])
+        : "f"(t[0]), "f"(t[1]), "f"(t[2]), "f"(t[3]), "f"(t[4]), "f"(t[5]), "f"(t[6]), "f"(t[7]));
+    return out;
+}
+
+// e = fma(q, -D, v) for the two grid values of an f16x2 word, with q and -D given in f16: the
+// product is exact and the sum is rounded once to binary32 (mixed-precision FMA).
+__device__ __forceinline__ void residual_pair_f16(uint32_t h, uint32_t nD16, float v0, float v1, float& e0, float& e1) {
+    asm("{\n"
+        " .reg .b16 lo, hi, d, dx;\n"
+        " mov.b32 {lo, hi}, %2;\n"
+        " mov.b32 {d, dx}, %3;\n"
+        " fma.rn.f32.f16 %0, lo, d, %4;\n"
+        " fma.rn.f32.f16 %1, hi, d, %5;\n"
+        "}"
+        : "=f"(e0), "=f"(e1)
+        : "r"(h), "r"(nD16), "f"(v0), "f"(v1));
+}
+
+template <int DT, int B>
+struct QuantShape {
+    static constexpr int EB = elem_bytes(DT);
+    static constexpr int C = (B * EB >= 64) ? B : 64 / EB;   // elements per thread-chunk (>= 64 bytes)
+    static constexpr int GE = (B < 8) ? 8 : B;               // elements per group
+    static constexpr int NG = C / GE;                        // groups per chunk
+    static constexpr int NBG = GE / B;                       // blocks per group
+    static constexpr int NBC = C / B;                        // blocks per chunk
+    static constexpr int PIECES = C * EB / 16;               // 16-byte pieces per chunk
+    static constexpr int SLOTS = 2;                          // ring depth per thread
+    static constexpr size_t RING_BYTES = (size_t)SLOTS * PIECES * 16 * kThreads;
+};
+
+// raw words -> binary32.  bf16 goes through the FMA pipe (mixed-precision add of -0, which keeps
+// the sign of a zero and every denormal) and leaves the integer pipe to the FP4 converts.
+template <int DT, int N>
+__device__ __forceinline__ void widen(const uint32_t* w, float* v) {
+    if constexpr (DT == kF32) {
 #pragma unroll
-    for (int j = 0; j < N / B; ++j) {
-        float m = 0.0f;
+        for (int i = 0; i < N; ++i) v[i] = __uint_as_float(w[i]);
+    } else {
 #pragma unroll
-        for (int i = 0; i < B; ++i) m = fmaxf(m, fabsf(v[j * B + i]));
-        a[j] = m;
+        for (int i = 0; i < N / 2; ++i) {
+            asm("{\n"
+                " .reg .b16 lo, hi;\n"
+                " mov.b32 {lo, hi}, %2;\n"
+                " add.rn.f32.bf16 %0, lo, %3;\n"
+                " add.rn.f32.bf16 %1, hi, %3;\n"
+                "}"
+                : "=f"(v[2 * i]), "=f"(v[2 * i + 1])
+                : "r"(w[i]), "f"(-0.0f));
+        }
     }
 }
 
-// Quantize the C elements of a chunk with one scale code per block; returns packed codes and
-// per-block SSE (e = fma(-q, D, v); sse = fma(e, e, sse), in element order).
-template <int B, int C>
-__device__ __forceinline__ void encode_chunk(const float (&v)[C], const float (&amax)[C / B], const int (&code)[C / B],
-                                             const float* tabD, const float* tabR, uint32_t (&packed)[C / 8],
-                                             float (&sse)[C / B]) {
-    constexpr int NB = C / B;
-    float t[C];
-    float D[NB];
+// Pack a group's quotients (GE / 8 code words) and accumulate the per-block SSE
+// (e = fma(-q, D, v); sse = fma(e, e, sse), in element order).
+template <int B, bool HALF>
+__device__ __forceinline__ void pack_and_score(const float* v, const float* t, const float4* E, uint32_t* packed,
+                                               float* sse) {
+    constexpr int GE = (B < 8) ? 8 : B;
+    constexpr int NBG = GE / B;
+    uint32_t h[GE / 2];
 #pragma unroll
-    for (int j = 0; j < NB; ++j) {
-        D[j] = tabD[code[j]];
-        const float R = tabR[code[j]];
-        if (R != 0.0f && amax[j] <= kFastMax) {
+    for (int k = 0; k < GE / 8; ++k) packed[k] = quantize_e2m1x8_h(&t[8 * k], &h[4 * k]);
 #pragma unroll
-            for (int i = 0; i < B; ++i) t[j * B + i] = quotient_corrected(v[j * B + i], D[j], R);
-        } else {
-#pragma unroll
-            for (int i = 0; i < B; ++i) t[j * B + i] = quotient_general(v[j * B + i], D[j]);
-        }
-    }
-    float q[C];
-#pragma unroll
-    for (int k = 0; k < C / 8; ++k) {
-        float q8[8];
-        packed[k] = quantize_e2m1x8(&t[8 * k], q8);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) q[8 * k + i] = q8[i];
-    }
-#pragma unroll
-    for (int j = 0; j < NB; ++j) {
+    for (int j = 0; j < NBG; ++j) {
         float s = 0.0f;
+        if constexpr (HALF) {
+            const uint32_t nD16 = __float_as_uint(E[j].z);
 #pragma unroll
-        for (int i = 0; i < B; ++i) {
-            const float e = __fmaf_rn(-q[j * B + i], D[j], v[j * B + i]);
-            s = __fmaf_rn(e, e, s);
+            for (int i = 0; i < B; i += 2) {
+                float e0, e1;
+                residual_pair_f16(h[(j * B + i) / 2], nD16, v[j * B + i], v[j * B + i + 1], e0, e1);
+                s = __fmaf_rn(e0, e0, s);
+                s = __fmaf_rn(e1, e1, s);
+            }
+        } else {
+            const float nD = -E[j].x;
+#pragma unroll
+            for (int i = 0; i < B; i += 2) {
+                const float2 q = __half22float2(*reinterpret_cast<const __half2*>(&h[(j * B + i) / 2]));
+                const float e0 = __fmaf_rn(q.x, nD, v[j * B + i]);
+                s = __fmaf_rn(e0, e0, s);
+                const float e1 = __fmaf_rn(q.y, nD, v[j * B + i + 1]);
+                s = __fmaf_rn(e1, e1, s);
+            }
         }
         sse[j] = s;
     }
 }
 
-template <int DT, int B, int FMT, bool DUAL>
-__global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
-    constexpr int C = (B < 8) ? 8 : B;
-    constexpr int NB = C / B;
-    __shared__ float tabD[256];
-    __shared__ float tabR[256];
-    const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    build_scale_tables<FMT>(tabD, tabR, g);
-    const bool unit_g = (g == 1.0f);
-    const bool pz = p.prevent_zero && FMT != kUE8M0;
-
-    const size_t stride = (size_t)gridDim.x * kThreads;
-    for (size_t chunk = (size_t)blockIdx.x * kThreads + threadIdx.x; chunk < p.n_items; chunk += stride) {
-        float v[C];
-        load_elems<DT, C>(p.x, chunk * C, v);
-        float amax[NB];
-        block_amax<B, C>(v, amax);
-
-        int c6[NB];
-        float u[NB];
+// One candidate set of a group with the shortcuts (every entry has w != 0, magnitudes in range).
+template <int B>
+__device__ __forceinline__ void encode_group_fast(const float* v, const float4* E, bool all_short, bool all_half,
+                                                  uint32_t* packed, float* sse) {
+    constexpr int GE = (B < 8) ? 8 : B;
+    constexpr int NBG = GE / B;
+    float t[GE];
+    if (all_short) {
 #pragma unroll
-        for (int j = 0; j < NB; ++j) {
-            u[j] = unit_g ? amax[j] : __fdiv_rn(amax[j], g);
-            c6[j] = round_scale<FMT>(__fdiv_rn(u[j], 6.0f));
-            if (pz) c6[j] = max(c6[j], 1);
-        }
-        uint32_t packed[C / 8];
-        float sse[NB];
-        encode_chunk<B, C>(v, amax, c6, tabD, tabR, packed, sse);
-
-        if constexpr (DUAL) {
-            int c4[NB];
-            bool any = false;
+        for (int j = 0; j < NBG; ++j)
 #pragma unroll
-            for (int j = 0; j < NB; ++j) {
-                c4[j] = round_scale<FMT>(__fdiv_rn(u[j], 4.0f));
-                if (pz) c4[j] = max(c4[j], 1);
-                any |= (c4[j] != c6[j]);
-            }
-            if (any) {
-                uint32_t packed4[C / 8];
-                float sse4[NB];
-                encode_chunk<B, C>(v, amax, c4, tabD, tabR, packed4, sse4);
-                if constexpr (NB == 1) {
-                    if (sse4[0] < sse[0]) {
-                        sse[0] = sse4[0];
-                        c6[0] = c4[0];
+            for (int i = 0; i < B; ++i) t[j * B + i] = quotient_short(v[j * B + i], E[j].x, E[j].y);
+    } else {
 #pragma unroll
-                        for (int k = 0; k < C / 8; ++k) packed[k] = packed4[k];
-                    }
-                } else {
-                    // several blocks share the one 32-bit code word: select by bit mask
-                    constexpr uint32_t kBlockMask = (B == 2) ? 0xFFu : 0xFFFFu;
-                    uint32_t take = 0;
+        for (int j = 0; j < NBG; ++j)
 #pragma unroll
-                    for (int j = 0; j < NB; ++j) {
-                        if (sse4[j] < sse[j]) {
-                            sse[j] = sse4[j];
-                            c6[j] = c4[j];
-                            take |= kBlockMask << (j * 4 * B);
-                        }
-                    }
-                    packed[0] = (packed4[0] & take) | (packed[0] & ~take);
-                }
-            }
-        }
-
-        store_bytes<C / 2>(p.codes + chunk * (C / 2), packed);
-        uint32_t sc = 0;
-#pragma unroll
-        for (int j = 0; j < NB; ++j) sc |= (uint32_t)c6[j] << (8 * j);
-        store_bytes<NB>(p.scales + chunk * NB, &sc);
-        if (p.block_sse) {
-            uint32_t sw[NB];
-#pragma unroll
-            for (int j = 0; j < NB; ++j) sw[j] = __float_as_uint(sse[j]);
-            store_bytes<4 * NB>(p.block_sse + chunk * NB, sw);
-        }
+            for (int i = 0; i < B; ++i) t[j * B + i] = quotient_corrected(v[j * B + i], E[j].x, E[j].y);
     }
+    if (all_half) pack_and_score<B, true>(v, t, E, packed, sse);
+    else pack_and_score<B, false>(v, t, E, packed, sse);
 }
 
-// Host side: pick the instantiation and launch a persistent grid.
+// One candidate set of a group on the general path (IEEE division; zero scale -> signed zeros).
+template <int B>
+__device__ __forceinline__ void encode_group_general(const float* v, const float4* E, uint32_t* packed, float* sse) {
+    constexpr int GE = (B < 8) ? 8 : B;
+    constexpr int NBG = GE / B;
+    float t[GE];
+#pragma unroll
+    for (int j = 0; j < NBG; ++j)
+#pragma unroll
+        for (int i = 0; i < B; ++i) t[j * B + i] = quotient_general(v[j * B + i], E[j].x);
+    pack_and_score<B, false>(v, t, E, packed, sse);
+}
+
+// CTA-uniform constants of a launch.
+struct QuantConsts {
+    float g, Rg;        // tensor scale and RN(1 / g)
+    float m_lo, m_hi;   // a block maximum m takes the shortcuts when m == 0 or m_lo <= m <= m_hi
+    bool unit_g, need_lo, pz, all_short;
+};
+
+template <int DT, int B, int FMT, bool DUAL>
+__device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
+                                               size_t chunk, const uint32_t* raw) {
+    using S = QuantShape<DT, B>;
+    constexpr int NBG = S::NBG;
+    uint32_t packed[S::C / 8];
+    uint32_t sc[(S::NBC + 3) / 4];
+    uint32_t sw[S::NBC];
+#pragma unroll
+    for (int i = 0; i < (S::NBC + 3) / 4; ++i) sc[i] = 0;
+
+#pragma unroll
+    for (int gi = 0; gi < S::NG; ++gi) {
+        float v[S::GE];
+        widen<DT, S::GE>(raw + gi * (S::GE * S::EB / 4), v);
+        float m[NBG], u[NBG];
+        int c6[NBG], c4[NBG];
+        float4 E6[NBG], E4[NBG];
+        float wmin = 2.0f, mmax = 0.0f, mmin = k.m_hi;
+#pragma unroll
+        for (int j = 0; j < NBG; ++j) {
+            float a = 0.0f;
+#pragma unroll
+            for (int i = 0; i < B; ++i) a = fmaxf(a, fabsf(v[j * B + i]));
+            m[j] = a;
+            mmax = fmaxf(mmax, a);
+            if (k.need_lo) mmin = fminf(mmin, a == 0.0f ? k.m_hi : a);
+            u[j] = k.unit_g ? a : quotient_corrected(a, k.g, k.Rg);
+            c6[j] = round_scale<FMT>(div6_fast(u[j]));
+            if (k.pz) c6[j] = max(c6[j], 1);
+            E6[j] = T.E[c6[j]];
+            wmin = fminf(wmin, E6[j].w);
+            if constexpr (DUAL) {
+                c4[j] = round_scale<FMT>(__fmul_rn(u[j], 0.25f));
+                if (k.pz) c4[j] = max(c4[j], 1);
+                E4[j] = T.E[c4[j]];
+                wmin = fminf(wmin, E4[j].w);
+            }
+        }
+        uint32_t pk[S::GE / 8], pk4[S::GE / 8];
+        float sse[NBG], sse4[NBG];
+        if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
+            encode_group_fast<B>(v, E6, k.all_short, wmin >= 2.0f, pk, sse);
+            if constexpr (DUAL) encode_group_fast<B>(v, E4, k.all_short, wmin >= 2.0f, pk4, sse4);
+        } else {
+#pragma unroll
+            for (int j = 0; j < NBG; ++j) {
+                u[j] = __fdiv_rn(m[j], k.g);
+                c6[j] = round_scale<FMT>(__fdiv_rn(u[j], 6.0f));
+                if (k.pz) c6[j] = max(c6[j], 1);
+                E6[j] = T.E[c6[j]];
+                if constexpr (DUAL) {
+                    c4[j] = round_scale<FMT>(__fmul_rn(u[j], 0.25f));
+                    if (k.pz) c4[j] = max(c4[j], 1);
+                    E4[j] = T.E[c4[j]];
+                }
+            }
+            encode_group_general<B>(v, E6, pk, sse);
+            if constexpr (DUAL) encode_group_general<B>(v, E4, pk4, sse4);
+        }
+
+        if constexpr (DUAL) {
+            if constexpr (NBG == 1) {
+                const bool take = sse4[0] < sse[0];
+                sse[0] = take ? sse4[0] : sse[0];
+                c6[0] = take ? c4[0] : c6[0];
+#pragma unroll
+                for (int i = 0; i < S::GE / 8; ++i) pk[i] = take ? pk4[i] : pk[i];
+            } else {
+                // several blocks share the one 32-bit code word: select by bit mask
+                constexpr uint32_t kBlockMask = (B == 2) ? 0xFFu : 0xFFFFu;
+                uint32_t take = 0;
+#pragma unroll
+                for (int j = 0; j < NBG; ++j) {
+                    const bool tj = sse4[j] < sse[j];
+                    sse[j] = tj ? sse4[j] : sse[j];
+                    c6[j] = tj ? c4[j] : c6[j];
+                    take |= tj ? (kBlockMask << (j * 4 * B)) : 0u;
+                }
+                pk[0] = (pk4[0] & take) | (pk[0] & ~take);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < S::GE / 8; ++i) packed[gi * (S::GE / 8) + i] = pk[i];
+#pragma unroll
+        for (int j = 0; j < NBG; ++j) {
+            const int b = gi * NBG + j;
+            sc[b / 4] |= (uint32_t)c6[j] << (8 * (b % 4));
+            sw[b] = __float_as_uint(sse[j]);
+        }
+    }
+    store_bytes<S::C / 2>(p.codes + chunk * (S::C / 2), packed);
+    store_bytes<S::NBC>(p.scales + chunk * S::NBC, sc);
+    if (p.block_sse) store_bytes<4 * S::NBC>(p.block_sse + chunk * S::NBC, sw);
+}
+
+// Asynchronous copy of one chunk (PIECES x 16 bytes) from global memory into this thread's pieces
+// of a ring slot (piece k of thread t at ((slot * PIECES + k) * 256 + t) * 16), as one commit
+// group.  An empty group is committed when there is no chunk left, so that the group count per
+// loop trip stays fixed.
+template <int PIECES>
+__device__ __forceinline__ void stage_chunk(uint32_t slot_addr, const void* src, bool valid) {
+    if (valid) {
+        const char* g = static_cast<const char*>(src);
+#pragma unroll
+        for (int k = 0; k < PIECES; ++k)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(slot_addr + k * (kThreads * 16)), "l"(g + 16 * k)
+                         : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+template <int DT, int B, int FMT, bool DUAL>
+__global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
+    using S = QuantShape<DT, B>;
+    extern __shared__ uint4 ring[];
+    __shared__ QuantTables T;
+    QuantConsts k;
+    k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
+    build_quant_tables<FMT>(T, k.g);
+    k.unit_g = (k.g == 1.0f);
+    k.pz = p.prevent_zero && FMT != kUE8M0;
+    k.all_short = T.all_short != 0;
+    k.Rg = 1.0f;
+    // Ranges of a block maximum m for which u = fl(m / g) and fl(u / 6) come out exact from the
+    // multiply-and-correct forms.  The FP8 formats round every u below 2^-20 to code 0, so an
+    // inexact tiny quotient cannot change their code; the power-of-two format reads the exponent
+    // of the quotient and needs it exact.
+    k.need_lo = (FMT == kUE8M0) || !k.unit_g;
+    k.m_hi = kFastMax;
+    k.m_lo = 0.0f;
+    if (k.unit_g) {
+        if (FMT == kUE8M0) k.m_lo = 1.0e-30f;
+    } else if (k.g >= kFastMin && k.g <= kFastMax) {
+        k.Rg = __frcp_rn(k.g);
+        k.m_hi = fminf(kFastMax, __fmul_rn(k.g, 1.0e29f));
+        k.m_lo = fmaxf(1.084202172485504434e-19f /* 2^-63 */, (FMT == kUE8M0) ? __fmul_rn(k.g, 1.0e-29f) : 0.0f);
+    } else {
+        k.m_hi = -1.0f;   // tensor scale outside the shortcut range: general path everywhere
+        k.m_lo = 0.0f;
+    }
+
+    const size_t stride = (size_t)gridDim.x * kThreads;
+    size_t chunk = (size_t)blockIdx.x * kThreads + threadIdx.x;
+    if (chunk >= p.n_items) return;   // no barrier follows
+    constexpr size_t kChunkBytes = (size_t)S::C * S::EB;
+    constexpr uint32_t kSlotBytes = S::PIECES * kThreads * 16;
+    constexpr int DIST = S::SLOTS - 1;   // chunks requested ahead of the one being processed
+    const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(ring) + threadIdx.x * 16;
+    const char* x = static_cast<const char*>(p.x);
+    {   // prologue: request the first DIST chunks
+        size_t c = chunk;
+#pragma unroll
+        for (int d = 0; d < DIST; ++d) {
+            stage_chunk<S::PIECES>(ring_base + d * kSlotBytes, x + c * kChunkBytes, c < p.n_items);
+            c += stride;
+        }
+    }
+    int slot = 0;                      // slot holding `chunk`
+    int fill = DIST % S::SLOTS;        // slot that the next request goes to
+    size_t ahead = chunk + (size_t)DIST * stride;
+    for (; chunk < p.n_items; chunk += stride) {
+        // all but the DIST - 1 most recent groups are complete: this thread's copy of `chunk` has landed
+        asm volatile("cp.async.wait_group %0;" ::"n"(DIST - 1) : "memory");
+        uint32_t raw[S::PIECES * 4];
+        const uint4* src = ring + (size_t)slot * (S::PIECES * kThreads) + threadIdx.x;
+#pragma unroll
+        for (int q = 0; q < S::PIECES; ++q) {
+            const uint4 w = src[q * kThreads];
+            raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
+        }
+        // the slot read one trip ago is free again (its words were consumed by the arithmetic of
+        // that trip): request the chunk DIST trips ahead into it
+        stage_chunk<S::PIECES>(ring_base + fill * kSlotBytes, x + ahead * kChunkBytes, ahead < p.n_items);
+        ahead += stride;
+        slot = (slot + 1 == S::SLOTS) ? 0 : slot + 1;
+        fill = (fill + 1 == S::SLOTS) ? 0 : fill + 1;
+        quantize_chunk<DT, B, FMT, DUAL>(p, T, k, chunk, raw);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+// Host side: pick the instantiation, launch a persistent grid over the whole chunks and hand the
+// blocks past the last whole chunk to the scalar tail kernel.
 template <int DT, int B, int FMT, bool DUAL>
 static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream) {
+    using S = QuantShape<DT, B>;
     static int ctas_per_sm[kMaxDevices] = {0};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (ctas_per_sm[dev] == 0) {
+        err = cudaFuncSetAttribute(k_quantize<DT, B, FMT, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)S::RING_BYTES);
+        if (err != cudaSuccess) return err;
         int n = 0;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_quantize<DT, B, FMT, DUAL>, kThreads, 0);
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_quantize<DT, B, FMT, DUAL>, kThreads, S::RING_BYTES);
         if (err != cudaSuccess) return err;
         ctas_per_sm[dev] = n > 0 ? n : 1;
     }
-    const size_t want = (a.n_items + kThreads - 1) / kThreads;
-    const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
-    const unsigned grid = (unsigned)(want < cap ? want : cap);
-    k_quantize<DT, B, FMT, DUAL><<<grid, kThreads, 0, stream>>>(a);
-    count_launch();
-    return cudaGetLastError();
+    const size_t n_blocks = a.n_items;
+    const size_t n_chunks = n_blocks / S::NBC;
+    if (n_chunks > 0) {
+        QuantArgs m = a;
+        m.n_items = n_chunks;
+        const size_t want = (n_chunks + kThreads - 1) / kThreads;
+        const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
+        const unsigned grid = (unsigned)(want < cap ? want : cap);
+        k_quantize<DT, B, FMT, DUAL><<<grid, kThreads, S::RING_BYTES, stream>>>(m);
+        count_launch();
+        err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+    }
+    const size_t done = n_chunks * S::NBC;
+    if (done < n_blocks) {
+        QuantArgs t = a;
+        t.first_item = done;
+        t.n_items = n_blocks - done;
+        err = launch_quantize_tail(t, DT, B, FMT, DUAL, stream);
+    }
+    return err;
 }
 
 template <int DT, int B, int FMT>
