@@ -45,6 +45,15 @@ RECIPE_NAME = {ABSMAX: "absmax", ABSMAX_PZ: "absmax_pz", R4O6: "4o6", BRUTE: "br
 N_CODES_UE4M3 = 127
 ALU_LANES_PER_SM = 128            # 4 schedulers x 32 lanes, one instruction per scheduler per clock
 CPU_SAMPLE_ELEMS = 1 << 20
+STREAM_ELEMS = 1 << 27            # tensor size of the streaming (HBM-bound) kernel measurements
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (same kernel build, same launch configuration); set an entry to None when its kernel changes.
+NCU_TRAFFIC_BYTES = {
+    "k_brute<bf16,B=16,UE4M3>@16Mi": 33.609984e6 + 7.68e3,
+    "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.478720e6 + 81.633280e6,
+    "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi": 268.494592e6 + 83.002624e6,
+    "k_quantize<f32,B=16,UE4M3,absmax>@128Mi": 536.896512e6 + 94.908672e6,
+}
 
 
 def pass_list():
@@ -235,6 +244,41 @@ def algorithmic_bytes(n: int, elem_bytes: int, B: int) -> float:
     return n * (elem_bytes + 0.5 + 5.0 / B)
 
 
+def streaming_rooflines(torch, mxq, device, peaks):
+    """HBM-bound kernels on a tensor far larger than L2 (134M elements), ten launches back to back
+    per CUDA-event pair, outside the timed region of the step: the 16.8M-element launches of the
+    step itself last 8-20 us and are dominated by launch ramp."""
+    from paper_2605_08565_b200 import inputs
+    out = {}
+    n = STREAM_ELEMS
+    codes, scales, sse = mxq.alloc_outputs(n, 16, device)
+    for name, dt, recipe, key in (
+            ("absmax_bf16_B16", torch.bfloat16, ABSMAX, "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi"),
+            ("4o6_bf16_B16", torch.bfloat16, R4O6, "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi"),
+            ("absmax_f32_B16", torch.float32, ABSMAX, "k_quantize<f32,B=16,UE4M3,absmax>@128Mi")):
+        x = inputs.student_t(n, 5, 0.02, 2, dt, device)
+        fn = lambda: mxq.mxq_quantize_ex(x, n, 16, UE4M3, recipe, 1.0, None, codes, scales, sse)
+        for _ in range(3):
+            fn()
+        times = []
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) / 10)
+        ms = statistics.median(times)
+        ach = algorithmic_bytes(n, x.element_size(), 16) / (ms * 1e-3) / 1e9
+        out[name] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0,
+                     "traffic": NCU_TRAFFIC_BYTES[key], "ms_per_launch": ms, "gelem_s": n / (ms * 1e-3) / 1e9,
+                     "elems": n, "peak_source": peaks["source"], "l2": "input larger than L2"}
+        del x
+    return out
+
+
 def run_gpu(args) -> None:
     import torch
     from paper_2605_08565_b200 import binding as mxq
@@ -312,7 +356,8 @@ def run_gpu(args) -> None:
     brute_ops = N_ELEM * N_CODES_UE4M3 * 4.0                                            # 4 lane-ops per element-code
     brute_ach = brute_ops / (brute_ms * 1e-3) / 1e12
     roofline = {"kernel": "k_brute<bf16,B=16,UE4M3>", "bound": "alu", "achieved": brute_ach, "peak": alu_peak_max,
-                "unit": "Tlaneop/s", "frac": brute_ach / alu_peak_max, "traffic": None,
+                "unit": "Tlaneop/s", "frac": brute_ach / alu_peak_max,
+                "traffic": NCU_TRAFFIC_BYTES["k_brute<bf16,B=16,UE4M3>@16Mi"],
                 "peak_source": f"{n_sm} SMs x 128 lanes x {peaks['sm_max_mhz']:.0f} MHz (max SM clock, {peaks['source']})",
                 "frac_at_observed_clock": brute_ach / (n_sm * ALU_LANES_PER_SM * sm_mhz * 1e6 / 1e12),
                 "ms_per_launch": brute_ms}
@@ -323,6 +368,7 @@ def run_gpu(args) -> None:
         hbm[name] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0, "traffic": None,
                      "ms_per_launch": ms, "gelem_s": N_ELEM / (ms * 1e-3) / 1e9, "peak_source": peaks["source"]}
+    streaming = streaming_rooflines(torch, mxq, device, peaks)
     per_recipe = {"brute_B16": N_ELEM / (brute_ms * 1e-3) / 1e9, "absmax_B16": hbm["absmax_B16"]["gelem_s"],
                   "4o6_B16": hbm["4o6_B16"]["gelem_s"]}
 
@@ -346,7 +392,8 @@ def run_gpu(args) -> None:
                                "+ hierarchical leg (amax, g, abs-max B=16, MSE) + dequantize",
                    "elements_per_step": wl.elems_per_step, "passes_per_step": len(wl.passes) + 1,
                    "l2": f"inputs rotate over {N_ROTATE} tensors (256 MiB) > 126 MB L2"},
-        "roofline": roofline, "roofline_hbm": hbm, "per_recipe_gelem_s": per_recipe,
+        "roofline": roofline, "roofline_hbm": hbm, "roofline_hbm_streaming": streaming,
+        "per_recipe_gelem_s": per_recipe,
         "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(host_in.numel() * 2),
                 "d2h_bytes_per_step": int(host_out.numel() * 8)},
@@ -422,7 +469,7 @@ def main() -> None:
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--global-scale", type=float, default=1.0)
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="mxq", choices=["mxq", "reference"])
     args = ap.parse_args()

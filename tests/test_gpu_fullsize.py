@@ -1,0 +1,167 @@
+"""GPU parity at the full sizes of the benchmark configurations, in the launch configuration the
+benchmark times (whole tensors, persistent grids): the CPU oracle cannot quantize these tensors
+whole in a test's time, so it computes sampled blocks one by one (blocks are independent given the
+tensor scale) and the rest is covered by properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mxq_oracle as orc
+from paper_2605_08565_b200 import binding as mxq
+from paper_2605_08565_b200 import dist, inputs
+
+pytestmark = pytest.mark.gpu
+
+ABSMAX, ABSMAX_PZ, R4O6, BRUTE = mxq.MXQ_ABSMAX, mxq.MXQ_ABSMAX_PZ, mxq.MXQ_4O6, mxq.MXQ_BRUTE
+
+
+def _sample_blocks(n_blocks, k, seed):
+    rng = np.random.default_rng(seed)
+    edge = np.concatenate([np.arange(min(96, n_blocks)), np.arange(max(0, n_blocks - 96), n_blocks)])
+    pick = rng.integers(0, n_blocks, size=k)
+    return np.unique(np.concatenate([edge, pick]))
+
+
+def _check_sampled(x, B, fmt, recipe, g, codes, scales, sse, k, seed):
+    """Oracle on the sampled blocks (gathered into one short tensor) against the GPU outputs."""
+    n_blocks = x.numel() // B
+    idx = _sample_blocks(n_blocks, k, seed)
+    t_idx = torch.from_numpy(idx).cuda()
+    xs = x.view(n_blocks, B)[t_idx].contiguous().view(-1)
+    oc, os_, oe = orc.quantize(inputs.to_numpy_bits(xs), B, fmt, recipe, g, threads=8)
+    gc = codes.view(n_blocks, B // 2)[t_idx].cpu().numpy().reshape(-1)
+    gs = scales[t_idx].cpu().numpy()
+    ge = sse[t_idx].cpu().numpy()
+    bad = np.flatnonzero(gs != os_)
+    assert bad.size == 0, f"scale bytes differ at sampled blocks {idx[bad[:8]]}: gpu={gs[bad[:8]]} oracle={os_[bad[:8]]}"
+    bad = np.flatnonzero(gc != oc)
+    assert bad.size == 0, f"code bytes differ in sampled blocks {idx[bad[:8] // (B // 2)]}"
+    bad = np.flatnonzero(ge.view(np.uint32) != oe.view(np.uint32))
+    assert bad.size == 0, f"block SSE differs at sampled blocks {idx[bad[:8]]}"
+
+
+def _mse_matches_sum(sse, n):
+    got = float(mxq.tensor_mse(sse, n).cpu()[0])
+    want = float(sse.double().sum().cpu()) / n       # another binary64 summation order
+    assert abs(got - want) <= 1e-6 * want
+    return got
+
+
+def test_weight_sweep_tensor_4096x4096_bf16_all_block_sizes():
+    """The tensor and the passes of the default benchmark step (seeded exactly as bench.py does)."""
+    n = 4096 * 4096
+    x = inputs.student_t(n, 5, 0.02, dist.rank_seed(2, 0, 0), torch.bfloat16, "cuda")
+    mse = {}
+    for B in (2, 4, 8, 16, 32, 64):
+        out = {}
+        for recipe in (ABSMAX, ABSMAX_PZ, R4O6, BRUTE):
+            codes, scales, sse = mxq.quantize(x, B, mxq.MXQ_SF_UE4M3, recipe)
+            torch.cuda.synchronize()
+            _check_sampled(x, B, mxq.MXQ_SF_UE4M3, recipe, 1.0, codes, scales, sse, 1500 if recipe != BRUTE else 400,
+                           100 * B + recipe)
+            out[recipe] = sse
+            mse[(B, recipe)] = _mse_matches_sum(sse, n)
+        # candidate sets nest, and the SSE is one function of (block, code): bitwise orderings
+        assert bool((out[BRUTE] <= out[R4O6]).all()) and bool((out[R4O6] <= out[ABSMAX]).all())
+        assert bool((out[ABSMAX_PZ] <= out[ABSMAX]).all())
+    # finer is better for the optimal scale (Results, numerical study): exact arithmetic would make it
+    # monotone; binary32 sums of different lengths get a little slack
+    bs = (2, 4, 8, 16, 32, 64)
+    for a, b in zip(bs[:-1], bs[1:]):
+        assert mse[(a, BRUTE)] <= mse[(b, BRUTE)] * (1 + 1e-6)
+
+
+def test_hierarchical_leg_of_the_benchmark_step():
+    n = 4096 * 4096
+    x = inputs.student_t(n, 5, 0.02, dist.rank_seed(2, 0, 1), torch.bfloat16, "cuda")
+    amax = torch.empty(1, dtype=torch.float32, device="cuda")
+    dg = torch.empty(1, dtype=torch.float32, device="cuda")
+    mxq.mxq_tensor_amax(x, n, amax, dg)
+    torch.cuda.synchronize()
+    assert float(amax.cpu()[0]) == float(x.float().abs().max().cpu())
+    g = float(dg.cpu()[0])
+    assert g == mxq.mxq_global_scale_from_amax(float(amax.cpu()[0]))
+    for recipe in (ABSMAX, R4O6):
+        codes, scales, sse = mxq.quantize(x, 16, mxq.MXQ_SF_UE4M3, recipe, 1.0, dg)
+        torch.cuda.synchronize()
+        _check_sampled(x, 16, mxq.MXQ_SF_UE4M3, recipe, g, codes, scales, sse, 3000, 7 + recipe)
+        _mse_matches_sum(sse, n)
+    # de-quantization of the whole tensor: every element is grid value times decode scale
+    xh = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    mxq.mxq_dequantize(codes, scales, n, 16, mxq.MXQ_SF_UE4M3, g, xh)
+    torch.cuda.synchronize()
+    idx = _sample_blocks(n // 16, 2000, 5)
+    t_idx = torch.from_numpy(idx).cuda()
+    want = orc.dequantize(codes.view(-1, 8)[t_idx].cpu().numpy().reshape(-1), scales[t_idx].cpu().numpy(), idx.size * 16,
+                          16, orc.UE4M3, g, orc.BF16)
+    got = inputs.to_numpy_bits(xh.view(-1, 16)[t_idx].contiguous())
+    assert np.array_equal(got, want.view(np.uint16))
+
+
+def test_activation_shaped_8192x4096_bf16_outlier_columns():
+    x = inputs.outlier_columns(8192, 4096, 3, dtype=torch.bfloat16, device="cuda")
+    n = x.numel()
+    amax = torch.empty(1, dtype=torch.float32, device="cuda")
+    dg = torch.empty(1, dtype=torch.float32, device="cuda")
+    mxq.mxq_tensor_amax(x, n, amax, dg)
+    torch.cuda.synchronize()
+    g = float(dg.cpu()[0])
+    for fmt, gg, d in ((mxq.MXQ_SF_UE4M3, g, dg), (mxq.MXQ_SF_UE5M3, 1.0, None)):
+        sses = {}
+        for recipe in (ABSMAX, R4O6):
+            codes, scales, sse = mxq.quantize(x, 16, fmt, recipe, 1.0, d)
+            torch.cuda.synchronize()
+            _check_sampled(x, 16, fmt, recipe, gg, codes, scales, sse, 3000, 31 + fmt + recipe)
+            _mse_matches_sum(sse, n)
+            sses[recipe] = sse
+        assert bool((sses[R4O6] <= sses[ABSMAX]).all())
+
+
+@pytest.mark.parametrize("name,rows,cols", [s for s in inputs.LLAMA8B_LAYER_SHAPES if s[0] in ("q", "k", "gate", "down")])
+def test_llama_shaped_weight_matrices_bf16(name, rows, cols):
+    """One matrix of each distinct shape of the Llama-3-8B-shaped set, all recipes, both FP8 scale formats."""
+    index = [s[0] for s in inputs.LLAMA8B_LAYER_SHAPES].index(name)
+    x = inputs.student_t(rows * cols, 4, 1.0 / np.sqrt(cols), 4 + index, torch.bfloat16, "cuda")
+    n = x.numel()
+    for fmt in (mxq.MXQ_SF_UE4M3, mxq.MXQ_SF_UE5M3):
+        best = {}
+        for B in (8, 16):
+            out = {}
+            for recipe in (ABSMAX, ABSMAX_PZ, R4O6, BRUTE):
+                codes, scales, sse = mxq.quantize(x, B, fmt, recipe)
+                torch.cuda.synchronize()
+                _check_sampled(x, B, fmt, recipe, 1.0, codes, scales, sse, 1000 if recipe != BRUTE else 250,
+                               B + fmt + recipe + index)
+                out[recipe] = sse
+            assert bool((out[BRUTE] <= out[R4O6]).all()) and bool((out[R4O6] <= out[ABSMAX]).all())
+            best[B] = _mse_matches_sum(out[BRUTE], n)
+        assert best[8] <= best[16] * (1 + 1e-6)
+
+
+@pytest.fixture(scope="module")
+def laplace_16384x16384():
+    n = 16384 * 16384
+    x = inputs.laplace(n, 5, torch.float32, "cuda")
+    amax = torch.empty(1, dtype=torch.float32, device="cuda")
+    dg = torch.empty(1, dtype=torch.float32, device="cuda")
+    mxq.mxq_tensor_amax(x, n, amax, dg)
+    torch.cuda.synchronize()
+    return x, dg, float(dg.cpu()[0])
+
+
+@pytest.mark.parametrize("fmt", [mxq.MXQ_SF_UE8M0, mxq.MXQ_SF_UE4M3, mxq.MXQ_SF_UE5M3])
+def test_bulk_brute_force_16384x16384_fp32_laplace_with_tensor_scale(laplace_16384x16384, fmt):
+    """The bulk scale-search case at full size: every block size, full code sweep per block."""
+    x, dg, g = laplace_16384x16384
+    n = x.numel()
+    prev = None
+    for B in (2, 4, 8, 16, 32):
+        codes, scales, sse = mxq.quantize(x, B, fmt, BRUTE, 1.0, dg)
+        torch.cuda.synchronize()
+        _check_sampled(x, B, fmt, BRUTE, g, codes, scales, sse, 250, 900 + B + fmt)
+        m = _mse_matches_sum(sse, n)
+        assert int(scales.max().cpu()) < (127 if fmt == mxq.MXQ_SF_UE4M3 else 255)
+        if prev is not None:
+            assert prev <= m * (1 + 1e-6)
+        prev = m
+        del codes, scales, sse
