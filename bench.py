@@ -368,7 +368,7 @@ def run_gpu(args) -> None:
         hbm[name] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0, "traffic": None,
                      "ms_per_launch": ms, "gelem_s": N_ELEM / (ms * 1e-3) / 1e9, "peak_source": peaks["source"]}
-    streaming = streaming_rooflines(torch, mxq, device, peaks)
+    streaming = None if args.skip_streaming else streaming_rooflines(torch, mxq, device, peaks)
     per_recipe = {"brute_B16": N_ELEM / (brute_ms * 1e-3) / 1e9, "absmax_B16": hbm["absmax_B16"]["gelem_s"],
                   "4o6_B16": hbm["4o6_B16"]["gelem_s"]}
 
@@ -471,6 +471,8 @@ def main() -> None:
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--skip-streaming", action="store_true",
+                    help="leave out the 134M-element streaming measurements (roofline_hbm_streaming = null)")
     ap.add_argument("--impl", default="mxq", choices=["mxq", "reference"])
     args = ap.parse_args()
     if args.kernel:
