@@ -344,3 +344,60 @@ int mxq_oracle_dequantize(const uint8_t *codes, const uint8_t *scales, size_t n,
     }
     return 0;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Analysis outputs of the numerical study and the appendix (Results, numerical study; Appendix:
+ * "Clipping only MSE", entry and scale histograms).
+ * ------------------------------------------------------------------------------------------- */
+
+/* Clipping part of the block SSE: the error of the elements whose scaled magnitude exceeds the
+ * largest FP4 value, |fl32(v / D)| > 6 (they are all mapped to +-6).  Same arithmetic and element
+ * order as the block SSE, restricted to those elements; a zero scale clips nothing (its error is
+ * underflow, not clipping).  scales: one code per block, as written by the quantizer. */
+int mxq_oracle_block_clip_sse(const void *x, int dtype, size_t n, int B, int fmt, const uint8_t *scales, float g,
+                              float *out_clip_sse)
+{
+    if (!x || !scales || !out_clip_sse || n == 0 || B < 2 || B > 64 || n % (size_t)B) return -1;
+    for (size_t b = 0; b < n / (size_t)B; ++b) {
+        if (scales[b] >= mxq_oracle_num_codes(fmt)) return -1;
+        float D = mxq_oracle_scale_value(fmt, scales[b]) * g;
+        float sse = 0.0f;
+        for (int i = 0; i < B; ++i) {
+            float v = load_elem(x, dtype, b * (size_t)B + (size_t)i);
+            if (D == 0.0f) continue;
+            float t = v / D;
+            if (fabsf(t) > 6.0f) {
+                float q = signbit(v) ? -6.0f : 6.0f;
+                float e = fmaf(-q, D, v);
+                sse = fmaf(e, e, sse);
+            }
+        }
+        out_clip_sse[b] = sse;
+    }
+    return 0;
+}
+
+/* Histograms of the quantized entries (16 bins: the 4-bit code, sign included) and of the block
+ * scale codes (256 bins).  Counts are ADDED to the arrays. */
+int mxq_oracle_histograms(const uint8_t *codes, const uint8_t *scales, size_t n, int B, uint64_t *code_hist,
+                          uint64_t *scale_hist)
+{
+    if (!codes || !scales || !code_hist || !scale_hist || n == 0 || n % (size_t)B) return -1;
+    for (size_t i = 0; i < n; ++i) code_hist[(codes[i / 2] >> ((i & 1) ? 4 : 0)) & 15] += 1;
+    for (size_t b = 0; b < n / (size_t)B; ++b) scale_hist[scales[b]] += 1;
+    return 0;
+}
+
+/* MSE of consecutive segments of equal length (one sigma of the numerical study per segment):
+ * out[s] = (sum of the block SSEs of segment s) / elems_per_segment, in binary64, block order. */
+int mxq_oracle_segment_mse(const float *block_sse, size_t n_blocks, size_t blocks_per_segment, size_t elems_per_segment,
+                           double *out)
+{
+    if (!block_sse || !out || blocks_per_segment == 0 || n_blocks % blocks_per_segment || elems_per_segment == 0) return -1;
+    for (size_t s = 0; s < n_blocks / blocks_per_segment; ++s) {
+        double acc = 0.0;
+        for (size_t b = 0; b < blocks_per_segment; ++b) acc += (double)block_sse[s * blocks_per_segment + b];
+        out[s] = acc / (double)elems_per_segment;
+    }
+    return 0;
+}

@@ -64,6 +64,13 @@ def lib() -> ctypes.CDLL:
         L.mxq_oracle_dequantize.restype = c.c_int
         L.mxq_oracle_dequantize.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_int, c.c_int, c.c_float,
                                             c.c_void_p, c.c_int]
+        L.mxq_oracle_block_clip_sse.restype = c.c_int
+        L.mxq_oracle_block_clip_sse.argtypes = [c.c_void_p, c.c_int, c.c_size_t, c.c_int, c.c_int, c.c_void_p, c.c_float,
+                                                c.c_void_p]
+        L.mxq_oracle_histograms.restype = c.c_int
+        L.mxq_oracle_histograms.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_int, c.c_void_p, c.c_void_p]
+        L.mxq_oracle_segment_mse.restype = c.c_int
+        L.mxq_oracle_segment_mse.argtypes = [c.c_void_p, c.c_size_t, c.c_size_t, c.c_size_t, c.c_void_p]
         _lib = L
     return _lib
 
@@ -145,3 +152,36 @@ def global_scale_from_amax(amax) -> np.float32:
     """Hierarchical tensor scale g = amax / (6 * 448) in float32 (1 when the tensor is all zero)."""
     a = np.float32(amax)
     return np.float32(a / np.float32(2688.0)) if a > 0 else np.float32(1.0)
+
+
+def block_clip_sse(x, scales, block_size: int, fmt: int, g: float = 1.0):
+    """Per-block SSE of the elements clipped to +-6 (float32[n/B])."""
+    x, dt = _as_input(x)
+    scales = np.ascontiguousarray(scales, dtype=np.uint8)
+    out = np.empty(x.size // block_size, dtype=np.float32)
+    rc = lib().mxq_oracle_block_clip_sse(x.ctypes.data, dt, x.size, block_size, fmt, scales.ctypes.data,
+                                         float(np.float32(g)), out.ctypes.data)
+    if rc != 0:
+        raise ValueError("mxq_oracle_block_clip_sse: bad argument")
+    return out
+
+
+def histograms(codes, scales, n: int, block_size: int):
+    """(code histogram uint64[16], scale-code histogram uint64[256])."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scales = np.ascontiguousarray(scales, dtype=np.uint8)
+    ch = np.zeros(16, dtype=np.uint64)
+    sh = np.zeros(256, dtype=np.uint64)
+    rc = lib().mxq_oracle_histograms(codes.ctypes.data, scales.ctypes.data, n, block_size, ch.ctypes.data, sh.ctypes.data)
+    if rc != 0:
+        raise ValueError("mxq_oracle_histograms: bad argument")
+    return ch, sh
+
+
+def segment_mse(block_sse_arr, blocks_per_segment: int, elems_per_segment: int):
+    s = np.ascontiguousarray(block_sse_arr, dtype=np.float32)
+    out = np.empty(s.size // blocks_per_segment, dtype=np.float64)
+    rc = lib().mxq_oracle_segment_mse(s.ctypes.data, s.size, blocks_per_segment, elems_per_segment, out.ctypes.data)
+    if rc != 0:
+        raise ValueError("mxq_oracle_segment_mse: bad argument")
+    return out

@@ -169,3 +169,20 @@ def choose_exact(v, fmt: int, recipe: int, g=1.0):
         if best is None or s < best[1]:
             best = (c, s)
     return best
+
+
+def clip_sse_exact(v, fmt: int, code: int, g=1.0):
+    """SSE restricted to the elements whose quotient by the decode scale exceeds 6 in magnitude,
+    every float operation emulated exactly (same order as eval_block_exact)."""
+    S = TABLES[fmt]()[code]
+    D = f32_mul(np.float32(S), np.float32(g))
+    sse = np.float32(0.0)
+    if D == 0:
+        return sse
+    for x in np.asarray(v, dtype=np.float32):
+        t = f32_div(x, D)
+        if abs(frac(t)) > 6:
+            q = -6.0 if np.signbit(x) else 6.0
+            e = f32_fma(-q, D, x)
+            sse = f32_fma(e, e, sse)
+    return sse

@@ -1,0 +1,82 @@
+"""Pins for the oracle's analysis outputs: clipping-only SSE, entry / scale histograms and the
+segment MSE of the numerical study (CPU only)."""
+from fractions import Fraction
+
+import numpy as np
+
+import exact_ref as ex
+from oracle import mxq_oracle as orc
+
+
+def test_clipping_sse_hand_worked_block():
+    # UE4M3 code 0x38 is S = 1: elements above 6 are cut to 6, the others contribute nothing
+    v = np.array([7.0, -9.0, 6.0, 5.9, 0.3, -6.0, 6.5, -0.0], dtype=np.float32)
+    clip = orc.block_clip_sse(v, np.array([0x38], dtype=np.uint8), 8, orc.UE4M3)
+    assert clip[0] == np.float32(1.0 + 9.0 + 0.25)
+    # with a scale of 2 nothing exceeds 6 * 2
+    clip = orc.block_clip_sse(v, np.array([0x40], dtype=np.uint8), 8, orc.UE4M3)
+    assert clip[0] == 0.0
+    # a zero scale clips nothing: its error is underflow
+    clip = orc.block_clip_sse(v, np.array([0], dtype=np.uint8), 8, orc.UE4M3)
+    assert clip[0] == 0.0
+
+
+def test_clipping_sse_against_exact_rational_arithmetic():
+    rng = np.random.default_rng(5)
+    for fmt, g in ((orc.UE4M3, 1.0), (orc.UE4M3, 0.0131), (orc.UE5M3, 1.0), (orc.UE8M0, 0.7)):
+        for trial in range(40):
+            B = int(rng.choice([2, 4, 8, 16]))
+            v = (rng.standard_normal(B) * np.exp2(rng.integers(-6, 3))).astype(np.float32)
+            code = int(rng.integers(1, orc.num_codes(fmt)))
+            if fmt != orc.UE8M0:
+                # keep the scale near the data so that some elements clip and some do not
+                w = np.float32(np.abs(v).max() / g / rng.choice([6.0, 9.0, 14.0, 30.0]))
+                code = max(1, orc.round_scale(fmt, w))
+            else:
+                code = int(np.clip(127 + np.floor(np.log2(np.abs(v).max() / g / rng.choice([6.0, 12.0, 40.0]))), 1, 254))
+            got = orc.block_clip_sse(v, np.array([code], dtype=np.uint8), B, fmt, g)[0]
+            want = ex.clip_sse_exact(v, fmt, code, g)
+            assert np.float32(got).view(np.uint32) == np.float32(want).view(np.uint32), (fmt, g, code, v)
+
+
+def test_clipping_sse_is_part_of_the_block_sse_and_vanishes_without_clipping():
+    rng = np.random.default_rng(9)
+    x = (rng.standard_normal(4096) * 0.02).astype(np.float32)
+    for B in (4, 16):
+        for recipe in (orc.ABSMAX, orc.ABSMAX_PZ, orc.R4O6, orc.BRUTE):
+            codes, scales, sse = orc.quantize(x, B, orc.UE4M3, recipe)
+            clip = orc.block_clip_sse(x, scales, B, orc.UE4M3)
+            assert np.all(clip <= sse)          # a subsequence of the same non-negative terms
+            # blocks whose largest quotient stays within 6 have no clipping error
+            S = np.array([orc.scale_value(orc.UE4M3, int(c)) for c in scales], dtype=np.float32)
+            amax = np.abs(x.reshape(-1, B)).max(axis=1)
+            inside = (S > 0) & (np.float32(amax) / np.where(S > 0, S, 1) <= 6.0)
+            assert np.all(clip[inside] == 0.0)
+            assert np.any(clip > 0) or recipe in (orc.R4O6, orc.BRUTE)
+
+
+def test_histograms_count_every_entry_once():
+    rng = np.random.default_rng(2)
+    x = (rng.standard_normal(2048) * 0.3).astype(np.float32)
+    codes, scales, _ = orc.quantize(x, 16, orc.UE4M3, orc.ABSMAX)
+    ch, sh = orc.histograms(codes, scales, x.size, 16)
+    assert int(ch.sum()) == x.size and int(sh.sum()) == x.size // 16
+    nib = np.stack([codes & 15, codes >> 4], axis=1).reshape(-1)
+    assert np.array_equal(ch, np.bincount(nib, minlength=16).astype(np.uint64))
+    assert np.array_equal(sh, np.bincount(scales, minlength=256).astype(np.uint64))
+    # every block of an abs-max quantization holds an entry of magnitude 4 or 6 (the maximum maps to ~6)
+    mags = (nib & 7).reshape(-1, 16).max(axis=1)
+    assert np.all(mags >= 6)
+    # the sign bit of the code is the sign of the input
+    assert np.array_equal((nib >> 3).astype(bool), np.signbit(x))
+
+
+def test_segment_mse_is_the_tensor_mse_of_each_segment():
+    rng = np.random.default_rng(4)
+    sse = (rng.random(7 * 50) * np.exp2(rng.integers(-20, 2, 350))).astype(np.float32)
+    out = orc.segment_mse(sse, 50, 50 * 16)
+    for s in range(7):
+        seg = sse[s * 50:(s + 1) * 50]
+        assert out[s] == orc.tensor_mse(seg, 50 * 16)
+        exact = sum(Fraction(float(v)) for v in seg) / (50 * 16)
+        assert abs(Fraction(out[s]) - exact) <= exact * Fraction(1, 10 ** 14)
