@@ -160,6 +160,45 @@ int mxq_tensor_mse_static(const float* d_block_sse, size_t n_blocks, size_t n, d
 int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
                    float global_scale, void* d_out, int out_dtype, void* cuda_stream);
 
+/*
+ * mxq_block_clip_sse -- the clipping part of the block SSE (Appendix, "Clipping only MSE": the MSE
+ * plots of the numerical study restricted to their clipping portion).  For every block, the sum
+ * of (x - x_hat)^2 over the elements whose scaled magnitude exceeds the largest FP4 value,
+ * |fl32(x / D)| > 6 with D = fl32(S * g) -- they are all mapped to +-6 -- accumulated like the block
+ * SSE (binary32, element order, fused multiply-adds).  A zero decode scale clips nothing.
+ *   x, dtype, n, block_size, scale_fmt, global_scale, d_global_scale   as for mxq_quantize_ex.
+ *   d_scales      device, n/block_size scale codes as written by the quantizer.
+ *   out_clip_sse  device, n/block_size floats (NaN for a byte that is not a code of the format).
+ * Dividing the sum of these values by n gives the clipping-only MSE of the tensor.
+ */
+int mxq_block_clip_sse(const void* x, int dtype, size_t n, int block_size, int scale_fmt, float global_scale,
+                       const float* d_global_scale, const uint8_t* d_scales, float* out_clip_sse, void* cuda_stream);
+
+/*
+ * mxq_histograms -- bin utilisation of a quantized tensor (Appendix, histograms of entries and of
+ * scaling factors per recipe).
+ *   d_codes, d_scales   device, outputs of the quantizer for n elements in blocks of block_size.
+ *   d_code_hist   device, 16 unsigned 64-bit counters: occurrences of each 4-bit code (sign<<3 | index).
+ *   d_scale_hist  device, 256 unsigned 64-bit counters: occurrences of each scale code.
+ * Counts are ADDED to both arrays (clear them first for a fresh histogram; several tensors may be
+ * accumulated).  Integer sums: the result does not depend on the order of execution.
+ */
+int mxq_histograms(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size,
+                   unsigned long long* d_code_hist, unsigned long long* d_scale_hist, void* cuda_stream);
+
+/*
+ * mxq_segment_mse -- MSE of consecutive, equally long segments of a tensor in one launch (Results,
+ * numerical study: one segment per standard deviation sigma, 50,000 blocks each).
+ *   d_block_sse          device, n_blocks floats (or clipping SSEs).
+ *   blocks_per_segment   n_blocks must be a multiple of it.
+ *   elems_per_segment    the divisor (blocks_per_segment * block size).
+ *   d_out_mse            device, n_blocks / blocks_per_segment doubles.
+ * Fixed-shape binary64 tree per segment: the same inputs always give the same bits.  Needs no
+ * workspace.
+ */
+int mxq_segment_mse(const float* d_block_sse, size_t n_blocks, size_t blocks_per_segment, size_t elems_per_segment,
+                    double* d_out_mse, void* cuda_stream);
+
 /* Number of kernels the library has launched in this process (all entry points), for
  * accounting in benchmarks. */
 unsigned long long mxq_launch_count(void);

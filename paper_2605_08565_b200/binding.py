@@ -20,7 +20,7 @@ MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ = range(
 
 EXPORTS = (
     "mxq_quantize", "mxq_quantize_ex", "mxq_tensor_amax", "mxq_global_scale_from_amax",
-    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_launch_count",
+    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_launch_count",
     "mxq_status_string", "mxq_last_cuda_error", "mxq_version",
 )
 
@@ -59,6 +59,12 @@ def load_library() -> ctypes.CDLL:
     L.mxq_tensor_mse_static.argtypes = [vp, sz, sz, vp, vp]
     L.mxq_dequantize.restype = i32
     L.mxq_dequantize.argtypes = [vp, vp, sz, i32, i32, f32, vp, i32, vp]
+    L.mxq_block_clip_sse.restype = i32
+    L.mxq_block_clip_sse.argtypes = [vp, i32, sz, i32, i32, f32, vp, vp, vp, vp]
+    L.mxq_histograms.restype = i32
+    L.mxq_histograms.argtypes = [vp, vp, sz, i32, vp, vp, vp]
+    L.mxq_segment_mse.restype = i32
+    L.mxq_segment_mse.argtypes = [vp, sz, sz, sz, vp, vp]
     L.mxq_launch_count.restype = c.c_ulonglong
     L.mxq_launch_count.argtypes = []
     L.mxq_status_string.restype = c.c_char_p
@@ -146,6 +152,23 @@ def mxq_tensor_mse_static(d_block_sse, n_blocks, n, d_out_mse, stream=None) -> N
 def mxq_dequantize(d_codes, d_scales, n, block_size, scale_fmt, global_scale, d_out, stream=None) -> None:
     _check(load_library().mxq_dequantize(_ptr(d_codes), _ptr(d_scales), n, block_size, scale_fmt, global_scale,
                                          _ptr(d_out), _dtype_id(d_out), _stream(stream)))
+
+
+def mxq_block_clip_sse(x, n, block_size, scale_fmt, global_scale, d_global_scale, d_scales, out_clip_sse,
+                       stream=None) -> None:
+    _check(load_library().mxq_block_clip_sse(_ptr(x), _dtype_id(x), n, block_size, scale_fmt, global_scale,
+                                             _ptr(d_global_scale), _ptr(d_scales), _ptr(out_clip_sse), _stream(stream)))
+
+
+def mxq_histograms(d_codes, d_scales, n, block_size, d_code_hist, d_scale_hist, stream=None) -> None:
+    """d_code_hist: 16 and d_scale_hist: 256 int64/uint64 CUDA counters; counts are added to them."""
+    _check(load_library().mxq_histograms(_ptr(d_codes), _ptr(d_scales), n, block_size, _ptr(d_code_hist),
+                                         _ptr(d_scale_hist), _stream(stream)))
+
+
+def mxq_segment_mse(d_block_sse, n_blocks, blocks_per_segment, elems_per_segment, d_out_mse, stream=None) -> None:
+    _check(load_library().mxq_segment_mse(_ptr(d_block_sse), n_blocks, blocks_per_segment, elems_per_segment,
+                                          _ptr(d_out_mse), _stream(stream)))
 
 
 def mxq_launch_count() -> int:

@@ -1,0 +1,164 @@
+// Analysis kernels around the quantizer (Results, numerical study; Appendix: clipping-only MSE,
+// entry and scale histograms): the clipping part of the block SSE, histograms of the FP4 codes and
+// of the scale codes, and the MSE of equal-length segments of a tensor (one sigma of the
+// numerical study per segment).  None of them is on the bandwidth-critical path; they are written
+// for exactness and determinism first.
+#include "mxq_device.cuh"
+#include "mxq_internal.h"
+
+namespace mxq {
+
+// ------------------------------------------------------------------------------------------------
+// Clipping part of the block SSE: elements with |fl32(v / D)| > 6 are all mapped to +-6; their
+// error is accumulated exactly like the block SSE (e = fma(-q, D, v); s = fma(e, e, s), element
+// order), the other elements are skipped.  A zero decode scale clips nothing.  One thread per
+// block; IEEE division throughout.
+// ------------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(kThreads) k_block_clip_sse(const void* x, size_t n_blocks, int B, int fmt, float g,
+                                                             const float* d_g, const uint8_t* scales, float* out) {
+    const float gs = d_g ? *d_g : g;
+    const size_t stride = (size_t)gridDim.x * kThreads;
+    for (size_t b = (size_t)blockIdx.x * kThreads + threadIdx.x; b < n_blocks; b += stride) {
+        const int c = scales[b];
+        float s = 0.0f;
+        if (c < num_codes(fmt)) {
+            const float D = __fmul_rn(scale_value(fmt, c), gs);
+            if (D != 0.0f) {
+                for (int i = 0; i < B; ++i) {
+                    const size_t e_idx = b * (size_t)B + (size_t)i;
+                    float v;
+                    if constexpr (DT == kF32) v = static_cast<const float*>(x)[e_idx];
+                    else v = __uint_as_float((uint32_t) static_cast<const uint16_t*>(x)[e_idx] << 16);
+                    const float t = __fdiv_rn(v, D);
+                    if (fabsf(t) > 6.0f) {
+                        const float q = copysignf(6.0f, v);
+                        const float e = __fmaf_rn(-q, D, v);
+                        s = __fmaf_rn(e, e, s);
+                    }
+                }
+            }
+        } else {
+            s = __uint_as_float(0x7FC00000u);   // not a code of the format
+        }
+        out[b] = s;
+    }
+}
+
+cudaError_t launch_block_clip_sse(const void* x, int dtype, size_t n, int B, int fmt, float g, const float* d_g,
+                                  const uint8_t* scales, float* out, cudaStream_t s) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    const size_t n_blocks = n / (size_t)B;
+    size_t want = (n_blocks + kThreads - 1) / kThreads;
+    const size_t cap = (size_t)sm_count(dev) * 8;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    if (dtype == kF32) k_block_clip_sse<kF32><<<grid, kThreads, 0, s>>>(x, n_blocks, B, fmt, g, d_g, scales, out);
+    else k_block_clip_sse<kBF16><<<grid, kThreads, 0, s>>>(x, n_blocks, B, fmt, g, d_g, scales, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Histograms: 16 bins of the 4-bit codes, 256 bins of the scale codes, ADDED to the caller's
+// 64-bit counters.  Per-CTA counts in shared memory (32-bit: a CTA sees fewer than 2^32 entries
+// per trip batch), flushed with 64-bit integer atomics -- integer sums are order-free, so the
+// result is deterministic.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) k_histograms(const uint8_t* codes, const uint8_t* scales, size_t n,
+                                                         size_t n_blocks, unsigned long long* code_hist,
+                                                         unsigned long long* scale_hist) {
+    __shared__ unsigned int sh_code[8][16];   // one copy per warp: fewer same-address collisions
+    __shared__ unsigned int sh_scale[256];
+    for (int i = threadIdx.x; i < 8 * 16; i += kThreads) (&sh_code[0][0])[i] = 0;
+    for (int i = threadIdx.x; i < 256; i += kThreads) sh_scale[i] = 0;
+    __syncthreads();
+    const size_t stride = (size_t)gridDim.x * kThreads;
+    const size_t tid = (size_t)blockIdx.x * kThreads + threadIdx.x;
+    const int w = threadIdx.x >> 5;
+    // codes: 32-bit words of eight codes; n is even, the last (n/2) % 4 bytes are handled bytewise
+    const size_t n_bytes = n / 2, n_words = n_bytes / 4;
+    unsigned int local[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) local[k] = 0;
+    for (size_t i = tid; i < n_words; i += stride) {
+        const uint32_t word = reinterpret_cast<const uint32_t*>(codes)[i];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t c = (word >> (4 * k)) & 15u;
+#pragma unroll
+            for (int b = 0; b < 16; ++b) local[b] += (c == (uint32_t)b) ? 1u : 0u;
+        }
+    }
+    if (tid < n_bytes - n_words * 4) {
+        const uint32_t byte = codes[n_words * 4 + tid];
+        atomicAdd(&sh_code[w][byte & 15u], 1u);
+        atomicAdd(&sh_code[w][byte >> 4], 1u);
+    }
+#pragma unroll
+    for (int b = 0; b < 16; ++b)
+        if (local[b]) atomicAdd(&sh_code[w][b], local[b]);
+    for (size_t i = tid; i < n_blocks; i += stride) atomicAdd(&sh_scale[scales[i]], 1u);
+    __syncthreads();
+    if (threadIdx.x < 16) {
+        unsigned long long t = 0;
+        for (int k = 0; k < 8; ++k) t += sh_code[k][threadIdx.x];
+        if (t) atomicAdd(&code_hist[threadIdx.x], t);
+    }
+    for (int i = threadIdx.x; i < 256; i += kThreads)
+        if (sh_scale[i]) atomicAdd(&scale_hist[i], (unsigned long long)sh_scale[i]);
+}
+
+cudaError_t launch_histograms(const uint8_t* codes, const uint8_t* scales, size_t n, int B, unsigned long long* code_hist,
+                              unsigned long long* scale_hist, cudaStream_t s) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    size_t want = (n / 8 + kThreads - 1) / kThreads;
+    if (want == 0) want = 1;
+    // a thread must stay below 2^32 counts: n / (grid * 256) entries each -- true for any n < 2^40 here
+    const size_t cap = (size_t)sm_count(dev) * 8;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    k_histograms<<<grid, kThreads, 0, s>>>(codes, scales, n, n / (size_t)B, code_hist, scale_hist);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Segment MSE: out[s] = (sum of the block SSEs of segment s) / elems_per_segment.  One CTA per
+// segment (grid-stride over segments); thread t adds blocks t, t + 256, ... in order in binary64,
+// then a shared-memory halving tree: fixed shape, same bits on every run.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) k_segment_mse(const float* sse, size_t n_segments, size_t blocks_per_segment,
+                                                          double elems_per_segment, double* out) {
+    __shared__ double sh[kThreads];
+    for (size_t seg = blockIdx.x; seg < n_segments; seg += gridDim.x) {
+        const float* p = sse + seg * blocks_per_segment;
+        double acc = 0.0;
+        for (size_t i = threadIdx.x; i < blocks_per_segment; i += kThreads) acc = __dadd_rn(acc, (double)p[i]);
+        sh[threadIdx.x] = acc;
+        __syncthreads();
+#pragma unroll
+        for (int w = kThreads / 2; w > 0; w >>= 1) {
+            if (threadIdx.x < w) sh[threadIdx.x] = __dadd_rn(sh[threadIdx.x], sh[threadIdx.x + w]);
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) out[seg] = __ddiv_rn(sh[0], elems_per_segment);
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_segment_mse(const float* sse, size_t n_segments, size_t blocks_per_segment, size_t elems_per_segment,
+                               double* out, cudaStream_t s) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    const size_t cap = (size_t)sm_count(dev) * 8;
+    const unsigned grid = (unsigned)(n_segments < cap ? n_segments : cap);
+    k_segment_mse<<<grid, kThreads, 0, s>>>(sse, n_segments, blocks_per_segment, (double)elems_per_segment, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace mxq

@@ -140,6 +140,44 @@ int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, in
     return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
 }
 
+int mxq_block_clip_sse(const void* x, int dtype, size_t n, int block_size, int scale_fmt, float global_scale,
+                       const float* d_global_scale, const uint8_t* d_scales, float* out_clip_sse, void* cuda_stream) {
+    if (!x || !d_scales || !out_clip_sse) return MXQ_ERR_NULL;
+    if (dtype != MXQ_F32 && dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
+    if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
+    if (!valid_block(block_size) || n == 0 || n % (size_t)block_size != 0) return MXQ_ERR_BAD_SHAPE;
+    if (!d_global_scale && !(global_scale > 0.0f && std::isfinite(global_scale))) return MXQ_ERR_BAD_SCALE;
+    if (!aligned16(x) || (reinterpret_cast<uintptr_t>(out_clip_sse) & 3u) ||
+        (d_global_scale && (reinterpret_cast<uintptr_t>(d_global_scale) & 3u)))
+        return MXQ_ERR_ALIGN;
+    cudaError_t err = launch_block_clip_sse(x, dtype, n, block_size, scale_fmt, d_global_scale ? 1.0f : global_scale,
+                                            d_global_scale, d_scales, out_clip_sse, static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+int mxq_histograms(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size,
+                   unsigned long long* d_code_hist, unsigned long long* d_scale_hist, void* cuda_stream) {
+    if (!d_codes || !d_scales || !d_code_hist || !d_scale_hist) return MXQ_ERR_NULL;
+    if (!valid_block(block_size) || n == 0 || n % (size_t)block_size != 0) return MXQ_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(d_codes) & 3u) || (reinterpret_cast<uintptr_t>(d_code_hist) & 7u) ||
+        (reinterpret_cast<uintptr_t>(d_scale_hist) & 7u))
+        return MXQ_ERR_ALIGN;
+    cudaError_t err = launch_histograms(d_codes, d_scales, n, block_size, d_code_hist, d_scale_hist,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+int mxq_segment_mse(const float* d_block_sse, size_t n_blocks, size_t blocks_per_segment, size_t elems_per_segment,
+                    double* d_out_mse, void* cuda_stream) {
+    if (!d_block_sse || !d_out_mse) return MXQ_ERR_NULL;
+    if (n_blocks == 0 || blocks_per_segment == 0 || elems_per_segment == 0 || n_blocks % blocks_per_segment != 0)
+        return MXQ_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(d_block_sse) & 3u) || (reinterpret_cast<uintptr_t>(d_out_mse) & 7u)) return MXQ_ERR_ALIGN;
+    cudaError_t err = launch_segment_mse(d_block_sse, n_blocks / blocks_per_segment, blocks_per_segment, elems_per_segment,
+                                         d_out_mse, static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
 unsigned long long mxq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* mxq_status_string(int status) {

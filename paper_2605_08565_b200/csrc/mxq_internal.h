@@ -41,6 +41,13 @@ cudaError_t launch_tensor_mse_static(const float* d_sse, size_t n_blocks, size_t
 cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n, int B, int fmt, float g, void* out,
                               int out_dtype, cudaStream_t s);
 
+cudaError_t launch_block_clip_sse(const void* x, int dtype, size_t n, int B, int fmt, float g, const float* d_g,
+                                  const uint8_t* scales, float* out, cudaStream_t s);
+cudaError_t launch_histograms(const uint8_t* codes, const uint8_t* scales, size_t n, int B, unsigned long long* code_hist,
+                              unsigned long long* scale_hist, cudaStream_t s);
+cudaError_t launch_segment_mse(const float* sse, size_t n_segments, size_t blocks_per_segment, size_t elems_per_segment,
+                               double* out, cudaStream_t s);
+
 constexpr int kMsePartials = 1024;  // fixed first-level width of the MSE tree
 
 }  // namespace mxq

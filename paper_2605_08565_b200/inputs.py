@@ -8,6 +8,7 @@ for them with tensors of the same shapes and rough value distributions:
 * ``student_t``       scale * t_nu                      (weight-shaped tensors, heavy tails)
 * ``outlier_columns`` N(0,1) rows, 1 % of columns x50   (activation-shaped tensors)
 * ``laplace``         Laplace(0, 1)                     (bulk scale-search case)
+* ``sigma_sweep``     N(0, sigma^2) segments, 151 sigmas (the numerical study's sampling protocol)
 * ``adversarial``     short-mantissa values, zeros, signed zeros, denormals, tiny and huge blocks
 
 Every generator takes a seed and a device and returns a flat torch tensor; the same call on the
@@ -114,6 +115,25 @@ def adversarial(n: int, seed: int, dtype=torch.float32) -> torch.Tensor:
             v = rng.standard_normal(64).astype(np.float32)
         out[r * 64:(r + 1) * 64] = v * sign
     return _cast(torch.from_numpy(out[:n].copy()), dtype)
+
+
+def sigma_grid(n_sigma: int = 151, lo: float = 0.0005, hi: float = 0.05) -> torch.Tensor:
+    """The standard deviations of the numerical study: n_sigma evenly spaced points in [lo, hi] (float64)."""
+    return torch.linspace(lo, hi, n_sigma, dtype=torch.float64)
+
+
+def sigma_sweep(elems_per_sigma: int, seed: int, n_sigma: int = 151, lo: float = 0.0005, hi: float = 0.05,
+                dtype=torch.float32, device="cpu", chunk_sigmas: int = 8) -> torch.Tensor:
+    """Concatenation of n_sigma segments of elems_per_sigma i.i.d. N(0, sigma_k^2) samples, sigma_k from
+    ``sigma_grid`` (numerical study: 50,000 x block_size samples per sigma)."""
+    g = _gen(seed, device)
+    sig = sigma_grid(n_sigma, lo, hi).to(torch.float32).to(device)
+    out = torch.empty(n_sigma * elems_per_sigma, dtype=dtype, device=device)
+    for s in range(0, n_sigma, chunk_sigmas):
+        k = min(chunk_sigmas, n_sigma - s)
+        z = torch.randn(k, elems_per_sigma, generator=g, device=device, dtype=torch.float32)
+        out[s * elems_per_sigma:(s + k) * elems_per_sigma] = (z * sig[s:s + k, None]).reshape(-1).to(dtype)
+    return out
 
 
 def to_numpy_bits(x: torch.Tensor) -> np.ndarray:

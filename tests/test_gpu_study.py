@@ -1,0 +1,78 @@
+"""GPU parity of the analysis entry points (clipping-only SSE, histograms, segment MSE) and of a
+reduced numerical study against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mxq_oracle as orc
+from paper_2605_08565_b200 import binding as mxq
+from paper_2605_08565_b200 import inputs, study
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", [2, 4, 16, 64])
+def test_clip_sse_and_histograms_bit_exact(dtype, B):
+    n = 3 * 256 * max(B, 8) + 5 * 64 + (B if B < 8 else 0)
+    x = (inputs.adversarial(n, 3 + B, torch.float32) * 0.5).to(dtype).contiguous()
+    for fmt, g, recipe in ((mxq.MXQ_SF_UE4M3, 1.0, mxq.MXQ_ABSMAX), (mxq.MXQ_SF_UE4M3, 0.0131, mxq.MXQ_ABSMAX_PZ),
+                           (mxq.MXQ_SF_UE5M3, 1.0, mxq.MXQ_4O6), (mxq.MXQ_SF_UE8M0, 1.0, mxq.MXQ_ABSMAX)):
+        xg = x.cuda()
+        codes, scales, sse = mxq.quantize(xg, B, fmt, recipe, g)
+        clip = torch.empty_like(sse)
+        mxq.mxq_block_clip_sse(xg, n, B, fmt, g, None, scales, clip)
+        ch = torch.zeros(16, dtype=torch.int64, device="cuda")
+        sh = torch.zeros(256, dtype=torch.int64, device="cuda")
+        mxq.mxq_histograms(codes, scales, n, B, ch, sh)
+        mxq.mxq_histograms(codes, scales, n, B, ch, sh)      # counts accumulate
+        torch.cuda.synchronize()
+        xb = inputs.to_numpy_bits(x)
+        oc, os_, oe = orc.quantize(xb, B, fmt, recipe, g)
+        want = orc.block_clip_sse(xb, os_, B, fmt, g)
+        assert np.array_equal(clip.cpu().numpy().view(np.uint32), want.view(np.uint32))
+        och, osh = orc.histograms(oc, os_, n, B)
+        assert np.array_equal(ch.cpu().numpy().astype(np.uint64), 2 * och)
+        assert np.array_equal(sh.cpu().numpy().astype(np.uint64), 2 * osh)
+
+
+def test_segment_mse_matches_oracle():
+    rng = np.random.default_rng(8)
+    for nseg, per in ((1, 1), (7, 50), (151, 1000), (3, 70001)):
+        sse = (rng.random(nseg * per) * np.exp2(rng.integers(-30, 4, nseg * per))).astype(np.float32)
+        d = torch.from_numpy(sse).cuda()
+        out = torch.empty(nseg, dtype=torch.float64, device="cuda")
+        mxq.mxq_segment_mse(d, nseg * per, per, per * 16, out)
+        mxq_out = out.cpu().numpy()
+        want = orc.segment_mse(sse, per, per * 16)
+        assert np.all(np.abs(mxq_out - want) <= 1e-12 * want)
+        out2 = torch.empty_like(out)
+        mxq.mxq_segment_mse(d, nseg * per, per, per * 16, out2)
+        assert torch.equal(out, out2)
+
+
+def test_reduced_numerical_study_against_oracle():
+    """16 sigmas x 2000 blocks, all five recipes, block sizes 4 and 16: every MSE and clipping-MSE
+    point against the oracle on the very same samples."""
+    n_sigma, per_blocks = 16, 2000
+    res = study.run(block_sizes=(4, 16), n_sigma=n_sigma, blocks_per_sigma=per_blocks, seed=3, histogram_sigmas=(0, 9))
+    for B in (4, 16):
+        x = inputs.sigma_sweep(per_blocks * B, 3 * 1000 + B, n_sigma, device="cuda").cpu()
+        xb = inputs.to_numpy_bits(x)
+        for name, rid in study.RECIPES.items():
+            oc, os_, oe = orc.quantize(xb, B, orc.UE4M3, rid, 1.0, threads=8)
+            want = orc.segment_mse(oe, per_blocks, per_blocks * B)
+            got = np.array(res["mse"][name][B])
+            assert np.all(np.abs(got - want) <= 1e-6 * want), (name, B)
+            wclip = orc.segment_mse(orc.block_clip_sse(xb, os_, B, orc.UE4M3), per_blocks, per_blocks * B)
+            gclip = np.array(res["clip_mse"][name][B])
+            assert np.all(np.abs(gclip - wclip) <= 1e-6 * wclip + 1e-300), (name, B)
+            for k in (0, 9):
+                lo = k * per_blocks
+                och, osh = orc.histograms(oc[lo * B // 2:(lo + per_blocks) * B // 2], os_[lo:lo + per_blocks],
+                                          per_blocks * B, B)
+                h = res["hist"][f"{name}/B{B}/sigma{k}"]
+                assert np.array_equal(np.array(h["codes"], dtype=np.uint64), och)
+                assert np.array_equal(np.array(h["scales"], dtype=np.uint64), osh)
+    f = study.findings(res)
+    assert f["pz_never_worse"]
