@@ -197,25 +197,17 @@ __device__ __forceinline__ void pack_and_score(const float* v, const float* t, c
 }
 
 // One candidate set of a group with the shortcuts (every entry has w != 0, magnitudes in range).
-template <int B>
-__device__ __forceinline__ void encode_group_fast(const float* v, const float4* E, bool all_short, bool all_half,
-                                                  uint32_t* packed, float* sse) {
+template <int B, bool SHORTQ, bool HALF>
+__device__ __forceinline__ void encode_group_fast(const float* v, const float4* E, uint32_t* packed, float* sse) {
     constexpr int GE = (B < 8) ? 8 : B;
     constexpr int NBG = GE / B;
     float t[GE];
-    if (all_short) {
 #pragma unroll
-        for (int j = 0; j < NBG; ++j)
+    for (int j = 0; j < NBG; ++j)
 #pragma unroll
-            for (int i = 0; i < B; ++i) t[j * B + i] = quotient_short(v[j * B + i], E[j].x, E[j].y);
-    } else {
-#pragma unroll
-        for (int j = 0; j < NBG; ++j)
-#pragma unroll
-            for (int i = 0; i < B; ++i) t[j * B + i] = quotient_corrected(v[j * B + i], E[j].x, E[j].y);
-    }
-    if (all_half) pack_and_score<B, true>(v, t, E, packed, sse);
-    else pack_and_score<B, false>(v, t, E, packed, sse);
+        for (int i = 0; i < B; ++i)
+            t[j * B + i] = SHORTQ ? quotient_short(v[j * B + i], E[j].x, E[j].y) : quotient_corrected(v[j * B + i], E[j].x, E[j].y);
+    pack_and_score<B, HALF>(v, t, E, packed, sse);
 }
 
 // One candidate set of a group on the general path (IEEE division; zero scale -> signed zeros).
@@ -238,7 +230,7 @@ struct QuantConsts {
     bool unit_g, need_lo, pz, all_short;
 };
 
-template <int DT, int B, int FMT, bool DUAL>
+template <int DT, int B, int FMT, bool DUAL, bool SHORTQ>
 __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
                                                size_t chunk, const uint32_t* raw) {
     using S = QuantShape<DT, B>;
@@ -280,8 +272,13 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
         uint32_t pk[S::GE / 8], pk4[S::GE / 8];
         float sse[NBG], sse4[NBG];
         if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
-            encode_group_fast<B>(v, E6, k.all_short, wmin >= 2.0f, pk, sse);
-            if constexpr (DUAL) encode_group_fast<B>(v, E4, k.all_short, wmin >= 2.0f, pk4, sse4);
+            if (wmin >= 2.0f) {   // one decision for both candidates
+                encode_group_fast<B, SHORTQ, true>(v, E6, pk, sse);
+                if constexpr (DUAL) encode_group_fast<B, SHORTQ, true>(v, E4, pk4, sse4);
+            } else {
+                encode_group_fast<B, SHORTQ, false>(v, E6, pk, sse);
+                if constexpr (DUAL) encode_group_fast<B, SHORTQ, false>(v, E4, pk4, sse4);
+            }
         } else {
 #pragma unroll
             for (int j = 0; j < NBG; ++j) {
@@ -415,7 +412,8 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
         ahead += stride;
         slot = (slot + 1 == S::SLOTS) ? 0 : slot + 1;
         fill = (fill + 1 == S::SLOTS) ? 0 : fill + 1;
-        quantize_chunk<DT, B, FMT, DUAL>(p, T, k, chunk, raw);
+        if (k.all_short) quantize_chunk<DT, B, FMT, DUAL, true>(p, T, k, chunk, raw);
+        else quantize_chunk<DT, B, FMT, DUAL, false>(p, T, k, chunk, raw);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
