@@ -33,7 +33,7 @@
 
 enum { ORC_F32 = 0, ORC_BF16 = 1 };
 enum { ORC_UE8M0 = 0, ORC_UE4M3 = 1, ORC_UE5M3 = 2 };
-enum { ORC_ABSMAX = 0, ORC_ABSMAX_PZ = 1, ORC_4O6 = 2, ORC_4O6_PZ = 3, ORC_BRUTE = 4, ORC_BRUTE_PZ = 5 };
+enum { ORC_ABSMAX = 0, ORC_ABSMAX_PZ = 1, ORC_4O6 = 2, ORC_4O6_PZ = 3, ORC_BRUTE = 4, ORC_BRUTE_PZ = 5, ORC_ABSMAX_OCP = 6 };
 
 /* ---------------------------------------------------------------------------------------------
  * Number formats (Background; Experimental Setup).
@@ -198,6 +198,23 @@ static int absmax_code(float amax, float g, float M, int fmt, int prevent_zero)
     return c;
 }
 
+/* The power-of-two rule as the OCP MX specification words it (Background: the paper paraphrases
+ * it in prose and prints Eq. 1, which differs): the shared exponent is the exponent of the block
+ * maximum minus the exponent of the largest element value, S = 2^(floor(log2 amax) - 2) for E2M1
+ * (6 = 1.5 * 2^2).  The maximum then lands in [4, 8) and is clipped when it exceeds 6.  UE8M0
+ * only; amax is first adjusted by the tensor scale like in the other recipes. */
+int mxq_oracle_ocp_code(float amax, float g)
+{
+    float u = amax / g;
+    if (!(u > 0.0f)) return 0;
+    int e;
+    (void)frexpf(u, &e);          /* u = f * 2^e, 0.5 <= f < 1: floor(log2 u) = e - 1 */
+    int c = 127 + (e - 1) - 2;
+    if (c < 0) c = 0;
+    if (c > 254) c = 254;
+    return c;
+}
+
 /* Choose the scale code of one block by recipe; returns the code, writes the block's SSE. */
 static int choose_code(const float *v, int B, int fmt, int recipe, float g, float *sse_out)
 {
@@ -211,6 +228,9 @@ static int choose_code(const float *v, int B, int fmt, int recipe, float g, floa
 
     if (recipe == ORC_ABSMAX || recipe == ORC_ABSMAX_PZ) {
         best = absmax_code(amax, g, 6.0f, fmt, pz);
+        best_sse = eval_block(v, B, fmt, best, g, NULL);
+    } else if (recipe == ORC_ABSMAX_OCP) {
+        best = mxq_oracle_ocp_code(amax, g);
         best_sse = eval_block(v, B, fmt, best, g, NULL);
     } else if (recipe == ORC_4O6 || recipe == ORC_4O6_PZ) {
         /* Eq. 4: argmin over M in {4, 6} of the block error; a tie keeps M = 6. */
@@ -267,7 +287,8 @@ int mxq_oracle_quantize(const void *x, int dtype, size_t n, int B, int fmt, int 
                         uint8_t *scales, float *block_sse)
 {
     if (!x || n == 0 || B < 2 || B > 64 || (B & (B - 1)) || n % (size_t)B) return -1;
-    if (mxq_oracle_num_codes(fmt) == 0 || recipe < 0 || recipe > ORC_BRUTE_PZ) return -1;
+    if (mxq_oracle_num_codes(fmt) == 0 || recipe < 0 || recipe > ORC_ABSMAX_OCP) return -1;
+    if (recipe == ORC_ABSMAX_OCP && fmt != ORC_UE8M0) return -1;
     if (!(g > 0.0f) || !isfinite(g)) return -1;
     quantize_range(x, dtype, 0, n / (size_t)B, B, fmt, recipe, g, codes, scales, block_sse);
     return 0;
@@ -292,7 +313,8 @@ int mxq_oracle_quantize_mt(const void *x, int dtype, size_t n, int B, int fmt, i
 {
     if (threads <= 1) return mxq_oracle_quantize(x, dtype, n, B, fmt, recipe, g, codes, scales, block_sse);
     if (!x || n == 0 || B < 2 || B > 64 || (B & (B - 1)) || n % (size_t)B) return -1;
-    if (mxq_oracle_num_codes(fmt) == 0 || recipe < 0 || recipe > ORC_BRUTE_PZ) return -1;
+    if (mxq_oracle_num_codes(fmt) == 0 || recipe < 0 || recipe > ORC_ABSMAX_OCP) return -1;
+    if (recipe == ORC_ABSMAX_OCP && fmt != ORC_UE8M0) return -1;
     if (!(g > 0.0f) || !isfinite(g)) return -1;
     if (threads > 256) threads = 256;
     pthread_t tid[256];

@@ -18,7 +18,7 @@ _LIB = os.path.join(_HERE, "libmxq_oracle.so")
 
 F32, BF16 = 0, 1
 UE8M0, UE4M3, UE5M3 = 0, 1, 2
-ABSMAX, ABSMAX_PZ, R4O6, R4O6_PZ, BRUTE, BRUTE_PZ = range(6)
+ABSMAX, ABSMAX_PZ, R4O6, R4O6_PZ, BRUTE, BRUTE_PZ, ABSMAX_OCP = range(7)
 
 _CFLAGS = ["-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared", "-pthread"]
 
@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.mxq_oracle_dequantize.restype = c.c_int
         L.mxq_oracle_dequantize.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t, c.c_int, c.c_int, c.c_float,
                                             c.c_void_p, c.c_int]
+        L.mxq_oracle_ocp_code.restype = c.c_int
+        L.mxq_oracle_ocp_code.argtypes = [c.c_float, c.c_float]
         L.mxq_oracle_block_clip_sse.restype = c.c_int
         L.mxq_oracle_block_clip_sse.argtypes = [c.c_void_p, c.c_int, c.c_size_t, c.c_int, c.c_int, c.c_void_p, c.c_float,
                                                 c.c_void_p]
@@ -185,3 +187,13 @@ def segment_mse(block_sse_arr, blocks_per_segment: int, elems_per_segment: int):
     if rc != 0:
         raise ValueError("mxq_oracle_segment_mse: bad argument")
     return out
+
+
+def ocp_code(amax, g: float = 1.0) -> int:
+    return lib().mxq_oracle_ocp_code(float(np.float32(amax)), float(np.float32(g)))
+
+
+def fake_quantize(x, block_size: int, fmt: int, recipe: int, g: float = 1.0, out_dtype: int = F32, threads: int = 1):
+    """dequantize(quantize(x)): what a model sees when its weights or activations are quantized."""
+    codes, scales, _ = quantize(x, block_size, fmt, recipe, g, threads)
+    return dequantize(codes, scales, np.ascontiguousarray(x).size, block_size, fmt, g, out_dtype)

@@ -80,3 +80,39 @@ def test_segment_mse_is_the_tensor_mse_of_each_segment():
         assert out[s] == orc.tensor_mse(seg, 50 * 16)
         exact = sum(Fraction(float(v)) for v in seg) / (50 * 16)
         assert abs(Fraction(out[s]) - exact) <= exact * Fraction(1, 10 ** 14)
+
+
+def test_ocp_power_of_two_rule_hand_worked_and_against_eq1():
+    # S = 2^(floor(log2 amax) - 2): amax 1 -> 2^-2, 3.9 -> 2^-1, 4 -> 1, 6 -> 1, 7.99 -> 1, 8 -> 2
+    for amax, code in ((1.0, 125), (3.9, 126), (4.0, 127), (6.0, 127), (7.99, 127), (8.0, 128), (0.75, 124)):
+        assert orc.ocp_code(amax) == code, amax
+    assert orc.ocp_code(0.0) == 0
+    assert orc.ocp_code(1.0, 0.25) == orc.ocp_code(4.0)          # the tensor scale divides the maximum first
+    rng = np.random.default_rng(12)
+    for a in np.exp2(rng.uniform(-20, 20, 2000)).astype(np.float32):
+        c_ocp, c_eq1 = orc.ocp_code(a), orc.round_scale(orc.UE8M0, np.float32(a) / np.float32(6.0))
+        assert c_ocp - c_eq1 in (0, 1)                           # same scale, or twice the one of Eq. 1
+        q = Fraction(float(a)) / Fraction(2) ** (c_ocp - 127)
+        assert 4 <= q < 8                                        # the maximum lands in [4, 8)
+    x = (rng.standard_normal(1024) * 0.3).astype(np.float32)
+    codes, scales, sse = orc.quantize(x, 32, orc.UE8M0, orc.ABSMAX_OCP)
+    amax = np.abs(x.reshape(-1, 32)).max(axis=1)
+    assert np.array_equal(scales, np.array([orc.ocp_code(a) for a in amax], dtype=np.uint8))
+    for b in range(4):
+        s_b, _ = orc.block_sse(x[b * 32:(b + 1) * 32], orc.UE8M0, int(scales[b]))
+        assert s_b == sse[b]
+
+
+def test_fake_quantize_is_dequantize_of_quantize():
+    rng = np.random.default_rng(13)
+    x = (rng.standard_normal(512) * 0.1).astype(np.float32)
+    for fmt, recipe, g in ((orc.UE4M3, orc.R4O6, 1.0), (orc.UE5M3, orc.ABSMAX_PZ, 0.37), (orc.UE8M0, orc.ABSMAX_OCP, 1.0)):
+        xh = orc.fake_quantize(x, 16, fmt, recipe, g)
+        codes, scales, sse = orc.quantize(x, 16, fmt, recipe, g)
+        # the block SSE is the squared distance between x and its fake-quantized copy (up to one rounding per term)
+        err = ((x.astype(np.float64) - xh.astype(np.float64)) ** 2).reshape(-1, 16).sum(axis=1)
+        assert np.allclose(err, sse, rtol=1e-5, atol=1e-30)
+        # every value is a grid value times the decode scale of its block
+        S = np.array([orc.scale_value(fmt, int(c)) for c in scales], dtype=np.float32) * np.float32(g)
+        ratio = np.abs(xh.reshape(-1, 16)) / S[:, None]
+        assert np.all(np.isin(np.round(ratio * 2) / 2, [0, .5, 1, 1.5, 2, 3, 4, 6]))
