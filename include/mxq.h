@@ -69,9 +69,14 @@ typedef enum { MXQ_SF_UE8M0 = 0, MXQ_SF_UE4M3 = 1, MXQ_SF_UE5M3 = 2 } mxq_scale_
  *   BRUTE      every finite scale code is tried (BRUTE_PZ: every code with a nonzero value);
  *              smallest SSE wins, equal SSE keeps the smaller code.  A code whose decode scale
  *              S*g is not a finite float is skipped.
+ *   ABSMAX_OCP MXQ_SF_UE8M0 only: the power-of-two rule as the OCP MX specification words it (the
+ *              Background paraphrases it; Eq. 1 as printed differs): scale exponent = exponent of the
+ *              block maximum minus the exponent of the largest FP4 value, S = 2^(floor(log2(amax/g)) - 2).
+ *              The maximum lands in [4, 8) and is clipped above 6; S is the scale of Eq. 1 or twice it.
  * Hierarchical scaling is any recipe called with global_scale != 1. */
 typedef enum {
-    MXQ_ABSMAX = 0, MXQ_ABSMAX_PZ = 1, MXQ_4O6 = 2, MXQ_4O6_PZ = 3, MXQ_BRUTE = 4, MXQ_BRUTE_PZ = 5
+    MXQ_ABSMAX = 0, MXQ_ABSMAX_PZ = 1, MXQ_4O6 = 2, MXQ_4O6_PZ = 3, MXQ_BRUTE = 4, MXQ_BRUTE_PZ = 5,
+    MXQ_ABSMAX_OCP = 6
 } mxq_recipe;
 
 /*
@@ -100,6 +105,21 @@ int mxq_quantize(const float* x, size_t n, int block_size, int scale_fmt, int re
 int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe,
                     float global_scale, const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales,
                     float* out_block_sse, void* cuda_stream);
+
+/*
+ * mxq_fake_quantize -- quantize and de-quantize in one pass: out_i = fl32(grid(code_i) * D_b), the
+ * values a model computes with when its MLP weights or activations are held in this format
+ * (Results, downstream experiments: "applying these scaling methods to the weight and activation
+ * quantization").  Bit-identical to mxq_quantize_ex followed by mxq_dequantize, without writing
+ * codes, scales or SSE.
+ *   x, dtype, n, block_size, scale_fmt, global_scale, d_global_scale, cuda_stream   as for mxq_quantize_ex.
+ *   recipe     any recipe except the brute-force ones (MXQ_ERR_BAD_ENUM for those: run mxq_quantize_ex
+ *              and mxq_dequantize instead).
+ *   d_out      device, n elements of out_dtype (MXQ_F32, or MXQ_BF16 = the binary32 value rounded to
+ *              bf16, round-to-nearest-even); may not alias x.
+ */
+int mxq_fake_quantize(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe,
+                      float global_scale, const float* d_global_scale, void* d_out, int out_dtype, void* cuda_stream);
 
 /*
  * mxq_tensor_amax -- first stage of hierarchical scaling (Experimental Setup, "a per-tensor scale

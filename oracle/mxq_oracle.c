@@ -207,6 +207,7 @@ int mxq_oracle_ocp_code(float amax, float g)
 {
     float u = amax / g;
     if (!(u > 0.0f)) return 0;
+    if (isinf(u)) return 254;     /* amax / g overflowed: the largest scale, as the floor rule of Eq. 1 gives */
     int e;
     (void)frexpf(u, &e);          /* u = f * 2^e, 0.5 <= f < 1: floor(log2 u) = e - 1 */
     int c = 127 + (e - 1) - 2;

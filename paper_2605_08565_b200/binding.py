@@ -16,10 +16,10 @@ LIB_PATH = os.path.join(_HERE, "libmxq.so")
 
 MXQ_F32, MXQ_BF16 = 0, 1
 MXQ_SF_UE8M0, MXQ_SF_UE4M3, MXQ_SF_UE5M3 = 0, 1, 2
-MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ = range(6)
+MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ, MXQ_ABSMAX_OCP = range(7)
 
 EXPORTS = (
-    "mxq_quantize", "mxq_quantize_ex", "mxq_tensor_amax", "mxq_global_scale_from_amax",
+    "mxq_quantize", "mxq_quantize_ex", "mxq_fake_quantize", "mxq_tensor_amax", "mxq_global_scale_from_amax",
     "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_launch_count",
     "mxq_status_string", "mxq_last_cuda_error", "mxq_version",
 )
@@ -47,6 +47,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_quantize.argtypes = [vp, sz, i32, i32, i32, f32, vp, vp, vp]
     L.mxq_quantize_ex.restype = i32
     L.mxq_quantize_ex.argtypes = [vp, i32, sz, i32, i32, i32, f32, vp, vp, vp, vp, vp]
+    L.mxq_fake_quantize.restype = i32
+    L.mxq_fake_quantize.argtypes = [vp, i32, sz, i32, i32, i32, f32, vp, vp, i32, vp]
     L.mxq_tensor_amax.restype = i32
     L.mxq_tensor_amax.argtypes = [vp, i32, sz, vp, vp, vp]
     L.mxq_global_scale_from_amax.restype = f32
@@ -123,6 +125,11 @@ def mxq_quantize_ex(x, n, block_size, scale_fmt, recipe, global_scale, d_global_
     _check(load_library().mxq_quantize_ex(_ptr(x), _dtype_id(x), n, block_size, scale_fmt, recipe, global_scale,
                                           _ptr(d_global_scale), _ptr(out_codes), _ptr(out_scales),
                                           _ptr(out_block_sse), _stream(stream)))
+
+
+def mxq_fake_quantize(x, n, block_size, scale_fmt, recipe, global_scale, d_global_scale, d_out, stream=None) -> None:
+    _check(load_library().mxq_fake_quantize(_ptr(x), _dtype_id(x), n, block_size, scale_fmt, recipe, global_scale,
+                                            _ptr(d_global_scale), _ptr(d_out), _dtype_id(d_out), _stream(stream)))
 
 
 def mxq_tensor_amax(x, n, d_out_amax, d_out_global_scale=None, stream=None) -> None:

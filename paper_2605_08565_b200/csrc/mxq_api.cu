@@ -38,16 +38,23 @@ using namespace mxq;
 
 extern "C" {
 
-int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,
-                    const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales, float* out_block_sse,
-                    void* cuda_stream) {
-    if (!x || !out_codes || !out_scales) return MXQ_ERR_NULL;
+}  // extern "C"
+
+// Shared by mxq_quantize_ex (codes + scales, optional SSE) and mxq_fake_quantize (x_hat only).
+static int quantize_common(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe,
+                           float global_scale, const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales,
+                           float* out_block_sse, void* out_xhat, int xhat_dtype, void* cuda_stream) {
+    if (!x || (!out_xhat && (!out_codes || !out_scales))) return MXQ_ERR_NULL;
     if (dtype != MXQ_F32 && dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
     if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
-    if (recipe < MXQ_ABSMAX || recipe > MXQ_BRUTE_PZ) return MXQ_ERR_BAD_ENUM;
+    if (recipe < MXQ_ABSMAX || recipe > MXQ_ABSMAX_OCP) return MXQ_ERR_BAD_ENUM;
+    if (recipe == MXQ_ABSMAX_OCP && scale_fmt != MXQ_SF_UE8M0) return MXQ_ERR_BAD_ENUM;
+    const bool brute = (recipe == MXQ_BRUTE || recipe == MXQ_BRUTE_PZ);
+    if (out_xhat && (brute || (xhat_dtype != MXQ_F32 && xhat_dtype != MXQ_BF16))) return MXQ_ERR_BAD_ENUM;
     if (!valid_block(block_size) || n == 0 || n % (size_t)block_size != 0) return MXQ_ERR_BAD_SHAPE;
     if (!d_global_scale && !(global_scale > 0.0f && std::isfinite(global_scale))) return MXQ_ERR_BAD_SCALE;
     if (!aligned16(x) || !aligned16(out_codes) || !aligned16(out_scales) || !aligned16(out_block_sse) ||
+        !aligned16(out_xhat) ||
         (d_global_scale && (reinterpret_cast<uintptr_t>(d_global_scale) & 3u)))
         return MXQ_ERR_ALIGN;
 
@@ -61,9 +68,12 @@ int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scal
     a.scales = out_scales;
     a.block_sse = out_block_sse;
     a.prevent_zero = (recipe == MXQ_ABSMAX_PZ || recipe == MXQ_4O6_PZ || recipe == MXQ_BRUTE_PZ) ? 1 : 0;
+    a.ocp_floor = (recipe == MXQ_ABSMAX_OCP) ? 1 : 0;
+    a.xhat = out_xhat;
+    a.xhat_dtype = xhat_dtype;
 
     cudaError_t err;
-    if (recipe == MXQ_BRUTE || recipe == MXQ_BRUTE_PZ) {
+    if (brute) {
         a.n_items = n / (size_t)block_size;
         err = (dtype == MXQ_F32) ? launch_brute_f32(a, block_size, scale_fmt, s)
                                  : launch_brute_bf16(a, block_size, scale_fmt, s);
@@ -71,9 +81,30 @@ int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scal
     }
     const bool dual = (recipe == MXQ_4O6 || recipe == MXQ_4O6_PZ);
     a.n_items = n / (size_t)block_size;
-    err = (dtype == MXQ_F32) ? launch_quantize_f32(a, block_size, scale_fmt, dual, s)
-                             : launch_quantize_bf16(a, block_size, scale_fmt, dual, s);
+    if (out_xhat)
+        err = (dtype == MXQ_F32) ? launch_fake_quantize_f32(a, block_size, scale_fmt, dual, s)
+                                 : launch_fake_quantize_bf16(a, block_size, scale_fmt, dual, s);
+    else
+        err = (dtype == MXQ_F32) ? launch_quantize_f32(a, block_size, scale_fmt, dual, s)
+                                 : launch_quantize_bf16(a, block_size, scale_fmt, dual, s);
     return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+extern "C" {
+
+int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,
+                    const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales, float* out_block_sse,
+                    void* cuda_stream) {
+    if (!out_codes || !out_scales) return MXQ_ERR_NULL;
+    return quantize_common(x, dtype, n, block_size, scale_fmt, recipe, global_scale, d_global_scale, out_codes, out_scales,
+                           out_block_sse, nullptr, MXQ_F32, cuda_stream);
+}
+
+int mxq_fake_quantize(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,
+                      const float* d_global_scale, void* d_out, int out_dtype, void* cuda_stream) {
+    if (!d_out) return MXQ_ERR_NULL;
+    return quantize_common(x, dtype, n, block_size, scale_fmt, recipe, global_scale, d_global_scale, nullptr, nullptr,
+                           nullptr, d_out, out_dtype, cuda_stream);
 }
 
 int mxq_quantize(const float* x, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,

@@ -51,6 +51,14 @@ __device__ __forceinline__ int round_scale(float w) {
     }
 }
 
+// The OCP MX wording of the power-of-two rule: scale exponent = exponent of the (tensor-scale
+// adjusted) block maximum minus the exponent of the largest FP4 value (2), clamped to the codes.
+__device__ __forceinline__ int ocp_scale_code(float u) {
+    const uint32_t b = __float_as_uint(u);               // u >= 0; subnormal u has exponent field 0
+    if (b >= 0x7F800000u) return 254;                    // amax / g overflowed: the largest scale
+    return max((int)(b >> 23) - 2, 0);
+}
+
 // Per-CTA lookup tables: D[c] = fl32(value(c) * g) and R[c] = RN(1 / D[c]), or R[c] = 0 when the
 // multiply-and-correct quotient must not be used with this scale (D zero, tiny, huge or not finite).
 template <int FMT>

@@ -1,0 +1,8 @@
+// Fused fake-quantize kernels (quantize + de-quantize in one pass) instantiated for bf16 input.
+#include "mxq_quantize.cuh"
+
+namespace mxq {
+cudaError_t launch_fake_quantize_bf16(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s) {
+    return launch_quantize_dt<kBF16, true>(a, B, fmt, dual, s);
+}
+}  // namespace mxq

@@ -21,6 +21,9 @@ struct QuantArgs {
     uint8_t* scales;
     float* block_sse;             // may be NULL
     int prevent_zero;
+    int ocp_floor;                // UE8M0 only: scale exponent = exponent of the block maximum - 2
+    void* xhat;                   // fused fake-quantize output (codes / scales may then be NULL), or NULL
+    int xhat_dtype;
 };
 
 int sm_count(int device);
@@ -28,6 +31,8 @@ void count_launch();
 
 cudaError_t launch_quantize_f32(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
 cudaError_t launch_quantize_bf16(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
+cudaError_t launch_fake_quantize_f32(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
+cudaError_t launch_fake_quantize_bf16(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
 cudaError_t launch_brute_f32(const QuantArgs& a, int B, int fmt, cudaStream_t s);
 cudaError_t launch_brute_bf16(const QuantArgs& a, int B, int fmt, cudaStream_t s);
 // Scalar kernel for the few blocks that do not fill a whole chunk (abs-max and 4-over-6 only).

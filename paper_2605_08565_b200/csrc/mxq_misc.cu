@@ -253,7 +253,7 @@ __global__ void k_quantize_tail(QuantArgs p, int dtype, int B, int dual) {
     }
     const bool pz = p.prevent_zero && FMT != kUE8M0;
     const float u = __fdiv_rn(amax, g);
-    int c = round_scale<FMT>(__fdiv_rn(u, 6.0f));
+    int c = (FMT == kUE8M0 && p.ocp_floor) ? ocp_scale_code(u) : round_scale<FMT>(__fdiv_rn(u, 6.0f));
     if (pz) c = max(c, 1);
     float s = tail_eval<FMT>(v, B, c, g, nullptr);
     if (dual) {
@@ -262,9 +262,22 @@ __global__ void k_quantize_tail(QuantArgs p, int dtype, int B, int dual) {
         const float s4 = tail_eval<FMT>(v, B, c4, g, nullptr);
         if (s4 < s) { s = s4; c = c4; }
     }
-    tail_eval<FMT>(v, B, c, g, p.codes + blk * (B / 2));
-    p.scales[blk] = (uint8_t)c;
+    uint8_t packed[8];
+    tail_eval<FMT>(v, B, c, g, packed);
+    if (p.codes)
+        for (int i = 0; i < B / 2; ++i) p.codes[blk * (B / 2) + i] = packed[i];
+    if (p.scales) p.scales[blk] = (uint8_t)c;
     if (p.block_sse) p.block_sse[blk] = s;
+    if (p.xhat) {
+        const float D = __fmul_rn(scale_value(FMT, c), g);
+        for (int i = 0; i < B; ++i) {
+            float q[8];
+            unpack_e2m1x8((uint32_t)((packed[i >> 1] >> ((i & 1) ? 4 : 0)) & 15u), q);
+            const float xh = __fmul_rn(q[0], D);
+            if (p.xhat_dtype == kF32) static_cast<float*>(p.xhat)[blk * B + i] = xh;
+            else static_cast<__nv_bfloat16*>(p.xhat)[blk * B + i] = __float2bfloat16_rn(xh);
+        }
+    }
 }
 
 cudaError_t launch_quantize_tail(const QuantArgs& a, int dtype, int B, int fmt, bool dual, cudaStream_t s) {

@@ -27,6 +27,7 @@
 // outside the ranges these shortcuts need are redone with IEEE divisions (general path).
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "mxq_device.cuh"
@@ -227,10 +228,19 @@ __device__ __forceinline__ void encode_group_general(const float* v, const float
 struct QuantConsts {
     float g, Rg;        // tensor scale and RN(1 / g)
     float m_lo, m_hi;   // a block maximum m takes the shortcuts when m == 0 or m_lo <= m <= m_hi
-    bool unit_g, need_lo, pz, all_short;
+    bool unit_g, need_lo, pz, all_short, ocp;
 };
 
-template <int DT, int B, int FMT, bool DUAL, bool SHORTQ>
+// Scale code for the M = 6 target from u = amax / g: Eq. 2 (Eq. 1 for UE8M0), or the OCP rule.
+template <int FMT, bool EXACT>
+__device__ __forceinline__ int target6_code(float u, bool ocp) {
+    if constexpr (FMT == kUE8M0) {
+        if (ocp) return ocp_scale_code(u);
+    }
+    return round_scale<FMT>(EXACT ? __fdiv_rn(u, 6.0f) : div6_fast(u));
+}
+
+template <int DT, int B, int FMT, bool DUAL, bool SHORTQ, bool FAKE>
 __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
                                                size_t chunk, const uint32_t* raw) {
     using S = QuantShape<DT, B>;
@@ -258,7 +268,7 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             mmax = fmaxf(mmax, a);
             if (k.need_lo) mmin = fminf(mmin, a == 0.0f ? k.m_hi : a);
             u[j] = k.unit_g ? a : quotient_corrected(a, k.g, k.Rg);
-            c6[j] = round_scale<FMT>(div6_fast(u[j]));
+            c6[j] = target6_code<FMT, false>(u[j], k.ocp);
             if (k.pz) c6[j] = max(c6[j], 1);
             E6[j] = T.E[c6[j]];
             wmin = fminf(wmin, E6[j].w);
@@ -283,7 +293,7 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
 #pragma unroll
             for (int j = 0; j < NBG; ++j) {
                 u[j] = __fdiv_rn(m[j], k.g);
-                c6[j] = round_scale<FMT>(__fdiv_rn(u[j], 6.0f));
+                c6[j] = target6_code<FMT, true>(u[j], k.ocp);
                 if (k.pz) c6[j] = max(c6[j], 1);
                 E6[j] = T.E[c6[j]];
                 if constexpr (DUAL) {
@@ -296,11 +306,15 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             if constexpr (DUAL) encode_group_general<B>(v, E4, pk4, sse4);
         }
 
+        float Dw[NBG];   // decode scale of the winner
+#pragma unroll
+        for (int j = 0; j < NBG; ++j) Dw[j] = E6[j].x;
         if constexpr (DUAL) {
             if constexpr (NBG == 1) {
                 const bool take = sse4[0] < sse[0];
                 sse[0] = take ? sse4[0] : sse[0];
                 c6[0] = take ? c4[0] : c6[0];
+                Dw[0] = take ? E4[0].x : Dw[0];
 #pragma unroll
                 for (int i = 0; i < S::GE / 8; ++i) pk[i] = take ? pk4[i] : pk[i];
             } else {
@@ -312,9 +326,32 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
                     const bool tj = sse4[j] < sse[j];
                     sse[j] = tj ? sse4[j] : sse[j];
                     c6[j] = tj ? c4[j] : c6[j];
+                    Dw[j] = tj ? E4[j].x : Dw[j];
                     take |= tj ? (kBlockMask << (j * 4 * B)) : 0u;
                 }
                 pk[0] = (pk4[0] & take) | (pk[0] & ~take);
+            }
+        }
+        if constexpr (FAKE) {   // fused fake-quantize: x_hat = fl32(grid(code) * D), optionally rounded to bf16
+            const size_t e0 = chunk * S::C + (size_t)gi * S::GE;
+#pragma unroll
+            for (int w8 = 0; w8 < S::GE / 8; ++w8) {
+                float q[8];
+                unpack_e2m1x8(pk[w8], q);
+                uint32_t o[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__fmul_rn(q[i], Dw[(w8 * 8 + i) / B]));
+                if (p.xhat_dtype == kF32) {
+                    store_bytes<32>(static_cast<float*>(p.xhat) + e0 + 8 * w8, o);
+                } else {
+                    uint32_t h[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[2 * i]), __uint_as_float(o[2 * i + 1]));
+                        h[i] = *reinterpret_cast<const uint32_t*>(&b2);
+                    }
+                    store_bytes<16>(static_cast<__nv_bfloat16*>(p.xhat) + e0 + 8 * w8, h);
+                }
             }
         }
 #pragma unroll
@@ -326,6 +363,7 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             sw[b] = __float_as_uint(sse[j]);
         }
     }
+    if constexpr (FAKE) return;
     store_bytes<S::C / 2>(p.codes + chunk * (S::C / 2), packed);
     store_bytes<S::NBC>(p.scales + chunk * S::NBC, sc);
     if (p.block_sse) store_bytes<4 * S::NBC>(p.block_sse + chunk * S::NBC, sw);
@@ -347,7 +385,7 @@ __device__ __forceinline__ void stage_chunk(uint32_t slot_addr, const void* src,
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
-template <int DT, int B, int FMT, bool DUAL>
+template <int DT, int B, int FMT, bool DUAL, bool FAKE>
 __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     using S = QuantShape<DT, B>;
     extern __shared__ uint4 ring[];
@@ -358,6 +396,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     k.unit_g = (k.g == 1.0f);
     k.pz = p.prevent_zero && FMT != kUE8M0;
     k.all_short = T.all_short != 0;
+    k.ocp = (FMT == kUE8M0) && p.ocp_floor != 0;
     k.Rg = 1.0f;
     // Ranges of a block maximum m for which u = fl(m / g) and fl(u / 6) come out exact from the
     // multiply-and-correct forms.  The FP8 formats round every u below 2^-20 to code 0, so an
@@ -412,15 +451,15 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
         ahead += stride;
         slot = (slot + 1 == S::SLOTS) ? 0 : slot + 1;
         fill = (fill + 1 == S::SLOTS) ? 0 : fill + 1;
-        if (k.all_short) quantize_chunk<DT, B, FMT, DUAL, true>(p, T, k, chunk, raw);
-        else quantize_chunk<DT, B, FMT, DUAL, false>(p, T, k, chunk, raw);
+        if (k.all_short) quantize_chunk<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, raw);
+        else quantize_chunk<DT, B, FMT, DUAL, false, FAKE>(p, T, k, chunk, raw);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // Host side: pick the instantiation, launch a persistent grid over the whole chunks and hand the
 // blocks past the last whole chunk to the scalar tail kernel.
-template <int DT, int B, int FMT, bool DUAL>
+template <int DT, int B, int FMT, bool DUAL, bool FAKE>
 static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream) {
     using S = QuantShape<DT, B>;
     static int ctas_per_sm[kMaxDevices] = {0};
@@ -429,11 +468,11 @@ static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream)
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (ctas_per_sm[dev] == 0) {
-        err = cudaFuncSetAttribute(k_quantize<DT, B, FMT, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        err = cudaFuncSetAttribute(k_quantize<DT, B, FMT, DUAL, FAKE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)S::RING_BYTES);
         if (err != cudaSuccess) return err;
         int n = 0;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_quantize<DT, B, FMT, DUAL>, kThreads, S::RING_BYTES);
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_quantize<DT, B, FMT, DUAL, FAKE>, kThreads, S::RING_BYTES);
         if (err != cudaSuccess) return err;
         ctas_per_sm[dev] = n > 0 ? n : 1;
     }
@@ -445,7 +484,7 @@ static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream)
         const size_t want = (n_chunks + kThreads - 1) / kThreads;
         const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
         const unsigned grid = (unsigned)(want < cap ? want : cap);
-        k_quantize<DT, B, FMT, DUAL><<<grid, kThreads, S::RING_BYTES, stream>>>(m);
+        k_quantize<DT, B, FMT, DUAL, FAKE><<<grid, kThreads, S::RING_BYTES, stream>>>(m);
         count_launch();
         err = cudaGetLastError();
         if (err != cudaSuccess) return err;
@@ -460,29 +499,30 @@ static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream)
     return err;
 }
 
-template <int DT, int B, int FMT>
+template <int DT, int B, int FMT, bool FAKE>
 static cudaError_t launch_quantize_kind(const QuantArgs& a, bool dual, cudaStream_t s) {
-    return dual ? launch_quantize_inst<DT, B, FMT, true>(a, s) : launch_quantize_inst<DT, B, FMT, false>(a, s);
+    return dual ? launch_quantize_inst<DT, B, FMT, true, FAKE>(a, s) : launch_quantize_inst<DT, B, FMT, false, FAKE>(a, s);
 }
 
-template <int DT, int B>
+template <int DT, int B, bool FAKE>
 static cudaError_t launch_quantize_fmt(const QuantArgs& a, int fmt, bool dual, cudaStream_t s) {
     switch (fmt) {
-    case kUE8M0: return launch_quantize_kind<DT, B, kUE8M0>(a, dual, s);
-    case kUE4M3: return launch_quantize_kind<DT, B, kUE4M3>(a, dual, s);
-    default: return launch_quantize_kind<DT, B, kUE5M3>(a, dual, s);
+    case kUE8M0: return launch_quantize_kind<DT, B, kUE8M0, FAKE>(a, dual, s);
+    case kUE4M3: return launch_quantize_kind<DT, B, kUE4M3, FAKE>(a, dual, s);
+    default: return launch_quantize_kind<DT, B, kUE5M3, FAKE>(a, dual, s);
     }
 }
 
-template <int DT>
+// FAKE = the fused fake-quantize variant (writes x_hat instead of codes, scales and SSE).
+template <int DT, bool FAKE>
 static cudaError_t launch_quantize_dt(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s) {
     switch (B) {
-    case 2: return launch_quantize_fmt<DT, 2>(a, fmt, dual, s);
-    case 4: return launch_quantize_fmt<DT, 4>(a, fmt, dual, s);
-    case 8: return launch_quantize_fmt<DT, 8>(a, fmt, dual, s);
-    case 16: return launch_quantize_fmt<DT, 16>(a, fmt, dual, s);
-    case 32: return launch_quantize_fmt<DT, 32>(a, fmt, dual, s);
-    default: return launch_quantize_fmt<DT, 64>(a, fmt, dual, s);
+    case 2: return launch_quantize_fmt<DT, 2, FAKE>(a, fmt, dual, s);
+    case 4: return launch_quantize_fmt<DT, 4, FAKE>(a, fmt, dual, s);
+    case 8: return launch_quantize_fmt<DT, 8, FAKE>(a, fmt, dual, s);
+    case 16: return launch_quantize_fmt<DT, 16, FAKE>(a, fmt, dual, s);
+    case 32: return launch_quantize_fmt<DT, 32, FAKE>(a, fmt, dual, s);
+    default: return launch_quantize_fmt<DT, 64, FAKE>(a, fmt, dual, s);
     }
 }
 

@@ -76,3 +76,46 @@ def test_reduced_numerical_study_against_oracle():
                 assert np.array_equal(np.array(h["scales"], dtype=np.uint64), osh)
     f = study.findings(res)
     assert f["pz_never_worse"]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", [2, 4, 8, 16, 32, 64])
+def test_ocp_power_of_two_recipe_bit_exact(dtype, B):
+    n = 3 * 256 * max(B, 8) + 5 * 64 + (B if B < 8 else 0)
+    x = inputs.adversarial(n, 21 + B, dtype)
+    for g in (1.0, 0.0131, 2.0 ** -100):
+        xg = x.cuda()
+        codes, scales, sse = mxq.quantize(xg, B, mxq.MXQ_SF_UE8M0, mxq.MXQ_ABSMAX_OCP, g)
+        torch.cuda.synchronize()
+        oc, os_, oe = orc.quantize(inputs.to_numpy_bits(x), B, orc.UE8M0, orc.ABSMAX_OCP, g)
+        assert np.array_equal(scales.cpu().numpy(), os_)
+        assert np.array_equal(codes.cpu().numpy(), oc)
+        assert np.array_equal(sse.cpu().numpy().view(np.uint32), oe.view(np.uint32))
+    with pytest.raises(mxq.MxqError):
+        mxq.quantize(x.cuda(), B, mxq.MXQ_SF_UE4M3, mxq.MXQ_ABSMAX_OCP)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", [2, 4, 8, 16, 32, 64])
+def test_fake_quantize_equals_quantize_then_dequantize(dtype, B):
+    n = 3 * 256 * max(B, 8) + 5 * 64 + (B if B < 8 else 0)
+    x = (inputs.adversarial(n, 33 + B, torch.float32) * 0.25).to(dtype).contiguous()
+    xg = x.cuda()
+    for fmt, recipe, g in ((mxq.MXQ_SF_UE4M3, mxq.MXQ_ABSMAX, 1.0), (mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6_PZ, 0.0131),
+                           (mxq.MXQ_SF_UE5M3, mxq.MXQ_4O6, 1.0), (mxq.MXQ_SF_UE8M0, mxq.MXQ_ABSMAX_OCP, 1.0),
+                           (mxq.MXQ_SF_UE8M0, mxq.MXQ_ABSMAX, 3.0e-37)):
+        for odt, oid in ((torch.float32, orc.F32), (torch.bfloat16, orc.BF16)):
+            out = torch.empty(n, dtype=odt, device="cuda")
+            mxq.mxq_fake_quantize(xg, n, B, fmt, recipe, g, None, out)
+            codes, scales, _ = mxq.quantize(xg, B, fmt, recipe, g)
+            two_step = torch.empty(n, dtype=odt, device="cuda")
+            mxq.mxq_dequantize(codes, scales, n, B, fmt, g, two_step)
+            torch.cuda.synchronize()
+            got = inputs.to_numpy_bits(out)
+            view = np.uint32 if odt == torch.float32 else np.uint16
+            assert np.array_equal(got.view(view), inputs.to_numpy_bits(two_step).view(view))
+            want = orc.fake_quantize(inputs.to_numpy_bits(x), B, fmt, recipe, g, oid)
+            assert np.array_equal(got.view(view), want.view(view))
+    out = torch.empty(n, dtype=torch.float32, device="cuda")
+    with pytest.raises(mxq.MxqError):
+        mxq.mxq_fake_quantize(xg, n, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_BRUTE, 1.0, None, out)
