@@ -20,9 +20,9 @@
 // D_c = Dref * 2^k, as long as D_c is a normal number.  Hence fl(v / D_c) = fl(v / Dref) * 2^-k
 // exactly: the correctly rounded quotient is formed once per class and element, and a candidate
 // costs one multiply by a power of two, the FP4 rounding, and the two FMAs of the SSE.  Codes
-// whose decode scale is zero, subnormal, not finite or above 2^126, and threads holding a magnitude
-// above 2^60 or a nonzero one below 2^-62, take the general path (IEEE division), candidate by
-// candidate.
+// whose decode scale is zero, subnormal or above 2^126 need no quotient at all (every element
+// rounds to zero, or saturates) and form one more list.  Threads holding a magnitude above 2^60
+// or a nonzero one below 2^-62 take the general path (IEEE division), candidate by candidate.
 //
 // Inside a class the members are visited in ascending code order and the smallest SSE bit pattern
 // is kept with a strict compare (SSE >= 0, so integer order is float order and the first of equals
@@ -45,67 +45,72 @@ __device__ __forceinline__ int code_class(int c) {
     return (int)((0x64204000u >> (4 * c)) & 7u);
 }
 
-// Per-CTA tables of the search.  A code is "paired" when its decode scale is a normal number with
-// a biased exponent of at most 253, so that D = Dref * 2^k and 2^-k are both representable.  The
-// paired codes of a mantissa class form two lists: kind 1 holds the codes whose -D is exactly
-// representable in f16 (their residual is one mixed-precision FMA from the unpacked f16 grid
-// value), kind 0 the others (f16 -> f32 convert, then an FFMA).  List index = 2 * class + kind.
-constexpr int kLists = 16;
+// Per-CTA tables of the search.  Every code with a finite decode scale D sits in one candidate list:
+//   * D normal with a biased exponent of at most 253 ("paired": D = Dref * 2^k and 2^-k are both
+//     representable): list 2 * class + kind, where kind 1 holds the codes whose -D is exactly
+//     representable in f16 (their residual is one mixed-precision FMA from the unpacked f16 grid
+//     value) and kind 0 the others (f16 -> f32 convert, then an FFMA);
+//   * the "flat" list kFlatList for the rest.  D = 0 or D >= 2^127: every quotient of a magnitude
+//     <= 2^60 rounds to FP4 zero, so the candidate is entered with the multiplier 0.  D subnormal:
+//     every nonzero magnitude >= 2^-62 divided by it exceeds 2^64 and saturates at 6, so it is
+//     entered with the multiplier 2^126.  The flat list is evaluated on the elements themselves
+//     (Dref = 1), which needs no quotient.
+constexpr int kLists = 17;
+constexpr int kFlatList = 16;
+constexpr int kCandSlots = 16 * kMaxMembers + 256;
 struct BruteTables {
     float D[256];            // decode scale of the code; NaN for codes that do not exist
     float R[256];            // RN(1 / D) when 2^-60 <= D <= 2^60, else 0 (used by the final encode)
-    float4 cand[kLists * kMaxMembers];    // per list, ascending code order: (-D, 2^-k, f16(-D) twice as bits, 0)
-    uint8_t member[kLists * kMaxMembers]; // the code of each slot of cand[]
-    uint8_t kind[256];       // 0, 1 as above; 2 = not paired
+    float4 cand[kCandSlots];    // per list, ascending code order: (-D, multiplier, f16(-D) twice as bits, 0)
+    uint8_t member[kCandSlots]; // the code of each slot of cand[]
+    uint8_t kind[256];       // 0, 1 paired as above; 3 = flat list; 2 = not a candidate
     float clsD[8];           // Dref of the class, in [1, 2)
     float clsR[8];           // RN(1 / Dref)
     int cnt[kLists];         // members per list
-    uint32_t kind_mask[2][8];
-    uint32_t unpaired_mask[8];
-    int n_unpaired;          // codes with a finite decode scale that are not paired
-    uint8_t unpaired[256];   // ... in ascending order
+    uint32_t kind_mask[3][8];
 };
 
 template <int FMT>
 __device__ __forceinline__ int members_base(int list) {
-    // the power-of-two format has one class: its two lists get half of the array each
-    return FMT == kUE8M0 ? list * (kLists * kMaxMembers / 2) : list * kMaxMembers;
+    if (list == kFlatList) return 16 * kMaxMembers;
+    // the power-of-two format has one class: its two lists get half of the class area each
+    return FMT == kUE8M0 ? list * (16 * kMaxMembers / 2) : list * kMaxMembers;
 }
 
+// first: smallest admissible code (1 under prevent-zero for the FP8 formats, else 0).
 template <int FMT>
-__device__ __forceinline__ void build_brute_tables(BruteTables& T, float g) {
+__device__ __forceinline__ void build_brute_tables(BruteTables& T, float g, int first) {
     static_assert(kThreads == 256, "one thread per table entry");
     build_scale_tables<FMT>(T.D, T.R, g);
     const int c = threadIdx.x;
     const float D = T.D[c];
     const uint32_t b = __float_as_uint(D);
     const uint32_t e = (b >> 23) & 0xFFu;
-    const bool is_paired = c < num_codes(FMT) && (b >> 31) == 0 && e >= 1 && e <= 253;
+    const bool usable = c >= first && c < num_codes(FMT) && (b >> 31) == 0 && e != 255;
+    const bool is_paired = usable && e >= 1 && e <= 253;
     const __half hD = __float2half_rn(-D);
-    const int kind = !is_paired ? 2 : (__half2float(hD) == -D ? 1 : 0);
+    const int kind = !usable ? 2 : (!is_paired ? 3 : (__half2float(hD) == -D ? 1 : 0));
     T.kind[c] = (uint8_t)kind;
     if (c < kLists) T.cnt[c] = 0;
     const uint32_t ballot0 = __ballot_sync(0xFFFFFFFFu, kind == 0);
     const uint32_t ballot1 = __ballot_sync(0xFFFFFFFFu, kind == 1);
-    // codes left to the general path: finite decode scale (zero and subnormal included), not paired
-    const bool is_unpaired = c < num_codes(FMT) && !is_paired && (b & 0x7FFFFFFFu) < 0x7F800000u;
-    const uint32_t ballot_u = __ballot_sync(0xFFFFFFFFu, is_unpaired);
+    const uint32_t ballot3 = __ballot_sync(0xFFFFFFFFu, kind == 3);
     if ((c & 31) == 0) {
         T.kind_mask[0][c >> 5] = ballot0;
         T.kind_mask[1][c >> 5] = ballot1;
-        T.unpaired_mask[c >> 5] = ballot_u;
+        T.kind_mask[2][c >> 5] = ballot3;
     }
     __syncthreads();
     const uint32_t below = (1u << (c & 31)) - 1u;
-    if (is_unpaired) {
-        int rank = __popc(ballot_u & below);
-        for (int w = 0; w < (c >> 5); ++w) rank += __popc(T.unpaired_mask[w]);
-        T.unpaired[rank] = (uint8_t)c;
-    }
-    if (c == 0) {
-        int n = 0;
-        for (int w = 0; w < 8; ++w) n += __popc(T.unpaired_mask[w]);
-        T.n_unpaired = n;
+    if (kind == 3) {
+        int rank = __popc(ballot3 & below);
+        for (int w = 0; w < (c >> 5); ++w) rank += __popc(T.kind_mask[2][w]);
+        // multiplier 0 -> every quotient is zero; 2^126 -> every nonzero quotient saturates
+        const float P = (e == 0 && D != 0.0f) ? __uint_as_float(0x7E800000u) : 0.0f;
+        const int slot = members_base<FMT>(kFlatList) + rank;
+        T.cand[slot] = make_float4(-D, P, 0.0f, 0.0f);
+        T.member[slot] = (uint8_t)c;
+        atomicAdd(&T.cnt[kFlatList], 1);
     }
     if (is_paired) {
         const int cls = code_class<FMT>(c);
@@ -314,8 +319,8 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
 
     __shared__ BruteTables T;
     const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    build_brute_tables<FMT>(T, g);
     const int first = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
+    build_brute_tables<FMT>(T, g, first);
 
     const size_t stride = (size_t)gridDim.x * kThreads;
     for (size_t grp = (size_t)blockIdx.x * kThreads + threadIdx.x; grp < p.n_items; grp += stride) {
@@ -351,14 +356,13 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
                 search_list<B, FMT, false>(T, 2 * cls, v2, tb, best);
                 search_list<B, FMT, true>(T, 2 * cls + 1, v2, tb, best);
             }
+            search_list<B, FMT, false>(T, kFlatList, v2, v2, best);   // Dref = 1: the elements are their own quotients
         }
 
-        // candidates on the general path (decode scale zero, subnormal or huge; all candidates when
-        // the thread holds a magnitude above 2^60 or a nonzero one below 2^-62)
-        const int n_general = fast_ok ? T.n_unpaired : num_codes(FMT);
-        for (int j = 0; j < n_general; ++j) {
-            const int c = fast_ok ? (int)T.unpaired[j] : j;
-            if (c < first) continue;
+        // general path (IEEE division), candidate by candidate: threads that hold a magnitude above
+        // 2^60 or a nonzero one below 2^-62
+        const int n_general = fast_ok ? 0 : num_codes(FMT);
+        for (int c = first; c < n_general; ++c) {
             const float D = T.D[c];
             if (!(fabsf(D) <= 3.402823466e38f)) continue;  // decode scale overflowed: not usable
             if constexpr (!SKEW) {
