@@ -219,6 +219,14 @@ int mxq_histograms(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, in
 int mxq_segment_mse(const float* d_block_sse, size_t n_blocks, size_t blocks_per_segment, size_t elems_per_segment,
                     double* d_out_mse, void* cuda_stream);
 
+/*
+ * mxq_mask_interval -- the pre-quantization diagnostic of the appendix ("masking specific magnitude
+ * intervals to zero" at full precision): out_i = 0 when lo <= |x_i| < hi, else x_i.
+ *   x, d_out   device, n elements of dtype (MXQ_F32 or MXQ_BF16); d_out may be x (in place).
+ *   lo, hi     0 <= lo <= hi, else MXQ_ERR_BAD_SCALE.  NaN entries pass unchanged.
+ */
+int mxq_mask_interval(const void* x, int dtype, size_t n, float lo, float hi, void* d_out, void* cuda_stream);
+
 /* Number of kernels the library has launched in this process (all entry points), for
  * accounting in benchmarks. */
 unsigned long long mxq_launch_count(void);

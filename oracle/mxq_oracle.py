@@ -197,3 +197,15 @@ def fake_quantize(x, block_size: int, fmt: int, recipe: int, g: float = 1.0, out
     """dequantize(quantize(x)): what a model sees when its weights or activations are quantized."""
     codes, scales, _ = quantize(x, block_size, fmt, recipe, g, threads)
     return dequantize(codes, scales, np.ascontiguousarray(x).size, block_size, fmt, g, out_dtype)
+
+
+def mask_interval(x, lo: float, hi: float):
+    """Magnitude-interval masking of the appendix ablation: entries with lo <= |x| < hi become zero
+    (+0), all others pass unchanged.  x: float32 array or uint16 bf16 bit patterns; same type out."""
+    x = np.ascontiguousarray(x)
+    if x.dtype == np.uint16:
+        mag = (x.astype(np.uint32) << 16).view(np.float32)
+        keep = ~((np.abs(mag) >= np.float32(lo)) & (np.abs(mag) < np.float32(hi)))
+        return np.where(keep, x, np.uint16(0)).astype(np.uint16)
+    keep = ~((np.abs(x) >= np.float32(lo)) & (np.abs(x) < np.float32(hi)))
+    return np.where(keep, x, np.float32(0.0)).astype(np.float32)

@@ -20,7 +20,7 @@ MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ, MXQ_ABS
 
 EXPORTS = (
     "mxq_quantize", "mxq_quantize_ex", "mxq_fake_quantize", "mxq_tensor_amax", "mxq_global_scale_from_amax",
-    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_launch_count",
+    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_mask_interval", "mxq_launch_count",
     "mxq_status_string", "mxq_last_cuda_error", "mxq_version",
 )
 
@@ -67,6 +67,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_histograms.argtypes = [vp, vp, sz, i32, vp, vp, vp]
     L.mxq_segment_mse.restype = i32
     L.mxq_segment_mse.argtypes = [vp, sz, sz, sz, vp, vp]
+    L.mxq_mask_interval.restype = i32
+    L.mxq_mask_interval.argtypes = [vp, i32, sz, f32, f32, vp, vp]
     L.mxq_launch_count.restype = c.c_ulonglong
     L.mxq_launch_count.argtypes = []
     L.mxq_status_string.restype = c.c_char_p
@@ -176,6 +178,10 @@ def mxq_histograms(d_codes, d_scales, n, block_size, d_code_hist, d_scale_hist, 
 def mxq_segment_mse(d_block_sse, n_blocks, blocks_per_segment, elems_per_segment, d_out_mse, stream=None) -> None:
     _check(load_library().mxq_segment_mse(_ptr(d_block_sse), n_blocks, blocks_per_segment, elems_per_segment,
                                           _ptr(d_out_mse), _stream(stream)))
+
+
+def mxq_mask_interval(x, n, lo, hi, d_out, stream=None) -> None:
+    _check(load_library().mxq_mask_interval(_ptr(x), _dtype_id(x), n, lo, hi, _ptr(d_out), _stream(stream)))
 
 
 def mxq_launch_count() -> int:

@@ -209,6 +209,16 @@ int mxq_segment_mse(const float* d_block_sse, size_t n_blocks, size_t blocks_per
     return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
 }
 
+int mxq_mask_interval(const void* x, int dtype, size_t n, float lo, float hi, void* d_out, void* cuda_stream) {
+    if (!x || !d_out) return MXQ_ERR_NULL;
+    if (dtype != MXQ_F32 && dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
+    if (n == 0) return MXQ_ERR_BAD_SHAPE;
+    if (!(lo >= 0.0f) || !(hi >= lo)) return MXQ_ERR_BAD_SCALE;
+    if (!aligned16(x) || !aligned16(d_out)) return MXQ_ERR_ALIGN;
+    cudaError_t err = launch_mask_interval(x, dtype, n, lo, hi, d_out, static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
 unsigned long long mxq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* mxq_status_string(int status) {

@@ -53,6 +53,8 @@ cudaError_t launch_histograms(const uint8_t* codes, const uint8_t* scales, size_
 cudaError_t launch_segment_mse(const float* sse, size_t n_segments, size_t blocks_per_segment, size_t elems_per_segment,
                                double* out, cudaStream_t s);
 
+cudaError_t launch_mask_interval(const void* x, int dtype, size_t n, float lo, float hi, void* out, cudaStream_t s);
+
 constexpr int kMsePartials = 1024;  // fixed first-level width of the MSE tree
 
 }  // namespace mxq

@@ -70,6 +70,54 @@ def rank_seed(base_seed: int, rank: int, index: int = 0) -> int:
     return int(base_seed) * 1_000_003 + int(rank) * 1009 + int(index)
 
 
+# ------------------------------------------------------------------------------------------------
+# One tensor sharded by rows over the ranks (blocks are independent, so whole rows of blocks go to
+# one rank).  Only hierarchical scaling and the tensor MSE need an exchange: one MAX all-reduce of
+# the tensor abs-max (exact, order-free) and one gather of the per-rank SSE sums, added in rank
+# order in binary64 so that the result does not depend on arrival order.
+# ------------------------------------------------------------------------------------------------
+def row_shard(n_rows: int, rank: int, world: int) -> tuple[int, int]:
+    """[first, last) rows of `rank` when n_rows are dealt out in contiguous, nearly equal ranges."""
+    return n_rows * rank // world, n_rows * (rank + 1) // world
+
+
+def global_amax(local_amax: torch.Tensor) -> torch.Tensor:
+    """MAX all-reduce of a one-element float32 tensor holding this rank's abs-max (in place)."""
+    if dist.is_initialized():
+        dist.all_reduce(local_amax, op=dist.ReduceOp.MAX)
+    return local_amax
+
+
+def global_mse(local_sse_sum: float, n_total: int) -> float:
+    """Tensor MSE from the per-rank sums of block SSE: gathered, then added in rank order."""
+    if not dist.is_initialized():
+        return float(local_sse_sum) / n_total
+    mine = torch.tensor([float(local_sse_sum)], dtype=torch.float64, device=_device())
+    parts = [torch.zeros_like(mine) for _ in range(dist.get_world_size())]
+    dist.all_gather(parts, mine)
+    total = 0.0
+    for p in parts:
+        total += float(p.item())
+    return total / n_total
+
+
+def sharded_hierarchical_quantize(x_local: torch.Tensor, n_total: int, block_size: int, scale_fmt: int, recipe: int):
+    """Quantize this rank's rows of a tensor that is sharded by rows, with ONE tensor scale
+    g = amax_of_the_whole_tensor / (6 * 448) shared by all ranks.  Returns (codes, scales, block_sse,
+    g tensor on the device, tensor MSE of the whole tensor).  Every rank reads only its own memory."""
+    from . import binding as mxq
+    n = x_local.numel()
+    amax = torch.empty(1, dtype=torch.float32, device=x_local.device)
+    mxq.mxq_tensor_amax(x_local, n, amax)
+    global_amax(amax)
+    g = mxq.mxq_global_scale_from_amax(float(amax.item()))
+    dg = torch.tensor([g], dtype=torch.float32, device=x_local.device)
+    codes, scales, sse = mxq.quantize(x_local, block_size, scale_fmt, recipe, 1.0, dg)
+    local_mse = mxq.tensor_mse(sse, n)                      # deterministic local tree
+    mse = global_mse(float(local_mse.item()) * n, n_total)
+    return codes, scales, sse, dg, mse
+
+
 def shutdown() -> None:
     if dist.is_initialized():
         dist.destroy_process_group()

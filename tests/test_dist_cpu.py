@@ -20,6 +20,10 @@ def _worker(rank, world, port, out):
     dist.barrier()
     # rank r processed (r+1)*1000 units in (r+1)*0.5 s: whole job = 3000 units / max time 1.0 s
     value, t = dist.whole_job_throughput((rank + 1) * 1000.0, (rank + 1) * 0.5)
+    import torch
+    amax = dist.global_amax(torch.tensor([1.5 + rank], dtype=torch.float32))
+    mse = dist.global_mse(10.0 * (rank + 1), 60)
+    assert float(amax) == 2.5 and mse == 0.5, (float(amax), mse)
     out.put((rank, value, t, dist.reduce_max(rank), dist.reduce_sum(rank + 1)))
     dist.barrier()
     dist.shutdown()
@@ -46,3 +50,9 @@ def test_rank_seeds_never_collide_and_single_process_is_a_no_op():
     assert len(seeds) == 64
     assert dist.reduce_max(3.5) == 3.5 and dist.reduce_sum(2.0) == 2.0
     assert dist.whole_job_throughput(10.0, 2.0) == (5.0, 2.0)
+    # row shards tile the rows without gaps or overlap
+    for rows, world in ((4096, 8), (1000, 3), (7, 8)):
+        edges = [dist.row_shard(rows, r, world) for r in range(world)]
+        assert edges[0][0] == 0 and edges[-1][1] == rows
+        assert all(a[1] == b[0] for a, b in zip(edges[:-1], edges[1:]))
+    assert dist.global_mse(12.0, 48) == 0.25

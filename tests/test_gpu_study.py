@@ -119,3 +119,26 @@ def test_fake_quantize_equals_quantize_then_dequantize(dtype, B):
     out = torch.empty(n, dtype=torch.float32, device="cuda")
     with pytest.raises(mxq.MxqError):
         mxq.mxq_fake_quantize(xg, n, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_BRUTE, 1.0, None, out)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_mask_interval_matches_definition(dtype):
+    for n in (1, 7, 8, 4096 + 5):
+        x = (inputs.normal(max(n, 8), 4 + n, 0.02, torch.float32)[:n]).to(dtype).contiguous()
+        xg = x.cuda()
+        out = torch.empty_like(xg)
+        for lo, hi in ((0.0, 0.0), (0.005, 0.015), (0.0, 0.035), (0.02, 1.0e9)):
+            mxq.mxq_mask_interval(xg, n, lo, hi, out)
+            torch.cuda.synchronize()
+            want = orc.mask_interval(inputs.to_numpy_bits(x), lo, hi)
+            got = inputs.to_numpy_bits(out)
+            view = np.uint32 if dtype == torch.float32 else np.uint16
+            assert np.array_equal(got.view(view), want.view(view)), (n, lo, hi)
+    y = xg.clone()
+    mxq.mxq_mask_interval(y, n, 0.005, 0.015, y)             # in place
+    mxq.mxq_mask_interval(xg, n, 0.005, 0.015, out)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16 if dtype == torch.bfloat16 else torch.int32),
+                       out.view(torch.int16 if dtype == torch.bfloat16 else torch.int32))
+    with pytest.raises(mxq.MxqError):
+        mxq.mxq_mask_interval(xg, n, 0.02, 0.01, out)

@@ -116,3 +116,22 @@ def test_fake_quantize_is_dequantize_of_quantize():
         S = np.array([orc.scale_value(fmt, int(c)) for c in scales], dtype=np.float32) * np.float32(g)
         ratio = np.abs(xh.reshape(-1, 16)) / S[:, None]
         assert np.all(np.isin(np.round(ratio * 2) / 2, [0, .5, 1, 1.5, 2, 3, 4, 6]))
+
+
+def test_mask_interval_definition():
+    x = np.array([0.0, -0.0, 0.01, -0.01, 0.02, 0.0199999, -0.035, 0.5, 1e-30], dtype=np.float32)
+    out = orc.mask_interval(x, 0.01, 0.02)
+    assert np.array_equal(out, np.array([0.0, -0.0, 0.0, 0.0, 0.02, 0.0, -0.035, 0.5, 1e-30], dtype=np.float32))
+    assert np.array_equal(orc.mask_interval(x, 0.0, 0.0), x)                       # empty interval
+    assert np.count_nonzero(orc.mask_interval(x, 0.0, 1.0)) == 0                   # everything below 1 goes
+    rng = np.random.default_rng(1)
+    y = (rng.standard_normal(4096) * 0.02).astype(np.float32)
+    lo, hi = 0.005, 0.015
+    m = orc.mask_interval(y, lo, hi)
+    inside = (np.abs(y) >= lo) & (np.abs(y) < hi)
+    assert np.count_nonzero(m) == y.size - inside.sum() and np.array_equal(m[~inside], y[~inside])
+    # bf16 bit patterns in, bf16 bit patterns out
+    yb = (y.view(np.uint32) >> 16).astype(np.uint16)
+    mb = orc.mask_interval(yb, lo, hi)
+    yf = (yb.astype(np.uint32) << 16).view(np.float32)
+    assert np.array_equal(mb == 0, ((np.abs(yf) >= lo) & (np.abs(yf) < hi)) | (yb == 0))
