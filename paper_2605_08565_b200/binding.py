@@ -108,10 +108,16 @@ def _dtype_id(t: torch.Tensor) -> int:
     raise MxqError(f"unsupported dtype {t.dtype}")
 
 
-def _stream(stream) -> int:
-    if stream is None:
-        stream = torch.cuda.current_stream()
-    return stream.cuda_stream
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
+def _stream(stream, like=None) -> int:
+    """cudaStream_t of `stream`, or of torch's current stream on the device of tensor `like`."""
+    if stream is not None:
+        return stream.cuda_stream
+    if _raw_stream is not None and like is not None and like.is_cuda:
+        return _raw_stream(like.device.index if like.device.index is not None else torch.cuda.current_device())
+    return torch.cuda.current_stream().cuda_stream
 
 
 # ---- C-ABI names ---------------------------------------------------------------------------
@@ -126,17 +132,17 @@ def mxq_quantize_ex(x, n, block_size, scale_fmt, recipe, global_scale, d_global_
                     out_block_sse, stream=None) -> None:
     _check(load_library().mxq_quantize_ex(_ptr(x), _dtype_id(x), n, block_size, scale_fmt, recipe, global_scale,
                                           _ptr(d_global_scale), _ptr(out_codes), _ptr(out_scales),
-                                          _ptr(out_block_sse), _stream(stream)))
+                                          _ptr(out_block_sse), _stream(stream, x)))
 
 
 def mxq_fake_quantize(x, n, block_size, scale_fmt, recipe, global_scale, d_global_scale, d_out, stream=None) -> None:
     _check(load_library().mxq_fake_quantize(_ptr(x), _dtype_id(x), n, block_size, scale_fmt, recipe, global_scale,
-                                            _ptr(d_global_scale), _ptr(d_out), _dtype_id(d_out), _stream(stream)))
+                                            _ptr(d_global_scale), _ptr(d_out), _dtype_id(d_out), _stream(stream, x)))
 
 
 def mxq_tensor_amax(x, n, d_out_amax, d_out_global_scale=None, stream=None) -> None:
     _check(load_library().mxq_tensor_amax(_ptr(x), _dtype_id(x), n, _ptr(d_out_amax), _ptr(d_out_global_scale),
-                                          _stream(stream)))
+                                          _stream(stream, x)))
 
 
 def mxq_global_scale_from_amax(amax: float) -> float:
@@ -150,38 +156,38 @@ def mxq_tensor_mse_workspace_bytes(n_blocks: int) -> int:
 def mxq_tensor_mse(d_block_sse, n_blocks, n, d_out_mse, d_workspace, stream=None) -> None:
     ws_bytes = d_workspace.numel() * d_workspace.element_size() if d_workspace is not None else 0
     _check(load_library().mxq_tensor_mse(_ptr(d_block_sse), n_blocks, n, _ptr(d_out_mse), _ptr(d_workspace),
-                                         ws_bytes, _stream(stream)))
+                                         ws_bytes, _stream(stream, d_block_sse)))
 
 
 def mxq_tensor_mse_static(d_block_sse, n_blocks, n, d_out_mse, stream=None) -> None:
     """Tensor MSE with the library's built-in scratch array: no workspace argument, nothing allocated."""
-    _check(load_library().mxq_tensor_mse_static(_ptr(d_block_sse), n_blocks, n, _ptr(d_out_mse), _stream(stream)))
+    _check(load_library().mxq_tensor_mse_static(_ptr(d_block_sse), n_blocks, n, _ptr(d_out_mse), _stream(stream, d_block_sse)))
 
 
 def mxq_dequantize(d_codes, d_scales, n, block_size, scale_fmt, global_scale, d_out, stream=None) -> None:
     _check(load_library().mxq_dequantize(_ptr(d_codes), _ptr(d_scales), n, block_size, scale_fmt, global_scale,
-                                         _ptr(d_out), _dtype_id(d_out), _stream(stream)))
+                                         _ptr(d_out), _dtype_id(d_out), _stream(stream, d_out)))
 
 
 def mxq_block_clip_sse(x, n, block_size, scale_fmt, global_scale, d_global_scale, d_scales, out_clip_sse,
                        stream=None) -> None:
     _check(load_library().mxq_block_clip_sse(_ptr(x), _dtype_id(x), n, block_size, scale_fmt, global_scale,
-                                             _ptr(d_global_scale), _ptr(d_scales), _ptr(out_clip_sse), _stream(stream)))
+                                             _ptr(d_global_scale), _ptr(d_scales), _ptr(out_clip_sse), _stream(stream, x)))
 
 
 def mxq_histograms(d_codes, d_scales, n, block_size, d_code_hist, d_scale_hist, stream=None) -> None:
     """d_code_hist: 16 and d_scale_hist: 256 int64/uint64 CUDA counters; counts are added to them."""
     _check(load_library().mxq_histograms(_ptr(d_codes), _ptr(d_scales), n, block_size, _ptr(d_code_hist),
-                                         _ptr(d_scale_hist), _stream(stream)))
+                                         _ptr(d_scale_hist), _stream(stream, d_codes)))
 
 
 def mxq_segment_mse(d_block_sse, n_blocks, blocks_per_segment, elems_per_segment, d_out_mse, stream=None) -> None:
     _check(load_library().mxq_segment_mse(_ptr(d_block_sse), n_blocks, blocks_per_segment, elems_per_segment,
-                                          _ptr(d_out_mse), _stream(stream)))
+                                          _ptr(d_out_mse), _stream(stream, d_block_sse)))
 
 
 def mxq_mask_interval(x, n, lo, hi, d_out, stream=None) -> None:
-    _check(load_library().mxq_mask_interval(_ptr(x), _dtype_id(x), n, lo, hi, _ptr(d_out), _stream(stream)))
+    _check(load_library().mxq_mask_interval(_ptr(x), _dtype_id(x), n, lo, hi, _ptr(d_out), _stream(stream, x)))
 
 
 def mxq_launch_count() -> int:

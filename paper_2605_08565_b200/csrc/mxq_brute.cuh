@@ -318,6 +318,7 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
     constexpr float kTiny = 2.168404344971009e-19f;  // 2^-62
 
     __shared__ BruteTables T;
+    wait_for_prior_grid();
     const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
     const int first = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     build_brute_tables<FMT>(T, g, first);
@@ -494,9 +495,8 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
         const size_t want = (n_groups + kThreads - 1) / kThreads;
         const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
         const unsigned grid = (unsigned)(want < cap ? want : cap);
-        k_brute<DT, B, FMT><<<grid, kThreads, 0, stream>>>(m);
+        err = launch_pdl(k_brute<DT, B, FMT>, grid, kThreads, 0, stream, m);
         count_launch();
-        err = cudaGetLastError();
         if (err != cudaSuccess) return err;
     }
     if constexpr (B < 32) {

@@ -13,6 +13,10 @@ constexpr int kF32 = 0, kBF16 = 1;
 constexpr int kUE8M0 = 0, kUE4M3 = 1, kUE5M3 = 2;
 constexpr int kThreads = 256;
 
+// See launch_pdl(): holds a programmatically staged grid until the kernel before it in the stream
+// has completed and its writes are visible.
+__device__ __forceinline__ void wait_for_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __host__ __device__ constexpr int num_codes(int fmt) { return fmt == kUE4M3 ? 127 : 255; }
 __host__ __device__ constexpr int elem_bytes(int dt) { return dt == kF32 ? 4 : 2; }
 

@@ -27,6 +27,26 @@ struct QuantArgs {
 };
 
 int sm_count(int device);
+
+// Launch with programmatic stream serialization: the grid may be staged while the kernel before
+// it in the stream still runs.  EVERY kernel launched this way calls wait_for_prior_grid() before
+// its first access to global memory; the wait returns once that kernel has completed and its
+// writes are visible (at once when there is nothing to wait for).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 void count_launch();
 
 cudaError_t launch_quantize_f32(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);

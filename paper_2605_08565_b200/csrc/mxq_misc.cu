@@ -70,6 +70,7 @@ __global__ void __launch_bounds__(kThreads) k_tensor_amax(const void* x, size_t 
 
 // g = amax / (6 * 448): the tensor maximum maps to the top of FP4 times the top of E4M3.
 __global__ void k_global_scale(const float* amax, float* g) {
+    wait_for_prior_grid();
     const float a = *amax;
     *g = (a > 0.0f && a <= 3.402823466e38f) ? __fdiv_rn(a, 2688.0f) : 1.0f;
 }
@@ -91,9 +92,8 @@ cudaError_t launch_tensor_amax(const void* x, int dtype, size_t n, float* d_amax
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     if (d_g) {
-        k_global_scale<<<1, 1, 0, s>>>(d_amax, d_g);
+        err = launch_pdl(k_global_scale, 1u, 1u, 0, s, (const float*)d_amax, d_g);
         count_launch();
-        err = cudaGetLastError();
     }
     return err;
 }
@@ -118,6 +118,7 @@ __device__ __forceinline__ double cta_tree_sum(double v, double* sh) {
 
 __global__ void __launch_bounds__(kThreads) k_mse_partial(const float* sse, size_t nb, size_t slice, double* partials) {
     __shared__ double sh[kThreads];
+    wait_for_prior_grid();
     const size_t lo = (size_t)blockIdx.x * slice;
     const size_t hi = (lo + slice < nb) ? lo + slice : nb;
     double acc = 0.0;
@@ -128,6 +129,7 @@ __global__ void __launch_bounds__(kThreads) k_mse_partial(const float* sse, size
 
 __global__ void __launch_bounds__(kMsePartials) k_mse_final(const double* partials, int n_partials, double n, double* out) {
     __shared__ double sh[kMsePartials];
+    wait_for_prior_grid();
     const double v = (int)threadIdx.x < n_partials ? partials[threadIdx.x] : 0.0;
     const double total = cta_tree_sum<kMsePartials>(v, sh);
     if (threadIdx.x == 0) *out = __ddiv_rn(total, n);
@@ -138,13 +140,13 @@ cudaError_t launch_tensor_mse(const float* d_sse, size_t n_blocks, size_t n, dou
     size_t P = (n_blocks + kThreads - 1) / kThreads;
     if (P > (size_t)kMsePartials) P = kMsePartials;
     const size_t slice = (n_blocks + P - 1) / P;
-    k_mse_partial<<<(unsigned)P, kThreads, 0, s>>>(d_sse, n_blocks, slice, d_partials);
+    // staged launches: the launch latency of these two small kernels comes off the critical path
+    cudaError_t err = launch_pdl(k_mse_partial, (unsigned)P, kThreads, 0, s, d_sse, n_blocks, slice, d_partials);
     count_launch();
-    cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-    k_mse_final<<<1, kMsePartials, 0, s>>>(d_partials, (int)P, (double)n, d_out);
+    err = launch_pdl(k_mse_final, 1u, (unsigned)kMsePartials, 0, s, (const double*)d_partials, (int)P, (double)n, d_out);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -158,6 +160,7 @@ __device__ __forceinline__ float decode_scale(int fmt, int c, float g) {
 template <int ODT>
 __global__ void __launch_bounds__(kThreads) k_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n,
                                                          int log2B, int fmt, float g, void* out) {
+    wait_for_prior_grid();
     const size_t n8 = n >> 3;
     const size_t stride = (size_t)gridDim.x * kThreads;
     for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n8; i += stride) {
@@ -210,10 +213,10 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_
     if (want == 0) want = 1;
     const size_t cap = (size_t)sm_count(dev) * 8;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
-    if (out_dtype == kF32) k_dequantize<kF32><<<grid, kThreads, 0, s>>>(codes, scales, n, log2B, fmt, g, out);
-    else k_dequantize<kBF16><<<grid, kThreads, 0, s>>>(codes, scales, n, log2B, fmt, g, out);
+    if (out_dtype == kF32) err = launch_pdl(k_dequantize<kF32>, grid, kThreads, 0, s, codes, scales, n, log2B, fmt, g, out);
+    else err = launch_pdl(k_dequantize<kBF16>, grid, kThreads, 0, s, codes, scales, n, log2B, fmt, g, out);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 // ------------------------------------------------------------------------------------------------

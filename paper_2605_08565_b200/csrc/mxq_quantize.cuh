@@ -390,6 +390,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     using S = QuantShape<DT, B>;
     extern __shared__ uint4 ring[];
     __shared__ QuantTables T;
+    wait_for_prior_grid();
     QuantConsts k;
     k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
     build_quant_tables<FMT>(T, k.g);
@@ -484,9 +485,8 @@ static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream)
         const size_t want = (n_chunks + kThreads - 1) / kThreads;
         const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
         const unsigned grid = (unsigned)(want < cap ? want : cap);
-        k_quantize<DT, B, FMT, DUAL, FAKE><<<grid, kThreads, S::RING_BYTES, stream>>>(m);
+        err = launch_pdl(k_quantize<DT, B, FMT, DUAL, FAKE>, grid, kThreads, S::RING_BYTES, stream, m);
         count_launch();
-        err = cudaGetLastError();
         if (err != cudaSuccess) return err;
     }
     const size_t done = n_chunks * S::NBC;
