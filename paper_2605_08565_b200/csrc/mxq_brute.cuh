@@ -237,8 +237,9 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, cons
     constexpr bool SKEW = (B >= 32);
     constexpr int BL = SKEW ? NP : B;
     constexpr int NBL = NP / BL;
-    const int cnt = T.cnt[list];
-    if (cnt == 0) return;
+    const int cnt_raw = T.cnt[list];
+    if (cnt_raw == 0) return;
+    [[maybe_unused]] const int cnt = cnt_raw;
     const int base = members_base<FMT>(list);
     const float4* cand = T.cand + base;
     uint32_t cbest[NBT];
@@ -248,7 +249,8 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, cons
 
     if constexpr (!SKEW) {
         // two members per trip: two independent SSE chains keep the FMA pipe fed
-        for (int m = 0; m < cnt; m += 2) {
+        const int pairs_end = cnt & ~1;
+        for (int m = 0; m < pairs_end; m += 2) {
             const float4 dpA = cand[m], dpB = cand[m + 1];
             const float2 nDA = make_float2(dpA.x, dpA.x), PA = make_float2(dpA.y, dpA.y);
             const float2 nDB = make_float2(dpB.x, dpB.x), PB = make_float2(dpB.y, dpB.y);
@@ -271,9 +273,29 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, cons
                 keep_smaller(cbest[NBL + k], cslot[NBL + k], __float_as_uint(sB[k].y), m + 1);
             }
         }
+        if (cnt & 1) {   // the odd member on its own
+            const int m = cnt - 1;
+            const float4 dpA = cand[m];
+            const float2 nDA = make_float2(dpA.x, dpA.x), PA = make_float2(dpA.y, dpA.y);
+            const uint32_t hA = __float_as_uint(dpA.z);
+            float2 sA[NBL];
+#pragma unroll
+            for (int k = 0; k < NBL; ++k) sA[k] = make_float2(0.0f, 0.0f);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const float2 eA = residual_pair<HALF>(tb[i], PA, v2[i], nDA, hA);
+                sA[i / BL] = __ffma2_rn(eA, eA, sA[i / BL]);
+            }
+#pragma unroll
+            for (int k = 0; k < NBL; ++k) {
+                keep_smaller(cbest[k], cslot[k], __float_as_uint(sA[k].x), m);
+                keep_smaller(cbest[NBL + k], cslot[NBL + k], __float_as_uint(sA[k].y), m);
+            }
+        }
     } else {
         // trip m: the low half evaluates members m and m + 1, the high half finishes members
         // m - 2 and m - 1 from the low-half sums of the previous trip
+        const int cnt = cnt_raw + (cnt_raw & 1);   // an odd list repeats its last member once (table build)
         float nDA_prev = cand[0].x, PA_prev = cand[0].y, nDB_prev = nDA_prev, PB_prev = PA_prev;
         uint32_t hA_prev = __float_as_uint(cand[0].z), hB_prev = hA_prev;
         float carryA = 0.0f, carryB = 0.0f;
