@@ -192,6 +192,14 @@ __device__ __forceinline__ float2 quotient_pair(float2 v, float2 nD, float2 R) {
     return q;
 }
 
+// The same with ONE correction: exact when the significand of Dref has at most 19 bits (see
+// quotient_short() of the one-pass kernels for the argument).
+__device__ __forceinline__ float2 quotient_pair_short(float2 v, float2 nD, float2 R) {
+    const float2 q = __fmul2_rn(v, R);
+    const float2 r = __ffma2_rn(q, nD, v);
+    return __ffma2_rn(r, R, q);
+}
+
 __device__ __forceinline__ unsigned long long sse_key(float s, int c) {
     return ((unsigned long long)__float_as_uint(s) << 32) | (unsigned long long)(unsigned)c;
 }
@@ -345,6 +353,9 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
     const int first = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     build_brute_tables<FMT>(T, g, first);
 
+    // all decode scales are short multiples of a class reference when g itself has few bits
+    const bool short_ref = (__float_as_uint(g) & 0x1FFu) == 0u;   // <= 15 bits of g, <= 19 bits of Dref
+
     const size_t stride = (size_t)gridDim.x * kThreads;
     for (size_t grp = (size_t)blockIdx.x * kThreads + threadIdx.x; grp < p.n_items; grp += stride) {
         float2 v2[NP];
@@ -375,7 +386,8 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
                 const float2 nDr2 = make_float2(-Dr, -Dr), Rr2 = make_float2(Rr, Rr);
                 float2 tb[NP];
 #pragma unroll
-                for (int i = 0; i < NP; ++i) tb[i] = quotient_pair(v2[i], nDr2, Rr2);
+                for (int i = 0; i < NP; ++i)
+                    tb[i] = short_ref ? quotient_pair_short(v2[i], nDr2, Rr2) : quotient_pair(v2[i], nDr2, Rr2);
                 search_list<B, FMT, false>(T, 2 * cls, v2, tb, best);
                 search_list<B, FMT, true>(T, 2 * cls + 1, v2, tb, best);
             }
