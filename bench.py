@@ -50,10 +50,10 @@ STREAM_ELEMS = 1 << 27            # tensor size of the streaming (HBM-bound) ker
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (same kernel build, same launch configuration); set an entry to None when its kernel changes.
 NCU_TRAFFIC_BYTES = {
-    "k_brute<bf16,B=16,UE4M3>@16Mi": 33.609984e6 + 7.68e3,
-    "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.478720e6 + 81.633280e6,
-    "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi": 268.494592e6 + 83.002624e6,
-    "k_quantize<f32,B=16,UE4M3,absmax>@128Mi": 536.896512e6 + 94.908672e6,
+    "k_brute<bf16,B=16,UE4M3>@16Mi": 33.620480e6 + 3.84e3,
+    "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.497920e6 + 81.853696e6,
+    "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi": 268.530432e6 + 83.161600e6,
+    "k_quantize<f32,B=16,UE4M3,absmax>@128Mi": 536.909824e6 + 95.663616e6,
 }
 
 
