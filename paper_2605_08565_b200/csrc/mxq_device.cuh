@@ -151,32 +151,6 @@ __device__ __forceinline__ void unpack_e2m1x8(uint32_t codes, float (&q)[8]) {
     }
 }
 
-// Eight quotients -> eight FP4 codes in one word AND the eight grid values they stand for, in one
-// step: the decoder reads the freshly converted bytes, so nothing is unpacked from the word.
-__device__ __forceinline__ uint32_t quantize_e2m1x8(const float* t, float (&q)[8]) {
-    uint32_t out, h0, h1, h2, h3;
-    asm("{\n"
-        " .reg .b8 b0, b1, b2, b3;\n"
-        " cvt.rn.satfinite.e2m1x2.f32 b0, %6, %5;\n"
-        " cvt.rn.satfinite.e2m1x2.f32 b1, %8, %7;\n"
-        " cvt.rn.satfinite.e2m1x2.f32 b2, %10, %9;\n"
-        " cvt.rn.satfinite.e2m1x2.f32 b3, %12, %11;\n"
-        " cvt.rn.f16x2.e2m1x2 %1, b0;\n"
-        " cvt.rn.f16x2.e2m1x2 %2, b1;\n"
-        " cvt.rn.f16x2.e2m1x2 %3, b2;\n"
-        " cvt.rn.f16x2.e2m1x2 %4, b3;\n"
-        " mov.b32 %0, {b0, b1, b2, b3};\n"
-        "}"
-        : "=r"(out), "=r"(h0), "=r"(h1), "=r"(h2), "=r"(h3)
-        : "f"(t[0]), "f"(t[1]), "f"(t[2]), "f"(t[3]), "f"(t[4]), "f"(t[5]), "f"(t[6]), "f"(t[7]));
-    float2 f;
-    f = __half22float2(*reinterpret_cast<__half2*>(&h0)); q[0] = f.x; q[1] = f.y;
-    f = __half22float2(*reinterpret_cast<__half2*>(&h1)); q[2] = f.x; q[3] = f.y;
-    f = __half22float2(*reinterpret_cast<__half2*>(&h2)); q[4] = f.x; q[5] = f.y;
-    f = __half22float2(*reinterpret_cast<__half2*>(&h3)); q[6] = f.x; q[7] = f.y;
-    return out;
-}
-
 // Two quotients -> the two grid values they round to, as floats (no code kept).
 __device__ __forceinline__ float2 round_e2m1x2(float t0, float t1) {
     uint32_t h;
