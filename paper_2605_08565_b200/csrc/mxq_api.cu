@@ -165,7 +165,7 @@ int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, in
     if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
     if (!valid_block(block_size) || n == 0 || n % (size_t)block_size != 0) return MXQ_ERR_BAD_SHAPE;
     if (!(global_scale > 0.0f && std::isfinite(global_scale))) return MXQ_ERR_BAD_SCALE;
-    if (!aligned16(d_codes) || !aligned16(d_out)) return MXQ_ERR_ALIGN;
+    if (!aligned16(d_codes) || !aligned16(d_out) || (reinterpret_cast<uintptr_t>(d_scales) & 3u)) return MXQ_ERR_ALIGN;
     cudaError_t err = launch_dequantize(d_codes, d_scales, n, block_size, scale_fmt, global_scale, d_out, out_dtype,
                                         static_cast<cudaStream_t>(cuda_stream));
     return err == cudaSuccess ? MXQ_OK : cuda_fail(err);

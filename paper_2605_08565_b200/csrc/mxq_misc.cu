@@ -157,42 +157,66 @@ __device__ __forceinline__ float decode_scale(int fmt, int c, float g) {
     return __fmul_rn(scale_value(fmt, c), g);
 }
 
+// A unit is the run of elements whose results one thread writes with ONE 16-byte store, so that a
+// warp's store covers 512 contiguous bytes: 8 elements for bf16 output, 4 for fp32 output.  Four
+// units per thread and trip keep four independent loads in flight.
 template <int ODT>
 __global__ void __launch_bounds__(kThreads) k_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n,
                                                          int log2B, int fmt, float g, void* out) {
     wait_for_prior_grid();
-    const size_t n8 = n >> 3;
+    constexpr int E = (ODT == kF32) ? 4 : 8;      // elements per unit
+    constexpr int LOG2E = (ODT == kF32) ? 2 : 3;
+    constexpr int U = 4;
+    const size_t n_units = n / E;
     const size_t stride = (size_t)gridDim.x * kThreads;
-    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n8; i += stride) {
-        const uint32_t w = __ldcs(reinterpret_cast<const uint32_t*>(codes) + i);
-        float q[8];
-        unpack_e2m1x8(w, q);
-        float xh[8];
-        if (log2B >= 3) {
-            const float D = decode_scale(fmt, scales[(i << 3) >> log2B], g);
+    for (size_t base = (size_t)blockIdx.x * kThreads + threadIdx.x; base < n_units; base += stride * U) {
+        uint32_t w[U], sc[U];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) xh[k] = __fmul_rn(q[k], D);
-        } else {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) xh[k] = __fmul_rn(q[k], decode_scale(fmt, scales[((i << 3) + k) >> log2B], g));
-        }
-        if constexpr (ODT == kF32) {
-            float4* o = static_cast<float4*>(out) + 2 * i;
-            __stcs(o, make_float4(xh[0], xh[1], xh[2], xh[3]));
-            __stcs(o + 1, make_float4(xh[4], xh[5], xh[6], xh[7]));
-        } else {
-            uint32_t h[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const __nv_bfloat162 b = __floats2bfloat162_rn(xh[2 * k], xh[2 * k + 1]);
-                h[k] = *reinterpret_cast<const uint32_t*>(&b);
+        for (int u = 0; u < U; ++u) {
+            const size_t i = base + (size_t)u * stride;
+            w[u] = 0;
+            sc[u] = 0;
+            if (i < n_units) {
+                if constexpr (E == 8) w[u] = __ldcs(reinterpret_cast<const uint32_t*>(codes) + i);
+                else w[u] = __ldcs(reinterpret_cast<const uint16_t*>(codes) + i);
+                // the scale codes of the unit's blocks (one byte when a block holds the whole unit)
+                if (log2B >= LOG2E) sc[u] = scales[(i << LOG2E) >> log2B];
+                else if (E >> log2B == 2) sc[u] = reinterpret_cast<const uint16_t*>(scales)[i];
+                else sc[u] = reinterpret_cast<const uint32_t*>(scales)[i];
             }
-            __stcs(static_cast<uint4*>(out) + i, make_uint4(h[0], h[1], h[2], h[3]));
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t i = base + (size_t)u * stride;
+            if (i >= n_units) continue;
+            float q[8];
+            unpack_e2m1x8(w[u], q);
+            float xh[E];
+            if (log2B >= LOG2E) {
+                const float D = decode_scale(fmt, (int)sc[u], g);
+#pragma unroll
+                for (int k = 0; k < E; ++k) xh[k] = __fmul_rn(q[k], D);
+            } else {
+#pragma unroll
+                for (int k = 0; k < E; ++k)
+                    xh[k] = __fmul_rn(q[k], decode_scale(fmt, (int)((sc[u] >> (8 * (k >> log2B))) & 0xFFu), g));
+            }
+            if constexpr (ODT == kF32) {
+                __stcs(static_cast<float4*>(out) + i, make_float4(xh[0], xh[1], xh[2], xh[3]));
+            } else {
+                uint32_t h[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const __nv_bfloat162 b = __floats2bfloat162_rn(xh[2 * k], xh[2 * k + 1]);
+                    h[k] = *reinterpret_cast<const uint32_t*>(&b);
+                }
+                __stcs(static_cast<uint4*>(out) + i, make_uint4(h[0], h[1], h[2], h[3]));
+            }
         }
     }
-    // ragged end (n not a multiple of 8; only possible for block sizes 2 and 4)
-    if (blockIdx.x == 0 && threadIdx.x < (unsigned)(n - (n8 << 3))) {
-        const size_t e = (n8 << 3) + threadIdx.x;
+    // ragged end (n not a multiple of the unit; only possible for block sizes 2 and 4)
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)(n - n_units * E)) {
+        const size_t e = n_units * E + threadIdx.x;
         const uint32_t c4 = (codes[e >> 1] >> ((e & 1) ? 4 : 0)) & 15u;
         float q[8];
         unpack_e2m1x8(c4, q);
@@ -209,7 +233,7 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_
     if (err != cudaSuccess) return err;
     int log2B = 0;
     while ((1 << log2B) < B) ++log2B;
-    size_t want = ((n >> 3) + kThreads - 1) / kThreads;
+    size_t want = ((n >> (out_dtype == kF32 ? 2 : 3)) / 4 + kThreads - 1) / kThreads;   // four units per thread
     if (want == 0) want = 1;
     const size_t cap = (size_t)sm_count(dev) * 8;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
