@@ -14,26 +14,26 @@ namespace mxq {
 // order), the other elements are skipped.  A zero decode scale clips nothing.  One thread per
 // block; IEEE division throughout.
 // ------------------------------------------------------------------------------------------------
-template <int DT>
-__global__ void __launch_bounds__(kThreads) k_block_clip_sse(const void* x, size_t n_blocks, int B, int fmt, float g,
+template <int DT, int B>
+__global__ void __launch_bounds__(kThreads) k_block_clip_sse(const void* x, size_t n_blocks, int fmt, float g,
                                                              const float* d_g, const uint8_t* scales, float* out) {
+    wait_for_prior_grid();
     const float gs = d_g ? *d_g : g;
     const size_t stride = (size_t)gridDim.x * kThreads;
     for (size_t b = (size_t)blockIdx.x * kThreads + threadIdx.x; b < n_blocks; b += stride) {
+        float v[B];
+        load_elems<DT, B>(x, b * B, v);      // vector loads: a block is 4 .. 256 contiguous bytes
         const int c = scales[b];
         float s = 0.0f;
         if (c < num_codes(fmt)) {
             const float D = __fmul_rn(scale_value(fmt, c), gs);
             if (D != 0.0f) {
+#pragma unroll
                 for (int i = 0; i < B; ++i) {
-                    const size_t e_idx = b * (size_t)B + (size_t)i;
-                    float v;
-                    if constexpr (DT == kF32) v = static_cast<const float*>(x)[e_idx];
-                    else v = __uint_as_float((uint32_t) static_cast<const uint16_t*>(x)[e_idx] << 16);
-                    const float t = __fdiv_rn(v, D);
+                    const float t = __fdiv_rn(v[i], D);
                     if (fabsf(t) > 6.0f) {
-                        const float q = copysignf(6.0f, v);
-                        const float e = __fmaf_rn(-q, D, v);
+                        const float q = copysignf(6.0f, v[i]);
+                        const float e = __fmaf_rn(-q, D, v[i]);
                         s = __fmaf_rn(e, e, s);
                     }
                 }
@@ -42,6 +42,19 @@ __global__ void __launch_bounds__(kThreads) k_block_clip_sse(const void* x, size
             s = __uint_as_float(0x7FC00000u);   // not a code of the format
         }
         out[b] = s;
+    }
+}
+
+template <int DT>
+static cudaError_t launch_clip_dt(const void* x, size_t n_blocks, int B, int fmt, float g, const float* d_g,
+                                  const uint8_t* scales, float* out, unsigned grid, cudaStream_t s) {
+    switch (B) {
+    case 2: return launch_pdl(k_block_clip_sse<DT, 2>, grid, kThreads, 0, s, x, n_blocks, fmt, g, d_g, scales, out);
+    case 4: return launch_pdl(k_block_clip_sse<DT, 4>, grid, kThreads, 0, s, x, n_blocks, fmt, g, d_g, scales, out);
+    case 8: return launch_pdl(k_block_clip_sse<DT, 8>, grid, kThreads, 0, s, x, n_blocks, fmt, g, d_g, scales, out);
+    case 16: return launch_pdl(k_block_clip_sse<DT, 16>, grid, kThreads, 0, s, x, n_blocks, fmt, g, d_g, scales, out);
+    case 32: return launch_pdl(k_block_clip_sse<DT, 32>, grid, kThreads, 0, s, x, n_blocks, fmt, g, d_g, scales, out);
+    default: return launch_pdl(k_block_clip_sse<DT, 64>, grid, kThreads, 0, s, x, n_blocks, fmt, g, d_g, scales, out);
     }
 }
 
@@ -54,10 +67,10 @@ cudaError_t launch_block_clip_sse(const void* x, int dtype, size_t n, int B, int
     size_t want = (n_blocks + kThreads - 1) / kThreads;
     const size_t cap = (size_t)sm_count(dev) * 8;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
-    if (dtype == kF32) k_block_clip_sse<kF32><<<grid, kThreads, 0, s>>>(x, n_blocks, B, fmt, g, d_g, scales, out);
-    else k_block_clip_sse<kBF16><<<grid, kThreads, 0, s>>>(x, n_blocks, B, fmt, g, d_g, scales, out);
+    err = (dtype == kF32) ? launch_clip_dt<kF32>(x, n_blocks, B, fmt, g, d_g, scales, out, grid, s)
+                          : launch_clip_dt<kBF16>(x, n_blocks, B, fmt, g, d_g, scales, out, grid, s);
     count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 // ------------------------------------------------------------------------------------------------
