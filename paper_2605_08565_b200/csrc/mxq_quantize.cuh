@@ -391,6 +391,22 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     extern __shared__ uint4 ring[];
     __shared__ QuantTables T;
     wait_for_prior_grid();
+    // request the first chunks before anything else: their latency hides behind the table build
+    const size_t stride = (size_t)gridDim.x * kThreads;
+    size_t chunk = (size_t)blockIdx.x * kThreads + threadIdx.x;
+    constexpr size_t kChunkBytes = (size_t)S::C * S::EB;
+    constexpr uint32_t kSlotBytes = S::PIECES * kThreads * 16;
+    constexpr int DIST = S::SLOTS - 1;   // chunks requested ahead of the one being processed
+    const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(ring) + threadIdx.x * 16;
+    const char* x = static_cast<const char*>(p.x);
+    {
+        size_t c = chunk;
+#pragma unroll
+        for (int d = 0; d < DIST; ++d) {
+            stage_chunk<S::PIECES>(ring_base + d * kSlotBytes, x + c * kChunkBytes, c < p.n_items);
+            c += stride;
+        }
+    }
     QuantConsts k;
     k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
     build_quant_tables<FMT>(T, k.g);
@@ -417,22 +433,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
         k.m_lo = 0.0f;
     }
 
-    const size_t stride = (size_t)gridDim.x * kThreads;
-    size_t chunk = (size_t)blockIdx.x * kThreads + threadIdx.x;
     if (chunk >= p.n_items) return;   // no barrier follows
-    constexpr size_t kChunkBytes = (size_t)S::C * S::EB;
-    constexpr uint32_t kSlotBytes = S::PIECES * kThreads * 16;
-    constexpr int DIST = S::SLOTS - 1;   // chunks requested ahead of the one being processed
-    const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(ring) + threadIdx.x * 16;
-    const char* x = static_cast<const char*>(p.x);
-    {   // prologue: request the first DIST chunks
-        size_t c = chunk;
-#pragma unroll
-        for (int d = 0; d < DIST; ++d) {
-            stage_chunk<S::PIECES>(ring_base + d * kSlotBytes, x + c * kChunkBytes, c < p.n_items);
-            c += stride;
-        }
-    }
     int slot = 0;                      // slot holding `chunk`
     int fill = DIST % S::SLOTS;        // slot that the next request goes to
     size_t ahead = chunk + (size_t)DIST * stride;
