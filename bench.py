@@ -295,6 +295,38 @@ def streaming_rooflines(torch, mxq, device, peaks):
     return out
 
 
+def pruned_sweep_report(torch, mxq, wl):
+    """The brute-force passes of the step once more with the pruned sweep switched on (outside the
+    timed region; `value` and `roofline` are always the full sweep): per block size the time of both
+    sweeps over the rotating tensors, launches back to back, and whether the outputs are identical."""
+    out = {}
+    x0 = wl.x[0]
+    n = x0.numel()
+    try:
+        for B in BLOCKS:
+            bufs = {}
+            ms = {}
+            for mode in (0, 1):
+                mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, mode)
+                codes, scales, sse = mxq.alloc_outputs(n, B, x0.device)
+                fn = lambda x: mxq.mxq_quantize_ex(x, n, B, UE4M3, BRUTE, 1.0, None, codes, scales, sse)
+                fn(x0)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for x in wl.x:
+                    fn(x)
+                e1.record()
+                fn(x0)
+                torch.cuda.synchronize()
+                ms[mode] = e0.elapsed_time(e1) / len(wl.x)
+                bufs[mode] = (codes, scales, sse)
+            same = all(torch.equal(a.view(torch.uint8), b.view(torch.uint8)) for a, b in zip(bufs[0], bufs[1]))
+            out[f"B{B}"] = {"full_ms": ms[0], "pruned_ms": ms[1], "speedup": ms[0] / ms[1], "outputs_identical": bool(same)}
+    finally:
+        mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 0)
+    return out
+
+
 def run_gpu(args) -> None:
     import torch
     from paper_2605_08565_b200 import binding as mxq
@@ -406,6 +438,7 @@ def run_gpu(args) -> None:
                      "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0, "traffic": None,
                      "ms_per_launch": ms, "gelem_s": N_ELEM / (ms * 1e-3) / 1e9, "peak_source": peaks["source"]}
     streaming = None if args.skip_streaming else streaming_rooflines(torch, mxq, device, peaks)
+    pruned = pruned_sweep_report(torch, mxq, wl)
     per_recipe = {"brute_B16": N_ELEM / (brute_ms * 1e-3) / 1e9, "absmax_B16": hbm["absmax_B16"]["gelem_s"],
                   "4o6_B16": hbm["4o6_B16"]["gelem_s"]}
 
@@ -430,7 +463,7 @@ def run_gpu(args) -> None:
                    "elements_per_step": wl.elems_per_step, "passes_per_step": len(wl.passes) + 1,
                    "l2": f"inputs rotate over {N_ROTATE} tensors (256 MiB) > 126 MB L2"},
         "roofline": roofline, "roofline_hbm": hbm, "roofline_hbm_streaming": streaming,
-        "per_recipe_gelem_s": per_recipe,
+        "per_recipe_gelem_s": per_recipe, "brute_pruned_sweep": pruned,
         "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(host_in.numel() * 2),
                 "d2h_bytes_per_step": int(host_out.numel() * 8)},

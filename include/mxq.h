@@ -227,6 +227,22 @@ int mxq_segment_mse(const float* d_block_sse, size_t n_blocks, size_t blocks_per
  */
 int mxq_mask_interval(const void* x, int dtype, size_t n, float lo, float hi, void* d_out, void* cuda_stream);
 
+/* Process-wide options, read by the entry points when they are called.
+ *
+ * MXQ_OPT_BRUTE_PRUNE (default 0).  With 0 the brute-force recipes evaluate every finite scale code
+ * on every block, exactly as the search is stated (Experimental Setup).  With 1 they leave out, per
+ * warp of the kernel, the codes whose decode scale is at least four times the largest magnitude the
+ * warp holds: every element then quantizes to zero (|v|/D <= 1/4 rounds to the grid value 0), so all
+ * those codes have the SSE of the all-zero quantization, which is entered once with the smallest of
+ * them.  The outputs are bit-identical to the full sweep; only the time differs, by an amount that
+ * depends on the data.  The paper states no such shortcut.
+ *
+ * mxq_set_option: MXQ_ERR_BAD_ENUM for an unknown option or a value outside {0, 1}.
+ * mxq_get_option: MXQ_ERR_NULL for a NULL out_value (host pointer). */
+enum { MXQ_OPT_BRUTE_PRUNE = 1 };
+int mxq_set_option(int option, int value);
+int mxq_get_option(int option, int* out_value);
+
 /* Number of kernels the library has launched in this process (all entry points), for
  * accounting in benchmarks. */
 unsigned long long mxq_launch_count(void);

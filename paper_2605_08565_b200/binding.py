@@ -17,10 +17,11 @@ LIB_PATH = os.path.join(_HERE, "libmxq.so")
 MXQ_F32, MXQ_BF16 = 0, 1
 MXQ_SF_UE8M0, MXQ_SF_UE4M3, MXQ_SF_UE5M3 = 0, 1, 2
 MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ, MXQ_ABSMAX_OCP = range(7)
+MXQ_OPT_BRUTE_PRUNE = 1
 
 EXPORTS = (
     "mxq_quantize", "mxq_quantize_ex", "mxq_fake_quantize", "mxq_tensor_amax", "mxq_global_scale_from_amax",
-    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_mask_interval", "mxq_launch_count",
+    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_mask_interval", "mxq_set_option", "mxq_get_option", "mxq_launch_count",
     "mxq_status_string", "mxq_last_cuda_error", "mxq_version",
 )
 
@@ -69,6 +70,10 @@ def load_library() -> ctypes.CDLL:
     L.mxq_segment_mse.argtypes = [vp, sz, sz, sz, vp, vp]
     L.mxq_mask_interval.restype = i32
     L.mxq_mask_interval.argtypes = [vp, i32, sz, f32, f32, vp, vp]
+    L.mxq_set_option.restype = i32
+    L.mxq_set_option.argtypes = [i32, i32]
+    L.mxq_get_option.restype = i32
+    L.mxq_get_option.argtypes = [i32, c.POINTER(c.c_int)]
     L.mxq_launch_count.restype = c.c_ulonglong
     L.mxq_launch_count.argtypes = []
     L.mxq_status_string.restype = c.c_char_p
@@ -188,6 +193,16 @@ def mxq_segment_mse(d_block_sse, n_blocks, blocks_per_segment, elems_per_segment
 
 def mxq_mask_interval(x, n, lo, hi, d_out, stream=None) -> None:
     _check(load_library().mxq_mask_interval(_ptr(x), _dtype_id(x), n, lo, hi, _ptr(d_out), _stream(stream, x)))
+
+
+def mxq_set_option(option: int, value: int) -> None:
+    _check(load_library().mxq_set_option(int(option), int(value)))
+
+
+def mxq_get_option(option: int) -> int:
+    out = ctypes.c_int(0)
+    _check(load_library().mxq_get_option(int(option), ctypes.byref(out)))
+    return int(out.value)
 
 
 def mxq_launch_count() -> int:

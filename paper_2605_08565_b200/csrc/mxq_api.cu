@@ -9,6 +9,7 @@
 namespace mxq {
 
 static std::atomic<unsigned long long> g_launches{0};
+static std::atomic<int> g_brute_prune{0};
 static thread_local int tl_cuda_error = 0;
 
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
@@ -75,8 +76,12 @@ static int quantize_common(const void* x, int dtype, size_t n, int block_size, i
     cudaError_t err;
     if (brute) {
         a.n_items = n / (size_t)block_size;
-        err = (dtype == MXQ_F32) ? launch_brute_f32(a, block_size, scale_fmt, s)
-                                 : launch_brute_bf16(a, block_size, scale_fmt, s);
+        if (g_brute_prune.load(std::memory_order_relaxed))
+            err = (dtype == MXQ_F32) ? launch_brute_pruned_f32(a, block_size, scale_fmt, s)
+                                     : launch_brute_pruned_bf16(a, block_size, scale_fmt, s);
+        else
+            err = (dtype == MXQ_F32) ? launch_brute_f32(a, block_size, scale_fmt, s)
+                                     : launch_brute_bf16(a, block_size, scale_fmt, s);
         return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
     }
     const bool dual = (recipe == MXQ_4O6 || recipe == MXQ_4O6_PZ);
@@ -217,6 +222,19 @@ int mxq_mask_interval(const void* x, int dtype, size_t n, float lo, float hi, vo
     if (!aligned16(x) || !aligned16(d_out)) return MXQ_ERR_ALIGN;
     cudaError_t err = launch_mask_interval(x, dtype, n, lo, hi, d_out, static_cast<cudaStream_t>(cuda_stream));
     return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+int mxq_set_option(int option, int value) {
+    if (option != MXQ_OPT_BRUTE_PRUNE || (value != 0 && value != 1)) return MXQ_ERR_BAD_ENUM;
+    g_brute_prune.store(value, std::memory_order_relaxed);
+    return MXQ_OK;
+}
+
+int mxq_get_option(int option, int* out_value) {
+    if (!out_value) return MXQ_ERR_NULL;
+    if (option != MXQ_OPT_BRUTE_PRUNE) return MXQ_ERR_BAD_ENUM;
+    *out_value = g_brute_prune.load(std::memory_order_relaxed);
+    return MXQ_OK;
 }
 
 unsigned long long mxq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

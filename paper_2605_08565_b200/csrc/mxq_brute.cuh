@@ -239,13 +239,28 @@ __device__ __forceinline__ void keep_smaller(uint32_t& best_bits, int& best_slot
 
 // All members of one list (one mantissa class, one residual kind) against the thread's elements;
 // the list winner of every block is folded into best[].
+// Number of leading members of a list that have to be evaluated when no magnitude the warp holds
+// exceeds limit / 4.  A member with D >= limit quantizes every such element to zero
+// (|v| / D <= 1/4, and the tie at 1/4 goes to the even index 0), so its SSE is the sum of squares
+// of the block for every such member alike; members are in ascending order of D, so these form a
+// suffix of the list.  The smallest code left out is folded into skipped_min.
+template <int FMT>
+__device__ __forceinline__ int admitted_members(const BruteTables& T, int list, float limit, int& skipped_min) {
+    const int cnt = T.cnt[list];
+    const int base = members_base<FMT>(list);
+    int n = cnt;
+    while (n > 0 && -T.cand[base + n - 1].x >= limit) --n;
+    if (n < cnt) skipped_min = min(skipped_min, (int)T.member[base + n]);
+    return n;
+}
+
+// cnt_raw: the first cnt_raw members of the list are evaluated.
 template <int B, int FMT, bool HALF, int NP, int NBT>
-__device__ __forceinline__ void search_list(const BruteTables& T, int list, const float2 (&v2)[NP],
+__device__ __forceinline__ void search_list(const BruteTables& T, int list, int cnt_raw, const float2 (&v2)[NP],
                                             const float2 (&tb)[NP], unsigned long long (&best)[NBT]) {
     constexpr bool SKEW = (B >= 32);
     constexpr int BL = SKEW ? NP : B;
     constexpr int NBL = NP / BL;
-    const int cnt_raw = T.cnt[list];
     if (cnt_raw == 0) return;
     [[maybe_unused]] const int cnt = cnt_raw;
     const int base = members_base<FMT>(list);
@@ -303,7 +318,9 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, cons
     } else {
         // trip m: the low half evaluates members m and m + 1, the high half finishes members
         // m - 2 and m - 1 from the low-half sums of the previous trip
-        const int cnt = cnt_raw + (cnt_raw & 1);   // an odd list repeats its last member once (table build)
+        // an odd count takes one more slot: the next member of the list, or the copy of the last
+        // member that the table build appends
+        const int cnt = cnt_raw + (cnt_raw & 1);
         float nDA_prev = cand[0].x, PA_prev = cand[0].y, nDB_prev = nDA_prev, PB_prev = PA_prev;
         uint32_t hA_prev = __float_as_uint(cand[0].z), hB_prev = hA_prev;
         float carryA = 0.0f, carryB = 0.0f;
@@ -336,8 +353,16 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, cons
         if (cbest[k] != 0xFFFFFFFFu) merge_class_winner(best[k], cbest[k], T.member[base + cslot[k]]);
 }
 
-template <int DT, int B, int FMT>
-__global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
+// PRUNE: the sweep leaves out, per warp, the candidates that provably tie with the all-zero
+// quantization (see admitted_members()); the outputs are the same.
+//
+// Resident CTAs per SM asked of the register allocator: two where measurement showed that the
+// second CTA outweighs the few spills it costs (B = 4; B = 2 and B = 32 with the pruned sweep),
+// else no constraint beyond one CTA.
+constexpr int brute_min_ctas(int B, bool prune) { return (B == 4 || ((B == 2 || B == 32) && prune)) ? 2 : 1; }
+
+template <int DT, int B, int FMT, bool PRUNE>
+__global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(QuantArgs p) {
     constexpr bool SKEW = (B >= 32);          // the pair's halves are the two halves of one block
     constexpr int G = SKEW ? B : 32;          // elements per thread
     constexpr int NP = G / 2;                 // pairs per thread
@@ -356,8 +381,13 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
     // all decode scales are short multiples of a class reference when g itself has few bits
     const bool short_ref = (__float_as_uint(g) & 0x1FFu) == 0u;   // <= 15 bits of g, <= 19 bits of Dref
 
+    // With PRUNE the loop is uniform per warp (lanes past the end repeat the warp's first group
+    // and store nothing), so that the warp can agree on the candidates it leaves out.
     const size_t stride = (size_t)gridDim.x * kThreads;
-    for (size_t grp = (size_t)blockIdx.x * kThreads + threadIdx.x; grp < p.n_items; grp += stride) {
+    const int lane = PRUNE ? (threadIdx.x & 31) : 0;
+    for (size_t wbase = (size_t)blockIdx.x * kThreads + threadIdx.x - lane; wbase < p.n_items; wbase += stride) {
+        const bool active = wbase + lane < p.n_items;
+        const size_t grp = active ? wbase + lane : wbase;
         float2 v2[NP];
         float amax = 0.0f;
         bool tiny = false;   // a nonzero magnitude below 2^-62: its quotient by Dref may be inexact
@@ -379,19 +409,61 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
 #pragma unroll
         for (int k = 0; k < NBT; ++k) best[k] = sse_key(__uint_as_float(0xFFFFFFFFu), first);
 
+        // Pruned sweep: candidates whose decode scale is at least four times the largest magnitude
+        // in the warp are not evaluated one by one; they all have the SSE of the all-zero
+        // quantization, which is entered once with the smallest such code.  4 * max is exact, or
+        // +inf when it overflows (nothing is left out then).
+        [[maybe_unused]] float limit = 0.0f;
+        if constexpr (PRUNE)
+            limit = __fmul_rn(4.0f, __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax))));
+        int skipped_min = 256;
+
         if (fast_ok) {
             for (int cls = 0; cls < NCLS; ++cls) {
-                if (T.cnt[2 * cls] + T.cnt[2 * cls + 1] == 0) continue;
+                int n0, n1;
+                if constexpr (PRUNE) {
+                    n0 = admitted_members<FMT>(T, 2 * cls, limit, skipped_min);
+                    n1 = admitted_members<FMT>(T, 2 * cls + 1, limit, skipped_min);
+                } else {
+                    n0 = T.cnt[2 * cls];
+                    n1 = T.cnt[2 * cls + 1];
+                }
+                if (n0 + n1 == 0) continue;
                 const float Dr = T.clsD[cls], Rr = T.clsR[cls];
                 const float2 nDr2 = make_float2(-Dr, -Dr), Rr2 = make_float2(Rr, Rr);
                 float2 tb[NP];
 #pragma unroll
                 for (int i = 0; i < NP; ++i)
                     tb[i] = short_ref ? quotient_pair_short(v2[i], nDr2, Rr2) : quotient_pair(v2[i], nDr2, Rr2);
-                search_list<B, FMT, false>(T, 2 * cls, v2, tb, best);
-                search_list<B, FMT, true>(T, 2 * cls + 1, v2, tb, best);
+                search_list<B, FMT, false>(T, 2 * cls, n0, v2, tb, best);
+                search_list<B, FMT, true>(T, 2 * cls + 1, n1, v2, tb, best);
             }
-            search_list<B, FMT, false>(T, kFlatList, v2, v2, best);   // Dref = 1: the elements are their own quotients
+            // Dref = 1: the elements are their own quotients
+            search_list<B, FMT, false>(T, kFlatList, T.cnt[kFlatList], v2, v2, best);
+            if (PRUNE && skipped_min < 256) {
+                // all-zero quantization: e = v, summed in element order like every other candidate
+                if constexpr (!SKEW) {
+                    float2 s0[NBL];
+#pragma unroll
+                    for (int k = 0; k < NBL; ++k) s0[k] = make_float2(0.0f, 0.0f);
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) s0[i / BL] = __ffma2_rn(v2[i], v2[i], s0[i / BL]);
+#pragma unroll
+                    for (int k = 0; k < NBL; ++k) {
+                        const unsigned long long k0 = sse_key(s0[k].x, skipped_min), k1 = sse_key(s0[k].y, skipped_min);
+                        if (k0 < best[k]) best[k] = k0;
+                        if (k1 < best[NBL + k]) best[NBL + k] = k1;
+                    }
+                } else {
+                    float s0 = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) s0 = __fmaf_rn(v2[i].x, v2[i].x, s0);
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) s0 = __fmaf_rn(v2[i].y, v2[i].y, s0);
+                    const unsigned long long k0 = sse_key(s0, skipped_min);
+                    if (k0 < best[0]) best[0] = k0;
+                }
+            }
         }
 
         // general path (IEEE division), candidate by candidate: threads that hold a magnitude above
@@ -459,9 +531,11 @@ __global__ void __launch_bounds__(kThreads) k_brute(QuantArgs p) {
                 packed[h * (NP / 8) + k] = pack_e2m1x8(t[8 * k], t[8 * k + 1], t[8 * k + 2], t[8 * k + 3], t[8 * k + 4],
                                                        t[8 * k + 5], t[8 * k + 6], t[8 * k + 7]);
         }
-        store_bytes<G / 2>(p.codes + grp * (G / 2), packed);
-        store_bytes<NBT>(p.scales + grp * NBT, sc);
-        if (p.block_sse) store_bytes<4 * NBT>(p.block_sse + grp * NBT, sw);
+        if (!PRUNE || active) {
+            store_bytes<G / 2>(p.codes + grp * (G / 2), packed);
+            store_bytes<NBT>(p.scales + grp * NBT, sc);
+            if (p.block_sse) store_bytes<4 * NBT>(p.block_sse + grp * NBT, sw);
+        }
     }
 }
 
@@ -507,7 +581,7 @@ __global__ void k_brute_tail(QuantArgs p) {
     if (p.block_sse) p.block_sse[blk] = __uint_as_float((uint32_t)(best >> 32));
 }
 
-template <int DT, int B, int FMT>
+template <int DT, int B, int FMT, bool PRUNE>
 static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
     static int ctas_per_sm[kMaxDevices] = {0};
     int dev = 0;
@@ -516,7 +590,7 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     if (ctas_per_sm[dev] == 0) {
         int n = 0;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_brute<DT, B, FMT>, kThreads, 0);
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_brute<DT, B, FMT, PRUNE>, kThreads, 0);
         if (err != cudaSuccess) return err;
         ctas_per_sm[dev] = n > 0 ? n : 1;
     }
@@ -529,7 +603,7 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
         const size_t want = (n_groups + kThreads - 1) / kThreads;
         const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
         const unsigned grid = (unsigned)(want < cap ? want : cap);
-        err = launch_pdl(k_brute<DT, B, FMT>, grid, kThreads, 0, stream, m);
+        err = launch_pdl(k_brute<DT, B, FMT, PRUNE>, grid, kThreads, 0, stream, m);
         count_launch();
         if (err != cudaSuccess) return err;
     }
@@ -547,24 +621,24 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
     return err;
 }
 
-template <int DT, int B>
+template <int DT, int B, bool PRUNE>
 static cudaError_t launch_brute_fmt(const QuantArgs& a, int fmt, cudaStream_t s) {
     switch (fmt) {
-    case kUE8M0: return launch_brute_inst<DT, B, kUE8M0>(a, s);
-    case kUE4M3: return launch_brute_inst<DT, B, kUE4M3>(a, s);
-    default: return launch_brute_inst<DT, B, kUE5M3>(a, s);
+    case kUE8M0: return launch_brute_inst<DT, B, kUE8M0, PRUNE>(a, s);
+    case kUE4M3: return launch_brute_inst<DT, B, kUE4M3, PRUNE>(a, s);
+    default: return launch_brute_inst<DT, B, kUE5M3, PRUNE>(a, s);
     }
 }
 
-template <int DT>
+template <int DT, bool PRUNE>
 static cudaError_t launch_brute_dt(const QuantArgs& a, int B, int fmt, cudaStream_t s) {
     switch (B) {
-    case 2: return launch_brute_fmt<DT, 2>(a, fmt, s);
-    case 4: return launch_brute_fmt<DT, 4>(a, fmt, s);
-    case 8: return launch_brute_fmt<DT, 8>(a, fmt, s);
-    case 16: return launch_brute_fmt<DT, 16>(a, fmt, s);
-    case 32: return launch_brute_fmt<DT, 32>(a, fmt, s);
-    default: return launch_brute_fmt<DT, 64>(a, fmt, s);
+    case 2: return launch_brute_fmt<DT, 2, PRUNE>(a, fmt, s);
+    case 4: return launch_brute_fmt<DT, 4, PRUNE>(a, fmt, s);
+    case 8: return launch_brute_fmt<DT, 8, PRUNE>(a, fmt, s);
+    case 16: return launch_brute_fmt<DT, 16, PRUNE>(a, fmt, s);
+    case 32: return launch_brute_fmt<DT, 32, PRUNE>(a, fmt, s);
+    default: return launch_brute_fmt<DT, 64, PRUNE>(a, fmt, s);
     }
 }
 

@@ -3,6 +3,6 @@
 
 namespace mxq {
 cudaError_t launch_brute_bf16(const QuantArgs& a, int B, int fmt, cudaStream_t s) {
-    return launch_brute_dt<kBF16>(a, B, fmt, s);
+    return launch_brute_dt<kBF16, false>(a, B, fmt, s);
 }
 }  // namespace mxq

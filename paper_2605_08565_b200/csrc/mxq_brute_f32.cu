@@ -3,6 +3,6 @@
 
 namespace mxq {
 cudaError_t launch_brute_f32(const QuantArgs& a, int B, int fmt, cudaStream_t s) {
-    return launch_brute_dt<kF32>(a, B, fmt, s);
+    return launch_brute_dt<kF32, false>(a, B, fmt, s);
 }
 }  // namespace mxq

@@ -55,6 +55,8 @@ cudaError_t launch_fake_quantize_f32(const QuantArgs& a, int B, int fmt, bool du
 cudaError_t launch_fake_quantize_bf16(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
 cudaError_t launch_brute_f32(const QuantArgs& a, int B, int fmt, cudaStream_t s);
 cudaError_t launch_brute_bf16(const QuantArgs& a, int B, int fmt, cudaStream_t s);
+cudaError_t launch_brute_pruned_f32(const QuantArgs& a, int B, int fmt, cudaStream_t s);
+cudaError_t launch_brute_pruned_bf16(const QuantArgs& a, int B, int fmt, cudaStream_t s);
 // Scalar kernel for the few blocks that do not fill a whole chunk (abs-max and 4-over-6 only).
 cudaError_t launch_quantize_tail(const QuantArgs& a, int dtype, int B, int fmt, bool dual, cudaStream_t s);
 

@@ -59,18 +59,60 @@ def test_one_pass_recipes_bit_exact(dtype, B, fmt):
         check_parity(x, B, fmt, recipe, 0.0131)
 
 
+@pytest.fixture(params=[0, 1], ids=["full_sweep", "pruned_sweep"])
+def sweep_mode(request):
+    """Both ways of running the brute-force kernels: every code evaluated, and the codes that provably
+    tie with the all-zero quantization left out.  The outputs must not depend on it."""
+    mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, request.param)
+    assert mxq.mxq_get_option(mxq.MXQ_OPT_BRUTE_PRUNE) == request.param
+    yield request.param
+    mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 0)
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("B", BLOCKS)
 @pytest.mark.parametrize("fmt", FMTS)
-def test_brute_force_bit_exact(dtype, B, fmt):
+def test_brute_force_bit_exact(dtype, B, fmt, sweep_mode):
     n = 2 * 256 * B + 7 * B
     x = _mixed(n, 40 + B + fmt, dtype)
     check_parity(x, B, fmt, mxq.MXQ_BRUTE, 1.0)
     check_parity(x, B, fmt, mxq.MXQ_BRUTE_PZ, 0.0131)
 
 
+@pytest.mark.parametrize("B", BLOCKS)
+@pytest.mark.parametrize("fmt", FMTS)
+def test_brute_force_on_small_magnitudes_and_quarter_scale_ties(B, fmt, sweep_mode):
+    """Inputs on which most codes quantize a whole warp's elements to zero: weight-like small values,
+    all-zero stretches as long as a warp's share, and magnitudes that are exactly a quarter of a
+    decode scale (the tie that still rounds to zero)."""
+    n = 3 * 256 * max(B, 32) + 11 * B
+    gen = torch.Generator().manual_seed(900 + B + fmt)
+    x = inputs.student_t(n, 5, 0.02, 70 + B, torch.float32)
+    span = 32 * max(B, 32)                                   # elements one warp holds per trip
+    x[span:2 * span] = 0.0
+    x[4 * span:5 * span] *= 2.0 ** -20
+    quarter = torch.exp2(torch.randint(-12, 3, (span,), generator=gen).float()) * (1.0 + torch.randint(0, 8, (span,), generator=gen).float() / 8)
+    sign = torch.where(torch.rand(span, generator=gen) < 0.5, -1.0, 1.0)
+    x[6 * span:7 * span] = 0.25 * quarter * sign
+    for dtype in (torch.float32, torch.bfloat16):
+        xd = x.to(dtype).contiguous()
+        check_parity(xd, B, fmt, mxq.MXQ_BRUTE, 1.0)
+        check_parity(xd, B, fmt, mxq.MXQ_BRUTE_PZ, 1.0)
+        check_parity(xd, B, fmt, mxq.MXQ_BRUTE, 3.7e-3)
+
+
+def test_option_calls_reject_bad_arguments():
+    with pytest.raises(mxq.MxqError):
+        mxq.mxq_set_option(99, 1)
+    with pytest.raises(mxq.MxqError):
+        mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 2)
+    with pytest.raises(mxq.MxqError):
+        mxq.mxq_get_option(99)
+    assert mxq.mxq_get_option(mxq.MXQ_OPT_BRUTE_PRUNE) == 0
+
+
 @pytest.mark.parametrize("recipe", RECIPES)
-def test_extreme_global_scales(recipe):
+def test_extreme_global_scales(recipe, sweep_mode):
     x = _mixed(4096, 77, torch.float32)
     for g in (2.0 ** -30, 2.0 ** 20, 3.0e-37, 1.0e30):
         check_parity(x, 16, mxq.MXQ_SF_UE4M3, recipe, g)
@@ -148,7 +190,7 @@ def test_config_activation_outlier_columns_bf16():
 
 
 @pytest.mark.parametrize("fmt", FMTS)
-def test_config_laplace_fp32_brute_force_with_tensor_scale(fmt):
+def test_config_laplace_fp32_brute_force_with_tensor_scale(fmt, sweep_mode):
     x = inputs.laplace(96 * 1024, 5, torch.float32)
     g = float(orc.global_scale_from_amax(orc.tensor_amax(x.numpy())))
     for B in (2, 4, 8, 16, 32):
