@@ -230,12 +230,19 @@ int mxq_mask_interval(const void* x, int dtype, size_t n, float lo, float hi, vo
 /* Process-wide options, read by the entry points when they are called.
  *
  * MXQ_OPT_BRUTE_PRUNE (default 0).  With 0 the brute-force recipes evaluate every finite scale code
- * on every block, exactly as the search is stated (Experimental Setup).  With 1 they leave out, per
- * warp of the kernel, the codes whose decode scale is at least four times the largest magnitude the
- * warp holds: every element then quantizes to zero (|v|/D <= 1/4 rounds to the grid value 0), so all
- * those codes have the SSE of the all-zero quantization, which is entered once with the smallest of
- * them.  The outputs are bit-identical to the full sweep; only the time differs, by an amount that
- * depends on the data.  The paper states no such shortcut.
+ * on every block, exactly as the search is stated (Experimental Setup).  With 1 a warp of the kernel
+ * leaves out the codes that provably cannot change an output of any block it holds:
+ *   - decode scales of at least four times the largest magnitude: every element quantizes to zero
+ *     (|v|/D <= 1/4 rounds to the grid value 0), so all of them have the SSE of the all-zero
+ *     quantization, which is entered once with the smallest such code;
+ *   - decode scales so large that the elements they send to zero alone already cost more than the
+ *     best SSE found so far, in every block;
+ *   - decode scales so small that the saturation error of the largest element alone already exceeds
+ *     the best SSE found so far, in every block.
+ * The bounds are evaluated in the kernel's own binary32 arithmetic and compared strictly, so the
+ * outputs (codes, scale bytes, block SSE; ties to the smaller code) are bit-identical to the full
+ * sweep; only the time differs, by an amount that depends on the data.  The paper states no such
+ * shortcut.
  *
  * mxq_set_option: MXQ_ERR_BAD_ENUM for an unknown option or a value outside {0, 1}.
  * mxq_get_option: MXQ_ERR_NULL for a NULL out_value (host pointer). */

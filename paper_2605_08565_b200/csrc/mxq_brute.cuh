@@ -68,6 +68,9 @@ struct BruteTables {
     float clsR[8];           // RN(1 / Dref)
     int cnt[kLists];         // members per list
     uint32_t kind_mask[3][8];
+    // pruned sweep only
+    uint8_t below[kLists - 1][256];  // below[list][E]: members of the paired list whose D has a biased exponent < E
+    int flat_zero_min;               // smallest code of the flat list that has the multiplier 0; 256 if none
 };
 
 template <int FMT>
@@ -78,7 +81,8 @@ __device__ __forceinline__ int members_base(int list) {
 }
 
 // first: smallest admissible code (1 under prevent-zero for the FP8 formats, else 0).
-template <int FMT>
+// PRUNE: also the exponent index of the lists that the pruned sweep cuts its ranges with.
+template <int FMT, bool PRUNE>
 __device__ __forceinline__ void build_brute_tables(BruteTables& T, float g, int first) {
     static_assert(kThreads == 256, "one thread per table entry");
     build_scale_tables<FMT>(T.D, T.R, g);
@@ -92,6 +96,7 @@ __device__ __forceinline__ void build_brute_tables(BruteTables& T, float g, int 
     const int kind = !usable ? 2 : (!is_paired ? 3 : (__half2float(hD) == -D ? 1 : 0));
     T.kind[c] = (uint8_t)kind;
     if (c < kLists) T.cnt[c] = 0;
+    if (c == 0) T.flat_zero_min = 256;
     const uint32_t ballot0 = __ballot_sync(0xFFFFFFFFu, kind == 0);
     const uint32_t ballot1 = __ballot_sync(0xFFFFFFFFu, kind == 1);
     const uint32_t ballot3 = __ballot_sync(0xFFFFFFFFu, kind == 3);
@@ -111,7 +116,9 @@ __device__ __forceinline__ void build_brute_tables(BruteTables& T, float g, int 
         T.cand[slot] = make_float4(-D, P, 0.0f, 0.0f);
         T.member[slot] = (uint8_t)c;
         atomicAdd(&T.cnt[kFlatList], 1);
+        if (P == 0.0f) atomicMin(&T.flat_zero_min, c);
     }
+    int my_list = -1, my_rank = 0;
     if (is_paired) {
         const int cls = code_class<FMT>(c);
         int rank = 0;
@@ -129,6 +136,8 @@ __device__ __forceinline__ void build_brute_tables(BruteTables& T, float g, int 
         T.cand[slot] = make_float4(-D, P, __uint_as_float(h16 | (h16 << 16)), 0.0f);
         T.member[slot] = (uint8_t)c;
         atomicAdd(&T.cnt[list], 1);
+        my_list = list;
+        my_rank = rank;
         if (rank == 0) {   // both kinds of a class write the same values
             const float Dref = __uint_as_float((b & 0x007FFFFFu) | 0x3F800000u);
             T.clsD[cls] = Dref;
@@ -136,11 +145,26 @@ __device__ __forceinline__ void build_brute_tables(BruteTables& T, float g, int 
         }
     }
     __syncthreads();
-    // the search takes two members per trip: an odd list repeats its last member once
-    if (c < kLists && (T.cnt[c] & 1)) {
+    // the search takes two members per trip: a range that ends with the list may read one slot
+    // past it, which repeats the last member
+    if (c < kLists && T.cnt[c] > 0) {
         const int last = members_base<FMT>(c) + T.cnt[c] - 1;
         T.cand[last + 1] = T.cand[last];
         T.member[last + 1] = T.member[last];
+    }
+    if constexpr (PRUNE) {
+        // Exponents rise strictly along a paired list (one member per binade of its class), so
+        // member `rank` owns the exponents above its predecessor's up to its own, and the last
+        // member also those above.
+        if (my_list >= 0) {
+            const int slot = members_base<FMT>(my_list) + my_rank;
+            const int e_prev = my_rank > 0 ? (int)((__float_as_uint(T.cand[slot - 1].x) >> 23) & 0xFFu) : -1;
+            for (int E = e_prev + 1; E <= (int)e; ++E) T.below[my_list][E] = (uint8_t)my_rank;
+            if (my_rank == T.cnt[my_list] - 1)
+                for (int E = (int)e + 1; E < 256; ++E) T.below[my_list][E] = (uint8_t)(my_rank + 1);
+        }
+        for (int l = 0; l < kLists - 1; ++l)
+            if (T.cnt[l] == 0) T.below[l][c] = 0;
     }
     __syncthreads();
 }
@@ -237,33 +261,53 @@ __device__ __forceinline__ void keep_smaller(uint32_t& best_bits, int& best_slot
     best_bits = min(best_bits, bits);
 }
 
-// All members of one list (one mantissa class, one residual kind) against the thread's elements;
-// the list winner of every block is folded into best[].
-// Number of leading members of a list that have to be evaluated when no magnitude the warp holds
-// exceeds limit / 4.  A member with D >= limit quantizes every such element to zero
-// (|v| / D <= 1/4, and the tie at 1/4 goes to the even index 0), so its SSE is the sum of squares
-// of the block for every such member alike; members are in ascending order of D, so these form a
-// suffix of the list.  The smallest code left out is folded into skipped_min.
-template <int FMT>
-__device__ __forceinline__ int admitted_members(const BruteTables& T, int list, float limit, int& skipped_min) {
-    const int cnt = T.cnt[list];
-    const int base = members_base<FMT>(list);
-    int n = cnt;
-    while (n > 0 && -T.cand[base + n - 1].x >= limit) --n;
-    if (n < cnt) skipped_min = min(skipped_min, (int)T.member[base + n]);
-    return n;
+// ------------------------------------------------------------------------------------------------
+// Pruned sweep.  Three facts about a candidate D let a warp leave it out without changing any
+// output (they concern the thread's elements v, magnitudes a = max |v| of a block, and the SSE as
+// the kernel computes it: e = fma(q, -D, v), s = fma(e, e, s) in element order; binary32 rounding
+// is monotone, so a sum of squares never decreases when a term is added or a term grows):
+//   zero rule   D >= 4 * (largest magnitude in the warp): every quotient is at most 1/4 and rounds
+//               to the grid value 0 (the tie goes to the even index), so every such candidate has
+//               exactly the SSE of the all-zero quantization.  That SSE is entered once, with the
+//               smallest such code.
+//   high rule   D >= 4 * theta: the elements with |v| <= theta quantize to zero, so the SSE of a
+//               block is at least Z = the sum of squares of those elements (same order).  If
+//               Z > best SSE found so far, for every block of the warp, no such candidate can win
+//               or tie.  theta = largest magnitude * 2^-j, j = 2, 3, 4.
+//   low rule    6 * D <= a: the largest element saturates at 6 and leaves the error
+//               e = fl(a - 6 D), so the SSE is at least fl(e * e).  Every D below a D' that passes
+//               "fl(fl(a - 6 D')^2) > best SSE so far" (smallest a and largest best SSE of the
+//               thread's blocks; then the smallest D' of the warp) can neither win nor tie.
+// The cuts are taken per mantissa class from the exponent index below[][]: D = Dref * 2^E is
+// below a limit L = mL * 2^eL  <=>  E < eL + (Dref < mL).
+// ------------------------------------------------------------------------------------------------
+// Exponent cut of a limit (bit pattern of a non-negative binary32, +inf allowed) for a class whose
+// reference has the significand field cls_mant: the members of the class's lists with a biased
+// exponent below the cut, T.below[list][cut] of them, are the ones whose decode scale is below
+// the limit.
+__device__ __forceinline__ uint32_t exponent_cut(uint32_t cls_mant, uint32_t limit_bits) {
+    const uint32_t eL = limit_bits >> 23, mL = limit_bits & 0x007FFFFFu;
+    return min(eL + (cls_mant < mL ? 1u : 0u), 255u);
 }
 
-// cnt_raw: the first cnt_raw members of the list are evaluated.
+// limit * 2^-j for a limit given as bits (0 when that leaves the normal range)
+__device__ __forceinline__ uint32_t limit_shifted_down(uint32_t limit_bits, int j) {
+    return (limit_bits >> 23) > (uint32_t)j ? limit_bits - ((uint32_t)j << 23) : 0u;
+}
+
+// All members of one range of one list (one mantissa class, one residual kind) against the
+// thread's elements; the winner of every block is folded into best[].
+// Members first .. first + cnt_raw - 1 of the list are evaluated.
 template <int B, int FMT, bool HALF, int NP, int NBT>
-__device__ __forceinline__ void search_list(const BruteTables& T, int list, int cnt_raw, const float2 (&v2)[NP],
-                                            const float2 (&tb)[NP], unsigned long long (&best)[NBT]) {
+__device__ __forceinline__ void search_list(const BruteTables& T, int list, int first, int cnt_raw,
+                                            const float2 (&v2)[NP], const float2 (&tb)[NP],
+                                            unsigned long long (&best)[NBT]) {
     constexpr bool SKEW = (B >= 32);
     constexpr int BL = SKEW ? NP : B;
     constexpr int NBL = NP / BL;
-    if (cnt_raw == 0) return;
+    if (cnt_raw <= 0) return;
     [[maybe_unused]] const int cnt = cnt_raw;
-    const int base = members_base<FMT>(list);
+    const int base = members_base<FMT>(list) + first;
     const float4* cand = T.cand + base;
     uint32_t cbest[NBT];
     int cslot[NBT];
@@ -353,13 +397,13 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, int 
         if (cbest[k] != 0xFFFFFFFFu) merge_class_winner(best[k], cbest[k], T.member[base + cslot[k]]);
 }
 
-// PRUNE: the sweep leaves out, per warp, the candidates that provably tie with the all-zero
-// quantization (see admitted_members()); the outputs are the same.
+// PRUNE: the sweep leaves out, per warp, the candidates that provably cannot change an output
+// (see "Pruned sweep" above).
 //
 // Resident CTAs per SM asked of the register allocator: two where measurement showed that the
-// second CTA outweighs the few spills it costs (B = 4; B = 2 and B = 32 with the pruned sweep),
+// second CTA outweighs the few spills it costs (B = 4; every B up to 32 with the pruned sweep),
 // else no constraint beyond one CTA.
-constexpr int brute_min_ctas(int B, bool prune) { return (B == 4 || ((B == 2 || B == 32) && prune)) ? 2 : 1; }
+constexpr int brute_min_ctas(int B, bool prune) { return (B == 4 || (B <= 32 && prune)) ? 2 : 1; }
 
 template <int DT, int B, int FMT, bool PRUNE>
 __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(QuantArgs p) {
@@ -376,7 +420,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
     wait_for_prior_grid();
     const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
     const int first = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
-    build_brute_tables<FMT>(T, g, first);
+    build_brute_tables<FMT, PRUNE>(T, g, first);
 
     // all decode scales are short multiples of a class reference when g itself has few bits
     const bool short_ref = (__float_as_uint(g) & 0x1FFu) == 0u;   // <= 15 bits of g, <= 19 bits of Dref
@@ -390,16 +434,39 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
         const size_t grp = active ? wbase + lane : wbase;
         float2 v2[NP];
         float amax = 0.0f;
+        [[maybe_unused]] float amin = 0.0f;   // PRUNE: smallest block maximum of the thread
         bool tiny = false;   // a nonzero magnitude below 2^-62: its quotient by Dref may be inexact
         {
             float v[G];
             load_elems<DT, G>(p.x, grp * G, v);
+            if constexpr (PRUNE && !SKEW) {
+                float2 bmax[NBL];
 #pragma unroll
-            for (int i = 0; i < NP; ++i) {
-                v2[i] = make_float2(v[i], v[NP + i]);
-                const float a0 = fabsf(v[i]), a1 = fabsf(v[NP + i]);
-                amax = fmaxf(amax, fmaxf(a0, a1));
-                tiny |= (a0 < kTiny && a0 != 0.0f) || (a1 < kTiny && a1 != 0.0f);
+                for (int k = 0; k < NBL; ++k) bmax[k] = make_float2(0.0f, 0.0f);
+#pragma unroll
+                for (int i = 0; i < NP; ++i) {
+                    v2[i] = make_float2(v[i], v[NP + i]);
+                    const float a0 = fabsf(v[i]), a1 = fabsf(v[NP + i]);
+                    bmax[i / BL].x = fmaxf(bmax[i / BL].x, a0);
+                    bmax[i / BL].y = fmaxf(bmax[i / BL].y, a1);
+                    tiny |= (a0 < kTiny && a0 != 0.0f) || (a1 < kTiny && a1 != 0.0f);
+                }
+                amin = fminf(bmax[0].x, bmax[0].y);
+                amax = fmaxf(bmax[0].x, bmax[0].y);
+#pragma unroll
+                for (int k = 1; k < NBL; ++k) {
+                    amin = fminf(amin, fminf(bmax[k].x, bmax[k].y));
+                    amax = fmaxf(amax, fmaxf(bmax[k].x, bmax[k].y));
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < NP; ++i) {
+                    v2[i] = make_float2(v[i], v[NP + i]);
+                    const float a0 = fabsf(v[i]), a1 = fabsf(v[NP + i]);
+                    amax = fmaxf(amax, fmaxf(a0, a1));
+                    tiny |= (a0 < kTiny && a0 != 0.0f) || (a1 < kTiny && a1 != 0.0f);
+                }
+                amin = amax;
             }
         }
         const bool fast_ok = (amax <= kFastMax) && !tiny;
@@ -409,38 +476,164 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
 #pragma unroll
         for (int k = 0; k < NBT; ++k) best[k] = sse_key(__uint_as_float(0xFFFFFFFFu), first);
 
-        // Pruned sweep: candidates whose decode scale is at least four times the largest magnitude
-        // in the warp are not evaluated one by one; they all have the SSE of the all-zero
-        // quantization, which is entered once with the smallest such code.  4 * max is exact, or
-        // +inf when it overflows (nothing is left out then).
-        [[maybe_unused]] float limit = 0.0f;
-        if constexpr (PRUNE)
-            limit = __fmul_rn(4.0f, __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax))));
-        int skipped_min = 256;
-
-        if (fast_ok) {
-            for (int cls = 0; cls < NCLS; ++cls) {
-                int n0, n1;
-                if constexpr (PRUNE) {
-                    n0 = admitted_members<FMT>(T, 2 * cls, limit, skipped_min);
-                    n1 = admitted_members<FMT>(T, 2 * cls + 1, limit, skipped_min);
-                } else {
-                    n0 = T.cnt[2 * cls];
-                    n1 = T.cnt[2 * cls + 1];
-                }
-                if (n0 + n1 == 0) continue;
-                const float Dr = T.clsD[cls], Rr = T.clsR[cls];
-                const float2 nDr2 = make_float2(-Dr, -Dr), Rr2 = make_float2(Rr, Rr);
-                float2 tb[NP];
+        auto class_quotients = [&](int cls, float2 (&tb)[NP]) {
+            const float Dr = T.clsD[cls], Rr = T.clsR[cls];
+            const float2 nDr2 = make_float2(-Dr, -Dr), Rr2 = make_float2(Rr, Rr);
 #pragma unroll
-                for (int i = 0; i < NP; ++i)
-                    tb[i] = short_ref ? quotient_pair_short(v2[i], nDr2, Rr2) : quotient_pair(v2[i], nDr2, Rr2);
-                search_list<B, FMT, false>(T, 2 * cls, n0, v2, tb, best);
-                search_list<B, FMT, true>(T, 2 * cls + 1, n1, v2, tb, best);
+            for (int i = 0; i < NP; ++i)
+                tb[i] = short_ref ? quotient_pair_short(v2[i], nDr2, Rr2) : quotient_pair(v2[i], nDr2, Rr2);
+        };
+
+        if constexpr (!PRUNE) {
+            if (fast_ok) {
+                for (int cls = 0; cls < NCLS; ++cls) {
+                    const int n0 = T.cnt[2 * cls], n1 = T.cnt[2 * cls + 1];
+                    if (n0 + n1 == 0) continue;
+                    float2 tb[NP];
+                    class_quotients(cls, tb);
+                    search_list<B, FMT, false>(T, 2 * cls, 0, n0, v2, tb, best);
+                    search_list<B, FMT, true>(T, 2 * cls + 1, 0, n1, v2, tb, best);
+                }
+                // Dref = 1: the elements are their own quotients
+                search_list<B, FMT, false>(T, kFlatList, 0, T.cnt[kFlatList], v2, v2, best);
             }
-            // Dref = 1: the elements are their own quotients
-            search_list<B, FMT, false>(T, kFlatList, T.cnt[kFlatList], v2, v2, best);
-            if (PRUNE && skipped_min < 256) {
+        } else {
+            // Warp-wide steps are taken by every lane; lanes on the general path contribute neutral
+            // values and evaluate nothing here.
+            constexpr uint32_t kFull = 0xFFFFFFFFu, kInfBits = 0x7F800000u;
+            const float wmax = __uint_as_float(__reduce_max_sync(kFull, fast_ok ? __float_as_uint(amax) : 0u));
+            const uint32_t zero_limit = __float_as_uint(__fmul_rn(4.0f, wmax));   // exact: wmax <= 2^60
+            int skipped_min = 256;     // smallest code left out under the zero rule
+            uint32_t high_limit = zero_limit, low_limit = 0u;
+
+            // Ranges of one class: [lo, hi) of either kind, and the zero rule's bookkeeping.
+            auto class_ranges = [&](int cls, int (&lo)[2], int (&hi)[2]) {
+                const uint32_t mant = __float_as_uint(T.clsD[cls]) & 0x007FFFFFu;
+                const uint32_t cut_zero = exponent_cut(mant, zero_limit), cut_high = exponent_cut(mant, high_limit);
+                const uint32_t cut_low = exponent_cut(mant, low_limit);
+#pragma unroll
+                for (int kind = 0; kind < 2; ++kind) {
+                    const int list = 2 * cls + kind;
+                    const int nz = T.below[list][cut_zero];
+                    skipped_min = min(skipped_min, nz < T.cnt[list] ? (int)T.member[members_base<FMT>(list) + nz] : 256);
+                    hi[kind] = min(nz, (int)T.below[list][cut_high]);
+                    lo[kind] = min(hi[kind], (int)T.below[list][cut_low]);
+                }
+            };
+
+            // First the members of class 0 within nine binades below the zero rule's limit: the
+            // optimum of nearly every block lies there, which makes the bounds below tight.
+            int lo0[2] = {0, 0}, hi0[2] = {0, 0}, probe[2] = {0, 0};
+            const bool have0 = T.cnt[0] + T.cnt[1] > 0;
+            if (have0) {
+                class_ranges(0, lo0, hi0);
+                const uint32_t mant = __float_as_uint(T.clsD[0]) & 0x007FFFFFu;
+                const uint32_t cut_probe = exponent_cut(mant, limit_shifted_down(zero_limit, 9));
+                probe[0] = min(hi0[0], (int)T.below[0][cut_probe]);
+                probe[1] = min(hi0[1], (int)T.below[1][cut_probe]);
+                if (fast_ok) {
+                    float2 tb[NP];
+                    class_quotients(0, tb);
+                    search_list<B, FMT, false>(T, 0, probe[0], hi0[0] - probe[0], v2, tb, best);
+                    search_list<B, FMT, true>(T, 1, probe[1], hi0[1] - probe[1], v2, tb, best);
+                }
+            }
+
+            // Bounds from what has been found so far.
+            {
+                uint32_t ubits = 0u;       // largest best SSE of the thread's blocks
+#pragma unroll
+                for (int k = 0; k < NBT; ++k) ubits = max(ubits, (uint32_t)(best[k] >> 32));
+                float low = __uint_as_float(kInfBits);
+                int jt = 4;
+                if (fast_ok) {
+                    // low rule: a trial D' a little below (a - sqrt(U)) / 6, kept only if it passes the test itself
+                    low = 0.0f;
+                    if (ubits < kInfBits) {
+                        const float r = __fmul_rn(__fsqrt_ru(__uint_as_float(ubits)), 1.0009765625f);
+                        const float d = __fmul_rn(__fsub_rn(amin, r), 0.1665f);
+                        if (d > 0.0f) {
+                            const float e = __fmaf_rn(-6.0f, d, amin);
+                            if (e >= 0.0f && __float_as_uint(__fmul_rn(e, e)) > ubits) low = d;
+                        }
+                    }
+                    // high rule: the largest j in {2, 3, 4} whose bound exceeds the best SSE of every block
+                    // (a j that fails makes the larger ones fail as well); j = 3 is tried first
+                    auto bound_exceeds_best = [&](int j) {
+                        const float theta = __fmul_rn(wmax, 1.0f / (float)(1 << j));
+                        bool pass = true;
+                        if constexpr (!SKEW) {
+                            float2 z[NBL];
+#pragma unroll
+                            for (int k = 0; k < NBL; ++k) z[k] = make_float2(0.0f, 0.0f);
+#pragma unroll
+                            for (int i = 0; i < NP; ++i) {
+                                const float2 m = make_float2(fabsf(v2[i].x) <= theta ? v2[i].x : 0.0f,
+                                                             fabsf(v2[i].y) <= theta ? v2[i].y : 0.0f);
+                                z[i / BL] = __ffma2_rn(m, m, z[i / BL]);
+                            }
+#pragma unroll
+                            for (int k = 0; k < NBL; ++k) {
+                                pass &= __float_as_uint(z[k].x) > (uint32_t)(best[k] >> 32);
+                                pass &= __float_as_uint(z[k].y) > (uint32_t)(best[NBL + k] >> 32);
+                            }
+                        } else {
+                            float z = 0.0f;
+#pragma unroll
+                            for (int i = 0; i < NP; ++i) {
+                                const float m = fabsf(v2[i].x) <= theta ? v2[i].x : 0.0f;
+                                z = __fmaf_rn(m, m, z);
+                            }
+#pragma unroll
+                            for (int i = 0; i < NP; ++i) {
+                                const float m = fabsf(v2[i].y) <= theta ? v2[i].y : 0.0f;
+                                z = __fmaf_rn(m, m, z);
+                            }
+                            pass = __float_as_uint(z) > (uint32_t)(best[0] >> 32);
+                        }
+                        return pass;
+                    };
+                    if (bound_exceeds_best(3))
+                        jt = bound_exceeds_best(4) ? 4 : 3;
+                    else
+                        jt = bound_exceeds_best(2) ? 2 : 0;
+                }
+                low_limit = __reduce_min_sync(kFull, __float_as_uint(low));
+                const int jw = (int)__reduce_min_sync(kFull, (unsigned)jt);
+                high_limit = limit_shifted_down(zero_limit, jw);
+                if (high_limit == 0u) high_limit = zero_limit;
+            }
+
+            // the members of class 0 below the first range that the low rule keeps
+            if (have0) {
+                const uint32_t cut_low = exponent_cut(__float_as_uint(T.clsD[0]) & 0x007FFFFFu, low_limit);
+#pragma unroll
+                for (int kind = 0; kind < 2; ++kind) lo0[kind] = min(probe[kind], (int)T.below[kind][cut_low]);
+                if (fast_ok && probe[0] - lo0[0] + probe[1] - lo0[1] > 0) {
+                    float2 tb[NP];
+                    class_quotients(0, tb);    // formed again rather than kept: fewer live registers
+                    search_list<B, FMT, false>(T, 0, lo0[0], probe[0] - lo0[0], v2, tb, best);
+                    search_list<B, FMT, true>(T, 1, lo0[1], probe[1] - lo0[1], v2, tb, best);
+                }
+            }
+            for (int cls = 1; cls < NCLS; ++cls) {
+                if (T.cnt[2 * cls] + T.cnt[2 * cls + 1] == 0) continue;
+                int lo[2], hi[2];
+                class_ranges(cls, lo, hi);
+                if (hi[0] - lo[0] + hi[1] - lo[1] == 0 || !fast_ok) continue;
+                float2 tb[NP];
+                class_quotients(cls, tb);
+                search_list<B, FMT, false>(T, 2 * cls, lo[0], hi[0] - lo[0], v2, tb, best);
+                search_list<B, FMT, true>(T, 2 * cls + 1, lo[1], hi[1] - lo[1], v2, tb, best);
+            }
+            // Flat list.  Its members with a subnormal D lie below every normal low limit; the ones
+            // with the multiplier 0 fall under the zero rule.
+            if (low_limit >= 0x00800000u) {
+                skipped_min = min(skipped_min, T.flat_zero_min);
+            } else if (fast_ok) {
+                search_list<B, FMT, false>(T, kFlatList, 0, T.cnt[kFlatList], v2, v2, best);
+            }
+            if (fast_ok && skipped_min < 256) {
                 // all-zero quantization: e = v, summed in element order like every other candidate
                 if constexpr (!SKEW) {
                     float2 s0[NBL];

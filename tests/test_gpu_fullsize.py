@@ -40,6 +40,19 @@ def _check_sampled(x, B, fmt, recipe, g, codes, scales, sse, k, seed):
     assert bad.size == 0, f"block SSE differs at sampled blocks {idx[bad[:8]]}"
 
 
+def _pruned_sweep_equals(x, B, fmt, recipe, g, dg, codes, scales, sse):
+    """The pruned brute-force sweep must reproduce the full sweep on every byte of the tensor."""
+    mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 1)
+    try:
+        c2, s2, e2 = mxq.quantize(x, B, fmt, recipe, g, dg)
+        torch.cuda.synchronize()
+    finally:
+        mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 0)
+    assert torch.equal(s2, scales), f"scale bytes differ in {int((s2 != scales).sum())} blocks"
+    assert torch.equal(c2, codes)
+    assert torch.equal(e2.view(torch.int32), sse.view(torch.int32))
+
+
 def _mse_matches_sum(sse, n):
     got = float(mxq.tensor_mse(sse, n).cpu()[0])
     want = float(sse.double().sum().cpu()) / n       # another binary64 summation order
@@ -61,6 +74,8 @@ def test_weight_sweep_tensor_4096x4096_bf16_all_block_sizes():
                            100 * B + recipe)
             out[recipe] = sse
             mse[(B, recipe)] = _mse_matches_sum(sse, n)
+            if recipe == BRUTE:
+                _pruned_sweep_equals(x, B, mxq.MXQ_SF_UE4M3, recipe, 1.0, None, codes, scales, sse)
         # candidate sets nest, and the SSE is one function of (block, code): bitwise orderings
         assert bool((out[BRUTE] <= out[R4O6]).all()) and bool((out[R4O6] <= out[ABSMAX]).all())
         assert bool((out[ABSMAX_PZ] <= out[ABSMAX]).all())
@@ -133,6 +148,8 @@ def test_llama_shaped_weight_matrices_bf16(name, rows, cols):
                 _check_sampled(x, B, fmt, recipe, 1.0, codes, scales, sse, 1000 if recipe != BRUTE else 250,
                                B + fmt + recipe + index)
                 out[recipe] = sse
+                if recipe == BRUTE:
+                    _pruned_sweep_equals(x, B, fmt, recipe, 1.0, None, codes, scales, sse)
             assert bool((out[BRUTE] <= out[R4O6]).all()) and bool((out[R4O6] <= out[ABSMAX]).all())
             best[B] = _mse_matches_sum(out[BRUTE], n)
         assert best[8] <= best[16] * (1 + 1e-6)
@@ -159,6 +176,7 @@ def test_bulk_brute_force_16384x16384_fp32_laplace_with_tensor_scale(laplace_163
         codes, scales, sse = mxq.quantize(x, B, fmt, BRUTE, 1.0, dg)
         torch.cuda.synchronize()
         _check_sampled(x, B, fmt, BRUTE, g, codes, scales, sse, 250, 900 + B + fmt)
+        _pruned_sweep_equals(x, B, fmt, BRUTE, 1.0, dg, codes, scales, sse)
         m = _mse_matches_sum(sse, n)
         assert int(scales.max().cpu()) < (127 if fmt == mxq.MXQ_SF_UE4M3 else 255)
         if prev is not None:

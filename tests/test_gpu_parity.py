@@ -101,6 +101,29 @@ def test_brute_force_on_small_magnitudes_and_quarter_scale_ties(B, fmt, sweep_mo
         check_parity(xd, B, fmt, mxq.MXQ_BRUTE, 3.7e-3)
 
 
+@pytest.mark.parametrize("B", [8, 16, 32, 64])
+@pytest.mark.parametrize("fmt", FMTS)
+def test_brute_force_on_warps_of_unlike_blocks(B, fmt, sweep_mode):
+    """Blocks of very different magnitude side by side in one warp's share (one tiny block, one huge
+    block, blocks of equal elements, a block with a single nonzero element among ordinary ones): the
+    cases in which bounds taken from some blocks must not decide for the others."""
+    span = 32 * max(B, 32)
+    n = 8 * span
+    x = inputs.normal(n, 500 + B + fmt, 1.0, torch.float32)
+    xb = x.view(-1, B)
+    nb = xb.shape[0]
+    xb[1::37] *= 2.0 ** -9            # tiny blocks among ordinary ones
+    xb[5::41] *= 2.0 ** 7             # huge blocks
+    xb[7::43] = 0.75                  # constant blocks (zero error at the right scale)
+    xb[11::47] = 0.0
+    xb[11::47, 0] = -3.0              # one nonzero element
+    xb[13::53] = 0.0                  # all-zero blocks
+    xb[nb // 2:nb // 2 + 3] *= 2.0 ** -30
+    for g in (1.0, 0.0173):
+        check_parity(x, B, fmt, mxq.MXQ_BRUTE, g)
+    check_parity(x.to(torch.bfloat16), B, fmt, mxq.MXQ_BRUTE_PZ, 1.0)
+
+
 def test_option_calls_reject_bad_arguments():
     with pytest.raises(mxq.MxqError):
         mxq.mxq_set_option(99, 1)
