@@ -50,10 +50,10 @@ STREAM_ELEMS = 1 << 27            # tensor size of the streaming (HBM-bound) ker
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (same kernel build, same launch configuration); set an entry to None when its kernel changes.
 NCU_TRAFFIC_BYTES = {
-    "k_brute<bf16,B=16,UE4M3>@16Mi": 33.620480e6 + 3.84e3,
-    "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.497920e6 + 81.853696e6,
-    "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi": 268.530432e6 + 83.161600e6,
-    "k_quantize<f32,B=16,UE4M3,absmax>@128Mi": 536.909824e6 + 95.663616e6,
+    "k_brute<bf16,B=16,UE4M3>@16Mi": 33.620480e6 + 11.776e3,
+    "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.498432e6 + 81.372672e6,
+    "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi": 268.504320e6 + 82.705408e6,
+    "k_quantize<f32,B=16,UE4M3,absmax>@128Mi": 536.908032e6 + 94.972672e6,
 }
 
 
@@ -438,7 +438,7 @@ def run_gpu(args) -> None:
                      "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0, "traffic": None,
                      "ms_per_launch": ms, "gelem_s": N_ELEM / (ms * 1e-3) / 1e9, "peak_source": peaks["source"]}
     streaming = None if args.skip_streaming else streaming_rooflines(torch, mxq, device, peaks)
-    pruned = pruned_sweep_report(torch, mxq, wl)
+    pruned = None if args.skip_streaming else pruned_sweep_report(torch, mxq, wl)
     per_recipe = {"brute_B16": N_ELEM / (brute_ms * 1e-3) / 1e9, "absmax_B16": hbm["absmax_B16"]["gelem_s"],
                   "4o6_B16": hbm["4o6_B16"]["gelem_s"]}
 
@@ -488,6 +488,8 @@ def run_single_kernel(args) -> None:
     codes, scales, sse = mxq.alloc_outputs(n, B, dev)
     g = args.global_scale
     recipe = {"absmax": 0, "absmax_pz": 1, "4o6": 2, "4o6_pz": 3, "brute": 4, "brute_pz": 5}.get(args.kernel)
+    if args.prune:
+        mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 1)
     out = torch.empty(n, dtype=dtype, device=dev)
     amax = torch.empty(1, dtype=torch.float32, device=dev)
     mse = torch.empty(1, dtype=torch.float64, device=dev)
@@ -520,7 +522,7 @@ def run_single_kernel(args) -> None:
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
     ms = statistics.median(times)
-    res = {"kernel": args.kernel, "block": B, "dtype": args.dtype, "fmt": args.fmt, "elems": n, "ms": ms,
+    res = {"kernel": args.kernel + ("+prune" if args.prune else ""), "block": B, "dtype": args.dtype, "fmt": args.fmt, "elems": n, "ms": ms,
            "gelem_s": n / ms / 1e6, "algorithmic_gb_s": nbytes / ms / 1e6,
            "l2": "flushed between iterations" if flush is not None else "input larger than L2"}
     if recipe in (4, 5):
@@ -538,11 +540,13 @@ def main() -> None:
     ap.add_argument("--elems", type=int, default=1 << 27)
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--global-scale", type=float, default=1.0)
+    ap.add_argument("--prune", action="store_true", help="with --kernel brute|brute_pz: the pruned sweep")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--skip-streaming", action="store_true",
-                    help="leave out the 134M-element streaming measurements (roofline_hbm_streaming = null)")
+                    help="leave out the measurements taken outside the timed step: the 134M-element streaming "
+                         "launches and the pruned brute-force sweep (roofline_hbm_streaming, brute_pruned_sweep = null)")
     ap.add_argument("--impl", default="mxq", choices=["mxq", "reference"])
     args = ap.parse_args()
     if args.kernel:
