@@ -49,6 +49,15 @@ class _Acc:
         self.ms, self.elems, self.mse = {}, {}, {}
 
     def run(self, key, xs, B, fmt, recipe, g, dgs, bufs, rounds=1):
+        self._run(key, xs, B, fmt, recipe, g, dgs, bufs, rounds)
+        if recipe in (mxq.MXQ_BRUTE, mxq.MXQ_BRUTE_PZ):   # the same pass with the pruned sweep, as a row of its own
+            mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 1)
+            try:
+                self._run(key + ("pruned",), xs, B, fmt, recipe, g, dgs, bufs, rounds)
+            finally:
+                mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 0)
+
+    def _run(self, key, xs, B, fmt, recipe, g, dgs, bufs, rounds):
         codes, scales, sse, mse_out, ws = bufs
         dgs = dgs if dgs is not None else [None] * len(xs)
         mxq.mxq_quantize_ex(xs[0], xs[0].numel(), B, fmt, recipe, g, dgs[0], codes, scales, sse)
@@ -74,12 +83,18 @@ class _Acc:
     def rows(self, cfg, elem_bytes, hbm_gbs, alu_peak):
         out = []
         for key, ms in self.ms.items():
-            B, fmt, recipe, gk = key
+            B, fmt, recipe, gk = key[:4]
+            pruned = len(key) > 4
             n = self.elems[key]
             ge = n / ms / 1e6
-            row = {"config": cfg, "block": B, "scale_fmt": FMT_NAMES[fmt], "recipe": RECIPE_NAMES[recipe], "tensor_scale": gk,
+            row = {"config": cfg, "block": B, "scale_fmt": FMT_NAMES[fmt],
+                   "recipe": RECIPE_NAMES[recipe] + ("+prune" if pruned else ""), "tensor_scale": gk,
                    "elements": n, "ms": ms, "gelem_s": ge, "mse": self.mse[key][0] / self.mse[key][1]}
-            if recipe in (mxq.MXQ_BRUTE, mxq.MXQ_BRUTE_PZ):
+            if pruned:
+                # codes left out are not work done: no roofline fraction, only the speed-up over the full sweep
+                full = self.elems[key[:4]] / self.ms[key[:4]] / 1e6
+                row.update(bound="alu", speedup_over_full_sweep=ge / full, frac=None)
+            elif recipe in (mxq.MXQ_BRUTE, mxq.MXQ_BRUTE_PZ):
                 ach = ge * 1e9 * N_CODES[fmt] * 4 / 1e12
                 row.update(bound="alu", achieved_tlaneop_s=ach, frac=ach / alu_peak)
             else:
@@ -176,10 +191,14 @@ def main() -> None:
     args = ap.parse_args()
     res = run(tuple(int(c) for c in args.configs.split(",")))
     for r in res["rows"]:
+        head = (f'{r["config"][:28]:28s} B={r["block"]:<2d} {r["scale_fmt"]:5s} {r["recipe"]:14s} g={r["tensor_scale"]:9s} '
+                f'{r["gelem_s"]:9.1f} GElem/s  ')
+        if r["frac"] is None:
+            print(head + f'{r["speedup_over_full_sweep"]:8.2f} x the full sweep{"":14s}  mse={r["mse"]:.4e}')
+            continue
         ach = r.get("achieved_gb_s", r.get("achieved_tlaneop_s"))
         unit = "GB/s" if r["bound"] == "hbm" else "Tlop/s"
-        print(f'{r["config"][:28]:28s} B={r["block"]:<2d} {r["scale_fmt"]:5s} {r["recipe"]:9s} g={r["tensor_scale"]:9s} '
-              f'{r["gelem_s"]:9.1f} GElem/s  {ach:8.1f} {unit:6s} {100 * r["frac"]:5.1f}% of {r["bound"]}  mse={r["mse"]:.4e}')
+        print(head + f'{ach:8.1f} {unit:6s} {100 * r["frac"]:5.1f}% of {r["bound"]}  mse={r["mse"]:.4e}')
     if args.out:
         with open(args.out, "w") as f:
             json.dump(res, f, indent=1)
