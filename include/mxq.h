@@ -73,10 +73,14 @@ typedef enum { MXQ_SF_UE8M0 = 0, MXQ_SF_UE4M3 = 1, MXQ_SF_UE5M3 = 2 } mxq_scale_
  *              Background paraphrases it; Eq. 1 as printed differs): scale exponent = exponent of the
  *              block maximum minus the exponent of the largest FP4 value, S = 2^(floor(log2(amax/g)) - 2).
  *              The maximum lands in [4, 8) and is clipped above 6; S is the scale of Eq. 1 or twice it.
+ *   ABSMAX_CLIP7 MXQ_SF_UE8M0 only: the power-of-two scale that maps the block maximum into [3.5, 7)
+ *              (the clipping recipe of a cited work that the Background describes):
+ *              S = 2^floor(log2(amax/g / 3.5)); a maximum that lands in (6, 7) is clipped to 6.
+ *              S is the scale of Eq. 1 or twice it.
  * Hierarchical scaling is any recipe called with global_scale != 1. */
 typedef enum {
     MXQ_ABSMAX = 0, MXQ_ABSMAX_PZ = 1, MXQ_4O6 = 2, MXQ_4O6_PZ = 3, MXQ_BRUTE = 4, MXQ_BRUTE_PZ = 5,
-    MXQ_ABSMAX_OCP = 6
+    MXQ_ABSMAX_OCP = 6, MXQ_ABSMAX_CLIP7 = 7
 } mxq_recipe;
 
 /*

@@ -33,7 +33,8 @@
 
 enum { ORC_F32 = 0, ORC_BF16 = 1 };
 enum { ORC_UE8M0 = 0, ORC_UE4M3 = 1, ORC_UE5M3 = 2 };
-enum { ORC_ABSMAX = 0, ORC_ABSMAX_PZ = 1, ORC_4O6 = 2, ORC_4O6_PZ = 3, ORC_BRUTE = 4, ORC_BRUTE_PZ = 5, ORC_ABSMAX_OCP = 6 };
+enum { ORC_ABSMAX = 0, ORC_ABSMAX_PZ = 1, ORC_4O6 = 2, ORC_4O6_PZ = 3, ORC_BRUTE = 4, ORC_BRUTE_PZ = 5, ORC_ABSMAX_OCP = 6,
+       ORC_ABSMAX_CLIP7 = 7 };
 
 /* ---------------------------------------------------------------------------------------------
  * Number formats (Background; Experimental Setup).
@@ -216,6 +217,24 @@ int mxq_oracle_ocp_code(float amax, float g)
     return c;
 }
 
+/* The power-of-two scale that maps the block maximum into [3.5, 7) (Background: the clipping
+ * recipe of a cited work; a maximum that lands above 6 is clipped): the largest e with
+ * 3.5 * 2^e <= amax / g, written out as that search.  UE8M0 only. */
+int mxq_oracle_clip7_code(float amax, float g)
+{
+    float u = amax / g;
+    if (!(u > 0.0f)) return 0;
+    if (isinf(u)) return 254;
+    int e;
+    (void)frexpf(u, &e);                              /* a starting point near log2 u */
+    while ((double)ldexp(3.5, e) > (double)u) --e;    /* 3.5 * 2^e is exact in binary64 */
+    while ((double)ldexp(3.5, e + 1) <= (double)u) ++e;
+    int c = 127 + e;
+    if (c < 0) c = 0;
+    if (c > 254) c = 254;
+    return c;
+}
+
 /* Choose the scale code of one block by recipe; returns the code, writes the block's SSE. */
 static int choose_code(const float *v, int B, int fmt, int recipe, float g, float *sse_out)
 {
@@ -230,8 +249,8 @@ static int choose_code(const float *v, int B, int fmt, int recipe, float g, floa
     if (recipe == ORC_ABSMAX || recipe == ORC_ABSMAX_PZ) {
         best = absmax_code(amax, g, 6.0f, fmt, pz);
         best_sse = eval_block(v, B, fmt, best, g, NULL);
-    } else if (recipe == ORC_ABSMAX_OCP) {
-        best = mxq_oracle_ocp_code(amax, g);
+    } else if (recipe == ORC_ABSMAX_OCP || recipe == ORC_ABSMAX_CLIP7) {
+        best = (recipe == ORC_ABSMAX_OCP) ? mxq_oracle_ocp_code(amax, g) : mxq_oracle_clip7_code(amax, g);
         best_sse = eval_block(v, B, fmt, best, g, NULL);
     } else if (recipe == ORC_4O6 || recipe == ORC_4O6_PZ) {
         /* Eq. 4: argmin over M in {4, 6} of the block error; a tie keeps M = 6. */
@@ -288,8 +307,8 @@ int mxq_oracle_quantize(const void *x, int dtype, size_t n, int B, int fmt, int 
                         uint8_t *scales, float *block_sse)
 {
     if (!x || n == 0 || B < 2 || B > 64 || (B & (B - 1)) || n % (size_t)B) return -1;
-    if (mxq_oracle_num_codes(fmt) == 0 || recipe < 0 || recipe > ORC_ABSMAX_OCP) return -1;
-    if (recipe == ORC_ABSMAX_OCP && fmt != ORC_UE8M0) return -1;
+    if (mxq_oracle_num_codes(fmt) == 0 || recipe < 0 || recipe > ORC_ABSMAX_CLIP7) return -1;
+    if ((recipe == ORC_ABSMAX_OCP || recipe == ORC_ABSMAX_CLIP7) && fmt != ORC_UE8M0) return -1;
     if (!(g > 0.0f) || !isfinite(g)) return -1;
     quantize_range(x, dtype, 0, n / (size_t)B, B, fmt, recipe, g, codes, scales, block_sse);
     return 0;
@@ -314,8 +333,8 @@ int mxq_oracle_quantize_mt(const void *x, int dtype, size_t n, int B, int fmt, i
 {
     if (threads <= 1) return mxq_oracle_quantize(x, dtype, n, B, fmt, recipe, g, codes, scales, block_sse);
     if (!x || n == 0 || B < 2 || B > 64 || (B & (B - 1)) || n % (size_t)B) return -1;
-    if (mxq_oracle_num_codes(fmt) == 0 || recipe < 0 || recipe > ORC_ABSMAX_OCP) return -1;
-    if (recipe == ORC_ABSMAX_OCP && fmt != ORC_UE8M0) return -1;
+    if (mxq_oracle_num_codes(fmt) == 0 || recipe < 0 || recipe > ORC_ABSMAX_CLIP7) return -1;
+    if ((recipe == ORC_ABSMAX_OCP || recipe == ORC_ABSMAX_CLIP7) && fmt != ORC_UE8M0) return -1;
     if (!(g > 0.0f) || !isfinite(g)) return -1;
     if (threads > 256) threads = 256;
     pthread_t tid[256];

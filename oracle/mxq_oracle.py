@@ -18,7 +18,7 @@ _LIB = os.path.join(_HERE, "libmxq_oracle.so")
 
 F32, BF16 = 0, 1
 UE8M0, UE4M3, UE5M3 = 0, 1, 2
-ABSMAX, ABSMAX_PZ, R4O6, R4O6_PZ, BRUTE, BRUTE_PZ, ABSMAX_OCP = range(7)
+ABSMAX, ABSMAX_PZ, R4O6, R4O6_PZ, BRUTE, BRUTE_PZ, ABSMAX_OCP, ABSMAX_CLIP7 = range(8)
 
 _CFLAGS = ["-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared", "-pthread"]
 
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
                                             c.c_void_p, c.c_int]
         L.mxq_oracle_ocp_code.restype = c.c_int
         L.mxq_oracle_ocp_code.argtypes = [c.c_float, c.c_float]
+        L.mxq_oracle_clip7_code.restype = c.c_int
+        L.mxq_oracle_clip7_code.argtypes = [c.c_float, c.c_float]
         L.mxq_oracle_block_clip_sse.restype = c.c_int
         L.mxq_oracle_block_clip_sse.argtypes = [c.c_void_p, c.c_int, c.c_size_t, c.c_int, c.c_int, c.c_void_p, c.c_float,
                                                 c.c_void_p]
@@ -191,6 +193,10 @@ def segment_mse(block_sse_arr, blocks_per_segment: int, elems_per_segment: int):
 
 def ocp_code(amax, g: float = 1.0) -> int:
     return lib().mxq_oracle_ocp_code(float(np.float32(amax)), float(np.float32(g)))
+
+
+def clip7_code(amax, g: float = 1.0) -> int:
+    return lib().mxq_oracle_clip7_code(float(np.float32(amax)), float(np.float32(g)))
 
 
 def fake_quantize(x, block_size: int, fmt: int, recipe: int, g: float = 1.0, out_dtype: int = F32, threads: int = 1):

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libmxq.so")
 
 MXQ_F32, MXQ_BF16 = 0, 1
 MXQ_SF_UE8M0, MXQ_SF_UE4M3, MXQ_SF_UE5M3 = 0, 1, 2
-MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ, MXQ_ABSMAX_OCP = range(7)
+MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ, MXQ_ABSMAX_OCP, MXQ_ABSMAX_CLIP7 = range(8)
 MXQ_OPT_BRUTE_PRUNE = 1
 
 EXPORTS = (

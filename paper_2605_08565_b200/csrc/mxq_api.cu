@@ -48,8 +48,8 @@ static int quantize_common(const void* x, int dtype, size_t n, int block_size, i
     if (!x || (!out_xhat && (!out_codes || !out_scales))) return MXQ_ERR_NULL;
     if (dtype != MXQ_F32 && dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
     if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
-    if (recipe < MXQ_ABSMAX || recipe > MXQ_ABSMAX_OCP) return MXQ_ERR_BAD_ENUM;
-    if (recipe == MXQ_ABSMAX_OCP && scale_fmt != MXQ_SF_UE8M0) return MXQ_ERR_BAD_ENUM;
+    if (recipe < MXQ_ABSMAX || recipe > MXQ_ABSMAX_CLIP7) return MXQ_ERR_BAD_ENUM;
+    if ((recipe == MXQ_ABSMAX_OCP || recipe == MXQ_ABSMAX_CLIP7) && scale_fmt != MXQ_SF_UE8M0) return MXQ_ERR_BAD_ENUM;
     const bool brute = (recipe == MXQ_BRUTE || recipe == MXQ_BRUTE_PZ);
     if (out_xhat && (brute || (xhat_dtype != MXQ_F32 && xhat_dtype != MXQ_BF16))) return MXQ_ERR_BAD_ENUM;
     if (!valid_block(block_size) || n == 0 || n % (size_t)block_size != 0) return MXQ_ERR_BAD_SHAPE;
@@ -69,7 +69,7 @@ static int quantize_common(const void* x, int dtype, size_t n, int block_size, i
     a.scales = out_scales;
     a.block_sse = out_block_sse;
     a.prevent_zero = (recipe == MXQ_ABSMAX_PZ || recipe == MXQ_4O6_PZ || recipe == MXQ_BRUTE_PZ) ? 1 : 0;
-    a.ocp_floor = (recipe == MXQ_ABSMAX_OCP) ? 1 : 0;
+    a.pow2_rule = (recipe == MXQ_ABSMAX_OCP) ? kPow2Ocp : (recipe == MXQ_ABSMAX_CLIP7) ? kPow2Clip7 : kPow2Eq1;
     a.xhat = out_xhat;
     a.xhat_dtype = xhat_dtype;
 

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "mxq_internal.h"
+
 namespace mxq {
 
 constexpr int kF32 = 0, kBF16 = 1;
@@ -61,6 +63,20 @@ __device__ __forceinline__ int ocp_scale_code(float u) {
     const uint32_t b = __float_as_uint(u);               // u >= 0; subnormal u has exponent field 0
     if (b >= 0x7F800000u) return 254;                    // amax / g overflowed: the largest scale
     return max((int)(b >> 23) - 2, 0);
+}
+
+// The power-of-two scale that maps the (tensor-scale adjusted) block maximum u into [3.5, 7):
+// exponent floor(log2(u / 3.5)).  With u = m * 2^E, 1 <= m < 2, u / 3.5 = (m / 1.75) * 2^(E - 1),
+// so the exponent is E - 2 when m < 1.75 and E - 1 otherwise.
+__device__ __forceinline__ int clip7_scale_code(float u) {
+    const uint32_t b = __float_as_uint(u);
+    if (b >= 0x7F800000u) return 254;
+    return max((int)(b >> 23) - 2 + ((b & 0x007FFFFFu) >= 0x00600000u ? 1 : 0), 0);
+}
+
+// Scale code of the alternative power-of-two rules (rule != kPow2Eq1).
+__device__ __forceinline__ int pow2_rule_code(float u, int rule) {
+    return rule == kPow2Ocp ? ocp_scale_code(u) : clip7_scale_code(u);
 }
 
 // Per-CTA lookup tables: D[c] = fl32(value(c) * g) and R[c] = RN(1 / D[c]), or R[c] = 0 when the

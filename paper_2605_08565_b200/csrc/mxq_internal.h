@@ -11,6 +11,9 @@ constexpr int kMaxDevices = 64;
 
 // Arguments of the quantization kernels.  The launchers receive n_items = number of blocks and
 // hand their kernels n_items = what one thread owns per loop trip (chunks of blocks, or blocks).
+// Power-of-two scale rules (UE8M0): Eq. 1 as printed; the OCP wording; the [3.5, 7) target.
+enum { kPow2Eq1 = 0, kPow2Ocp = 1, kPow2Clip7 = 2 };
+
 struct QuantArgs {
     const void* x;
     size_t n_items;
@@ -21,7 +24,7 @@ struct QuantArgs {
     uint8_t* scales;
     float* block_sse;             // may be NULL
     int prevent_zero;
-    int ocp_floor;                // UE8M0 only: scale exponent = exponent of the block maximum - 2
+    int pow2_rule;                // UE8M0 only: which power-of-two rule (kPow2Eq1, kPow2Ocp, kPow2Clip7)
     void* xhat;                   // fused fake-quantize output (codes / scales may then be NULL), or NULL
     int xhat_dtype;
 };

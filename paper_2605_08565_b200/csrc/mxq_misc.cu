@@ -280,7 +280,7 @@ __global__ void k_quantize_tail(QuantArgs p, int dtype, int B, int dual) {
     }
     const bool pz = p.prevent_zero && FMT != kUE8M0;
     const float u = __fdiv_rn(amax, g);
-    int c = (FMT == kUE8M0 && p.ocp_floor) ? ocp_scale_code(u) : round_scale<FMT>(__fdiv_rn(u, 6.0f));
+    int c = (FMT == kUE8M0 && p.pow2_rule != kPow2Eq1) ? pow2_rule_code(u, p.pow2_rule) : round_scale<FMT>(__fdiv_rn(u, 6.0f));
     if (pz) c = max(c, 1);
     float s = tail_eval<FMT>(v, B, c, g, nullptr);
     if (dual) {

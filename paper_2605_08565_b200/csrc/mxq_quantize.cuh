@@ -228,14 +228,16 @@ __device__ __forceinline__ void encode_group_general(const float* v, const float
 struct QuantConsts {
     float g, Rg;        // tensor scale and RN(1 / g)
     float m_lo, m_hi;   // a block maximum m takes the shortcuts when m == 0 or m_lo <= m <= m_hi
-    bool unit_g, need_lo, pz, all_short, ocp;
+    bool unit_g, need_lo, pz, all_short;
+    int pow2_rule;      // kPow2Eq1 unless the format is UE8M0 and another rule was asked for
 };
 
-// Scale code for the M = 6 target from u = amax / g: Eq. 2 (Eq. 1 for UE8M0), or the OCP rule.
+// Scale code for the M = 6 target from u = amax / g: Eq. 2 (Eq. 1 for UE8M0), or one of the
+// alternative power-of-two rules.
 template <int FMT, bool EXACT>
-__device__ __forceinline__ int target6_code(float u, bool ocp) {
+__device__ __forceinline__ int target6_code(float u, int pow2_rule) {
     if constexpr (FMT == kUE8M0) {
-        if (ocp) return ocp_scale_code(u);
+        if (pow2_rule != kPow2Eq1) return pow2_rule_code(u, pow2_rule);
     }
     return round_scale<FMT>(EXACT ? __fdiv_rn(u, 6.0f) : div6_fast(u));
 }
@@ -268,7 +270,7 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             mmax = fmaxf(mmax, a);
             if (k.need_lo) mmin = fminf(mmin, a == 0.0f ? k.m_hi : a);
             u[j] = k.unit_g ? a : quotient_corrected(a, k.g, k.Rg);
-            c6[j] = target6_code<FMT, false>(u[j], k.ocp);
+            c6[j] = target6_code<FMT, false>(u[j], k.pow2_rule);
             if (k.pz) c6[j] = max(c6[j], 1);
             E6[j] = T.E[c6[j]];
             wmin = fminf(wmin, E6[j].w);
@@ -293,7 +295,7 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
 #pragma unroll
             for (int j = 0; j < NBG; ++j) {
                 u[j] = __fdiv_rn(m[j], k.g);
-                c6[j] = target6_code<FMT, true>(u[j], k.ocp);
+                c6[j] = target6_code<FMT, true>(u[j], k.pow2_rule);
                 if (k.pz) c6[j] = max(c6[j], 1);
                 E6[j] = T.E[c6[j]];
                 if constexpr (DUAL) {
@@ -413,7 +415,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     k.unit_g = (k.g == 1.0f);
     k.pz = p.prevent_zero && FMT != kUE8M0;
     k.all_short = T.all_short != 0;
-    k.ocp = (FMT == kUE8M0) && p.ocp_floor != 0;
+    k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;
     k.Rg = 1.0f;
     // Ranges of a block maximum m for which u = fl(m / g) and fl(u / 6) come out exact from the
     // multiply-and-correct forms.  The FP8 formats round every u below 2^-20 to code 0, so an

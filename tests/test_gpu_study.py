@@ -80,19 +80,25 @@ def test_reduced_numerical_study_against_oracle():
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("B", [2, 4, 8, 16, 32, 64])
-def test_ocp_power_of_two_recipe_bit_exact(dtype, B):
+@pytest.mark.parametrize("recipe", [mxq.MXQ_ABSMAX_OCP, mxq.MXQ_ABSMAX_CLIP7])
+def test_alternative_power_of_two_recipes_bit_exact(dtype, B, recipe):
     n = 3 * 256 * max(B, 8) + 5 * 64 + (B if B < 8 else 0)
     x = inputs.adversarial(n, 21 + B, dtype)
+    if recipe == mxq.MXQ_ABSMAX_CLIP7:      # block maxima on both sides of the 1.75 * 2^k edges of the rule
+        xb = x.view(-1, B)
+        k = torch.arange(xb.shape[0] // 3)
+        edge = torch.tensor([1.75, 1.7421875, 1.765625])[k % 3] * torch.exp2(((k // 3) % 24 - 12).float())
+        xb[::3][:k.numel(), 0] = edge.to(dtype)
     for g in (1.0, 0.0131, 2.0 ** -100):
         xg = x.cuda()
-        codes, scales, sse = mxq.quantize(xg, B, mxq.MXQ_SF_UE8M0, mxq.MXQ_ABSMAX_OCP, g)
+        codes, scales, sse = mxq.quantize(xg, B, mxq.MXQ_SF_UE8M0, recipe, g)
         torch.cuda.synchronize()
-        oc, os_, oe = orc.quantize(inputs.to_numpy_bits(x), B, orc.UE8M0, orc.ABSMAX_OCP, g)
+        oc, os_, oe = orc.quantize(inputs.to_numpy_bits(x), B, orc.UE8M0, recipe, g)
         assert np.array_equal(scales.cpu().numpy(), os_)
         assert np.array_equal(codes.cpu().numpy(), oc)
         assert np.array_equal(sse.cpu().numpy().view(np.uint32), oe.view(np.uint32))
     with pytest.raises(mxq.MxqError):
-        mxq.quantize(x.cuda(), B, mxq.MXQ_SF_UE4M3, mxq.MXQ_ABSMAX_OCP)
+        mxq.quantize(x.cuda(), B, mxq.MXQ_SF_UE4M3, recipe)
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])

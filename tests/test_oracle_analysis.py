@@ -3,6 +3,7 @@ segment MSE of the numerical study (CPU only)."""
 from fractions import Fraction
 
 import numpy as np
+import pytest
 
 import exact_ref as ex
 from oracle import mxq_oracle as orc
@@ -101,6 +102,34 @@ def test_ocp_power_of_two_rule_hand_worked_and_against_eq1():
     for b in range(4):
         s_b, _ = orc.block_sse(x[b * 32:(b + 1) * 32], orc.UE8M0, int(scales[b]))
         assert s_b == sse[b]
+
+
+def test_clip7_power_of_two_rule_hand_worked_and_against_eq1():
+    # S = 2^floor(log2(amax / 3.5)): the maximum lands in [3.5, 7) and is clipped above 6 (Background)
+    for amax, code in ((3.5, 127), (6.0, 127), (6.99, 127), (7.0, 128), (3.49, 126), (1.0, 125), (0.875, 125),
+                       (0.874, 124), (14.0, 129), (1.75, 126), (1.74, 125)):
+        assert orc.clip7_code(amax) == code, amax
+    assert orc.clip7_code(0.0) == 0
+    assert orc.clip7_code(1.0, 0.25) == orc.clip7_code(4.0)
+    assert orc.clip7_code(3.0e38, 1.0e-3) == 254                 # amax / g overflows: the largest scale
+    rng = np.random.default_rng(14)
+    for a in np.exp2(rng.uniform(-20, 20, 2000)).astype(np.float32):
+        c7, c_eq1 = orc.clip7_code(a), orc.round_scale(orc.UE8M0, np.float32(a) / np.float32(6.0))
+        q = Fraction(float(a)) / Fraction(2) ** (c7 - 127)
+        assert Fraction(7, 2) <= q < 7
+        # Eq. 1 takes the largest power of two <= fl(a / 6); on a binade edge the rounding of a / 6 may lift it
+        assert c7 - c_eq1 in (0, 1)
+    # the bottom of the code range: maxima below 3.5 * 2^-127 clamp to code 0
+    assert orc.clip7_code(np.float32(2.0 ** -126)) == 0 and orc.clip7_code(np.float32(3.5 * 2.0 ** -126)) == 1
+    x = (rng.standard_normal(1024) * 0.3).astype(np.float32)
+    codes, scales, sse = orc.quantize(x, 32, orc.UE8M0, orc.ABSMAX_CLIP7)
+    amax = np.abs(x.reshape(-1, 32)).max(axis=1)
+    assert np.array_equal(scales, np.array([orc.clip7_code(a) for a in amax], dtype=np.uint8))
+    for b in range(4):
+        s_b, _ = orc.block_sse(x[b * 32:(b + 1) * 32], orc.UE8M0, int(scales[b]))
+        assert s_b == sse[b]
+    with pytest.raises(Exception):
+        orc.quantize(x, 32, orc.UE4M3, orc.ABSMAX_CLIP7)
 
 
 def test_fake_quantize_is_dequantize_of_quantize():
