@@ -1,6 +1,6 @@
 """The five benchmark configurations of this library, timed one recipe at a time.
 
-    python -m paper_2605_08565_b200.configs [--configs 1,2,3,4,5] [--out results.json]
+    python -m paper_2605_08565_b200.configs [--configs 1,2,3,4,5] [--out results.json] [--hash-inputs]
 
 For every (configuration, block size, scale format, recipe) the quantize pass is timed with CUDA
 events over the whole synthetic workload (launches back to back; tensors larger than L2 or rotated
@@ -15,6 +15,7 @@ kernels; there is no CPU fallback.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import math
 import os
@@ -104,6 +105,25 @@ class _Acc:
         return out
 
 
+class _InputDigest:
+    """SHA-256 over the bytes of a configuration's input tensors, in generation order (so that a run
+    can be tied to the exact inputs it quantized); computed on the host, only when asked for."""
+
+    def __init__(self, enabled):
+        self.h = hashlib.sha256() if enabled else None
+        self.tensors, self.elements = 0, 0
+
+    def add(self, x):
+        self.tensors += 1
+        self.elements += x.numel()
+        if self.h is not None:
+            self.h.update(x.view(torch.uint8).cpu().numpy().tobytes())
+
+    def result(self):
+        return {"tensors": self.tensors, "elements": self.elements,
+                "sha256": self.h.hexdigest() if self.h is not None else None}
+
+
 def _bufs(n, B, dev):
     codes, scales, sse = mxq.alloc_outputs(n, B, dev)
     return (codes, scales, sse, torch.empty(1, dtype=torch.float64, device=dev),
@@ -117,7 +137,7 @@ def _tensor_scale(x):
     return dg
 
 
-def run(configs=(1, 2, 3, 4, 5), device="cuda"):
+def run(configs=(1, 2, 3, 4, 5), device="cuda", hash_inputs=False):
     if not torch.cuda.is_available():
         raise mxq.MxqError("needs a CUDA device (no CPU fallback)")
     dev = torch.device(device)
@@ -127,12 +147,15 @@ def run(configs=(1, 2, 3, 4, 5), device="cuda"):
     A, P, R4, BR = mxq.MXQ_ABSMAX, mxq.MXQ_ABSMAX_PZ, mxq.MXQ_4O6, mxq.MXQ_BRUTE
     U4, U5, U8 = mxq.MXQ_SF_UE4M3, mxq.MXQ_SF_UE5M3, mxq.MXQ_SF_UE8M0
     rows = []
+    digests = {}
     warm = inputs.normal(1 << 20, 0, 1.0, torch.float32, dev)          # first-launch costs out of the way
     for r in (A, R4, BR):
         mxq.quantize(warm, 16, U4, r)
 
     if 1 in configs:   # 1024 x 1024 fp32 N(0,1), B=16, UE4M3 + tensor scale; 4 MB: L2-resident, launch-bound
         x = inputs.normal(1024 * 1024, 1, 1.0, torch.float32, dev)
+        digests["C1"] = _InputDigest(hash_inputs)
+        digests["C1"].add(x)
         dg = _tensor_scale(x)
         acc, bufs = _Acc(), _bufs(x.numel(), 16, dev)
         for r in (A, R4, BR):
@@ -141,6 +164,9 @@ def run(configs=(1, 2, 3, 4, 5), device="cuda"):
 
     if 2 in configs:   # 4096 x 4096 bf16 0.02 * t5, all block sizes, UE4M3, no tensor scale; 8 rotating tensors
         xs = [inputs.student_t(4096 * 4096, 5, 0.02, 2 * 1_000_003 + i, torch.bfloat16, dev) for i in range(8)]
+        digests["C2"] = _InputDigest(hash_inputs)
+        for x in xs:
+            digests["C2"].add(x)
         acc = _Acc()
         for B in (2, 4, 8, 16, 32, 64):
             bufs = _bufs(xs[0].numel(), B, dev)
@@ -151,6 +177,9 @@ def run(configs=(1, 2, 3, 4, 5), device="cuda"):
 
     if 3 in configs:   # 8192 x 4096 bf16 N(0,1) with 1 % outlier columns x50, B=16; 4 rotating tensors
         xs = [inputs.outlier_columns(8192, 4096, 3 + i, dtype=torch.bfloat16, device=dev) for i in range(4)]
+        digests["C3"] = _InputDigest(hash_inputs)
+        for x in xs:
+            digests["C3"].add(x)
         dgs = [_tensor_scale(x) for x in xs]
         acc, bufs = _Acc(), _bufs(xs[0].numel(), 16, dev)
         for r in (A, R4):
@@ -161,9 +190,11 @@ def run(configs=(1, 2, 3, 4, 5), device="cuda"):
 
     if 4 in configs:   # Llama-3-8B-shaped weight set, 224 matrices, one at a time
         acc = _Acc()
+        digests["C4"] = _InputDigest(hash_inputs)
         for layer in range(inputs.LLAMA8B_LAYERS):
             for idx, (name, rows_, cols) in enumerate(inputs.LLAMA8B_LAYER_SHAPES):
                 x = inputs.student_t(rows_ * cols, 4, 1.0 / math.sqrt(cols), 4 + layer * 7 + idx, torch.bfloat16, dev)
+                digests["C4"].add(x)
                 for B in (8, 16):
                     bufs = _bufs(x.numel(), B, dev)
                     for fmt in (U4, U5):
@@ -174,6 +205,8 @@ def run(configs=(1, 2, 3, 4, 5), device="cuda"):
 
     if 5 in configs:   # 16384 x 16384 fp32 Laplace, brute force, tensor scale
         x = inputs.laplace(16384 * 16384, 5, torch.float32, dev)
+        digests["C5"] = _InputDigest(hash_inputs)
+        digests["C5"].add(x)
         dg = _tensor_scale(x)
         acc = _Acc()
         for B in (2, 4, 8, 16, 32):
@@ -181,15 +214,18 @@ def run(configs=(1, 2, 3, 4, 5), device="cuda"):
             for fmt in (U8, U4, U5):
                 acc.run((B, fmt, BR, "amax/2688"), [x], B, fmt, BR, 1.0, [dg], bufs)
         rows += acc.rows("C5 16384x16384 fp32 Laplace", 4, hbm, alu_peak)
-    return {"hbm_gbs": hbm, "alu_peak_tlaneop_s": alu_peak, "peak_source": src, "rows": rows}
+    return {"hbm_gbs": hbm, "alu_peak_tlaneop_s": alu_peak, "peak_source": src, "rows": rows,
+            "inputs": {k: d.result() for k, d in digests.items()}}
 
 
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--out", default=None)
+    ap.add_argument("--hash-inputs", action="store_true",
+                    help="record the SHA-256 of every configuration's input bytes (copies each tensor to the host once)")
     args = ap.parse_args()
-    res = run(tuple(int(c) for c in args.configs.split(",")))
+    res = run(tuple(int(c) for c in args.configs.split(",")), hash_inputs=args.hash_inputs)
     for r in res["rows"]:
         head = (f'{r["config"][:28]:28s} B={r["block"]:<2d} {r["scale_fmt"]:5s} {r["recipe"]:14s} g={r["tensor_scale"]:9s} '
                 f'{r["gelem_s"]:9.1f} GElem/s  ')
@@ -199,6 +235,8 @@ def main() -> None:
         ach = r.get("achieved_gb_s", r.get("achieved_tlaneop_s"))
         unit = "GB/s" if r["bound"] == "hbm" else "Tlop/s"
         print(head + f'{ach:8.1f} {unit:6s} {100 * r["frac"]:5.1f}% of {r["bound"]}  mse={r["mse"]:.4e}')
+    for cfg, d in res["inputs"].items():
+        print(f'{cfg}: {d["tensors"]} tensors, {d["elements"]} elements' + (f', sha256 {d["sha256"]}' if d["sha256"] else ""))
     if args.out:
         with open(args.out, "w") as f:
             json.dump(res, f, indent=1)
