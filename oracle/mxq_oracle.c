@@ -226,9 +226,8 @@ int mxq_oracle_clip7_code(float amax, float g)
     if (!(u > 0.0f)) return 0;
     if (isinf(u)) return 254;
     int e;
-    (void)frexpf(u, &e);                              /* a starting point near log2 u */
+    (void)frexpf(u, &e);                              /* u = f * 2^e with f < 1, so 3.5 * 2^e > u: start above */
     while ((double)ldexp(3.5, e) > (double)u) --e;    /* 3.5 * 2^e is exact in binary64 */
-    while ((double)ldexp(3.5, e + 1) <= (double)u) ++e;
     int c = 127 + e;
     if (c < 0) c = 0;
     if (c > 254) c = 254;

@@ -38,7 +38,9 @@ _lib = None
 def lib() -> ctypes.CDLL:
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(build())
+        # MXQ_ORACLE_LIB: load another build of the oracle (the tests plant mistakes in copies of the
+        # C source to show that the pins notice them)
+        L = ctypes.CDLL(os.environ.get("MXQ_ORACLE_LIB") or build())
         c = ctypes
         L.mxq_oracle_num_codes.restype = c.c_int
         L.mxq_oracle_num_codes.argtypes = [c.c_int]

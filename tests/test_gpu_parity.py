@@ -144,6 +144,61 @@ def test_extreme_global_scales(recipe, sweep_mode):
     check_parity(x, 8, mxq.MXQ_SF_UE5M3, recipe, 5.0e-33)
 
 
+def _ulp_neighbours(center, span):
+    """float32 values from `span` units in the last place below `center` to `span` above."""
+    c = np.float32(center)
+    out = [c]
+    lo = hi = c
+    for _ in range(span):
+        lo = np.nextafter(lo, np.float32(-np.inf), dtype=np.float32)
+        hi = np.nextafter(hi, np.float32(np.inf), dtype=np.float32)
+        out += [lo, hi]
+    return out
+
+
+@pytest.mark.parametrize("fmt", [mxq.MXQ_SF_UE4M3, mxq.MXQ_SF_UE5M3])
+@pytest.mark.parametrize("g", [1.0, 0.0371, 1.0 / 3.0, 0.7, 1.9e-3])
+def test_elements_and_maxima_next_to_rounding_midpoints(fmt, g):
+    """Blocks built so that quotients fall within a few units in the last place of an FP4 midpoint of
+    the block's own decode scale, and block maxima within a few units of a scale-code midpoint (for
+    both 4-over-6 targets): the inputs on which a quotient that is not correctly rounded, or a target
+    computed with one division instead of two, picks the neighbouring code."""
+    B = 16
+    mids = [0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0]
+    blocks = []
+    n_codes = orc.num_codes(fmt)
+    for code in range(9, n_codes - 8, 7):
+        S = np.float32(orc.scale_value(fmt, code))
+        a = np.float32(np.float32(6.0) * np.float32(S * np.float32(g)))        # a block maximum that selects about this scale
+        head = np.zeros(B, dtype=np.float32)
+        head[0] = a
+        _, sc, _ = orc.quantize(head, B, fmt, orc.ABSMAX, g)
+        D = np.float32(np.float32(orc.scale_value(fmt, int(sc[0]))) * np.float32(g))
+        near = [v for m in mids for v in _ulp_neighbours(np.float32(m) * D, 2)]   # 35 values, all below the maximum
+        for i in range(0, len(near), B - 1):
+            blk = np.zeros(B, dtype=np.float32)
+            part = near[i:i + B - 1]
+            blk[1:1 + len(part)] = part
+            blk[1::2] *= -1
+            blk[0] = a
+            blocks.append(blk)
+        # maxima next to the midpoint between this scale code and the next, for M = 6 and M = 4
+        mid = (np.float64(orc.scale_value(fmt, code)) + np.float64(orc.scale_value(fmt, code + 1))) / 2
+        for M in (6.0, 4.0):
+            for a2 in _ulp_neighbours(np.float32(mid * M * g), 3):
+                blk = np.zeros(B, dtype=np.float32)
+                blk[5] = -a2
+                blk[9] = a2 * np.float32(0.37)
+                blocks.append(blk)
+    x = torch.from_numpy(np.concatenate(blocks))
+    if not np.all(np.isfinite(x.numpy())):
+        x = torch.nan_to_num(x, nan=0.0, posinf=0.0, neginf=0.0)
+    for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_ABSMAX_PZ, mxq.MXQ_4O6, mxq.MXQ_4O6_PZ):
+        check_parity(x, B, fmt, recipe, g)
+        check_parity(x, B, fmt, recipe, g, device_g=True)
+    check_parity(x[: 64 * B], B, fmt, mxq.MXQ_BRUTE, g)
+
+
 def test_device_resident_global_scale_matches_host_scale():
     x = _mixed(8192, 5, torch.bfloat16)
     for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_4O6, mxq.MXQ_BRUTE):
