@@ -2,15 +2,17 @@
 // factors to minimize the MSE"): every finite scale code of the format is tried on every block and
 // the code with the smallest SSE is kept (equal SSE: the smaller code).
 //
-// Work layout.  A thread keeps its elements in registers as float pairs and runs every step of a
-// candidate on both halves of the pair at once with the packed binary32 instructions of sm_100
-// (fma.rn.f32x2 / mul.rn.f32x2), so one issue slot serves two elements:
-//   B <= 16   the thread owns 32 consecutive elements; pair i = (element i, element 16 + i), i.e.
-//             the two halves of a pair belong to different blocks and their SSE chains are
-//             independent.
-//   B >= 32   the thread owns one block; pair i = (element i, element B/2 + i).  The SSE of a
-//             block is one sequential chain, so the second half runs one candidate behind the
-//             first and starts from the first half's sum of the previous step.
+// Work layout.  A thread keeps its elements in registers as float pairs and the candidate loop
+// works on float pairs with the packed binary32 instructions of sm_100 (fma.rn.f32x2 /
+// mul.rn.f32x2, FP4 pack and unpack two at a time):
+//   B <= 16   the thread owns 32 consecutive elements, pair i = (element i, element 16 + i): the
+//             two halves of a pair belong to different blocks, so one instruction serves two
+//             elements of one candidate and the two SSE chains are independent.  Two candidates
+//             per trip.
+//   B >= 32   the thread owns one block, pair i = (element 2i, element 2i + 1).  Its SSE is one
+//             sequential chain over all elements, so the two lanes of the SSE pair are two
+//             CANDIDATES: the scaling multiplies run on element pairs, the FP4 rounding and the
+//             residuals on candidate pairs of one element, and the elements are walked in order.
 // The candidate loop is uniform across the CTA: decode scales come from shared memory as
 // broadcasts.
 //
@@ -204,6 +206,39 @@ __device__ __forceinline__ float2 residual_pair(float2 tb, float2 P2, float2 v, 
     }
 }
 
+// Residuals of ONE element for TWO candidates A, B, given its scaled quotients tA = tb * 2^-kA and
+// tB: q = FP4 rounding of t, e = fma(q, -D, v) for either candidate (.x = A, .y = B).  HALF: nD16
+// holds f16(-D_A) in the low half and f16(-D_B) in the high half.
+template <bool HALF>
+__device__ __forceinline__ float2 residual_two_candidates(float tA, float tB, float v, float nDA, float nDB,
+                                                          uint32_t nD16) {
+    uint32_t h;
+    asm("{\n"
+        " .reg .b8 b0;\n"
+        " cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n"
+        " cvt.rn.f16x2.e2m1x2 %0, b0;\n"
+        "}"
+        : "=r"(h)
+        : "f"(tA), "f"(tB));
+    float2 e;
+    if constexpr (HALF) {
+        asm("{\n"
+            " .reg .b16 qlo, qhi, dlo, dhi;\n"
+            " mov.b32 {qlo, qhi}, %2;\n"
+            " mov.b32 {dlo, dhi}, %3;\n"
+            " fma.rn.f32.f16 %0, qlo, dlo, %4;\n"
+            " fma.rn.f32.f16 %1, qhi, dhi, %4;\n"
+            "}"
+            : "=f"(e.x), "=f"(e.y)
+            : "r"(h), "r"(nD16), "f"(v));
+    } else {
+        const float2 q = __half22float2(*reinterpret_cast<__half2*>(&h));
+        e.x = __fmaf_rn(q.x, nDA, v);
+        e.y = __fmaf_rn(q.y, nDB, v);
+    }
+    return e;
+}
+
 // fl32(v / Dref) for both halves; nD = -Dref, R = RN(1 / Dref), Dref in [1, 2), |v| <= 2^60.
 // Same value as quotient_corrected() except for the sign of a zero quotient, which the search
 // does not use.
@@ -302,8 +337,8 @@ template <int B, int FMT, bool HALF, int NP, int NBT>
 __device__ __forceinline__ void search_list(const BruteTables& T, int list, int first, int cnt_raw,
                                             const float2 (&v2)[NP], const float2 (&tb)[NP],
                                             unsigned long long (&best)[NBT]) {
-    constexpr bool SKEW = (B >= 32);
-    constexpr int BL = SKEW ? NP : B;
+    constexpr bool ONEBLK = (B >= 32);
+    constexpr int BL = ONEBLK ? NP : B;
     constexpr int NBL = NP / BL;
     if (cnt_raw <= 0) return;
     [[maybe_unused]] const int cnt = cnt_raw;
@@ -314,7 +349,7 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, int 
 #pragma unroll
     for (int k = 0; k < NBT; ++k) { cbest[k] = 0xFFFFFFFFu; cslot[k] = 0; }
 
-    if constexpr (!SKEW) {
+    if constexpr (!ONEBLK) {
         // two members per trip: two independent SSE chains keep the FMA pipe fed
         const int pairs_end = cnt & ~1;
         for (int m = 0; m < pairs_end; m += 2) {
@@ -360,36 +395,23 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, int 
             }
         }
     } else {
-        // trip m: the low half evaluates members m and m + 1, the high half finishes members
-        // m - 2 and m - 1 from the low-half sums of the previous trip
-        // an odd count takes one more slot: the next member of the list, or the copy of the last
-        // member that the table build appends
-        const int cnt = cnt_raw + (cnt_raw & 1);
-        float nDA_prev = cand[0].x, PA_prev = cand[0].y, nDB_prev = nDA_prev, PB_prev = PA_prev;
-        uint32_t hA_prev = __float_as_uint(cand[0].z), hB_prev = hA_prev;
-        float carryA = 0.0f, carryB = 0.0f;
-        for (int m = 0; m < cnt + 2; m += 2) {
-            const int mm = m < cnt ? m : 0;   // past the end: repeat a trip, low-half result unused
-            const float4 dpA = cand[mm], dpB = cand[mm + 1];
-            const float2 nDA = make_float2(dpA.x, nDA_prev), PA = make_float2(dpA.y, PA_prev);
-            const float2 nDB = make_float2(dpB.x, nDB_prev), PB = make_float2(dpB.y, PB_prev);
-            const uint32_t hA = (__float_as_uint(dpA.z) & 0xFFFFu) | (hA_prev & 0xFFFF0000u);
-            const uint32_t hB = (__float_as_uint(dpB.z) & 0xFFFFu) | (hB_prev & 0xFFFF0000u);
-            float2 sA = make_float2(0.0f, carryA), sB = make_float2(0.0f, carryB);
+        // one block per thread: lane .x of the SSE pair is member m, lane .y member m + 1 (the
+        // slot behind an odd range holds a real member or the copy of the last one: harmless)
+        for (int m = 0; m < cnt; m += 2) {
+            const float4 dpA = cand[m], dpB = cand[m + 1];
+            const float2 PA = make_float2(dpA.y, dpA.y), PB = make_float2(dpB.y, dpB.y);
+            const uint32_t nD16 = (__float_as_uint(dpA.z) & 0xFFFFu) | (__float_as_uint(dpB.z) << 16);
+            float2 s = make_float2(0.0f, 0.0f);
 #pragma unroll
             for (int i = 0; i < NP; ++i) {
-                const float2 eA = residual_pair<HALF>(tb[i], PA, v2[i], nDA, hA);
-                const float2 eB = residual_pair<HALF>(tb[i], PB, v2[i], nDB, hB);
-                sA = __ffma2_rn(eA, eA, sA);
-                sB = __ffma2_rn(eB, eB, sB);
+                const float2 tA = __fmul2_rn(tb[i], PA), tB = __fmul2_rn(tb[i], PB);   // elements 2i, 2i + 1
+                const float2 e0 = residual_two_candidates<HALF>(tA.x, tB.x, v2[i].x, dpA.x, dpB.x, nD16);
+                s = __ffma2_rn(e0, e0, s);
+                const float2 e1 = residual_two_candidates<HALF>(tA.y, tB.y, v2[i].y, dpA.x, dpB.x, nD16);
+                s = __ffma2_rn(e1, e1, s);
             }
-            if (m > 0) {
-                keep_smaller(cbest[0], cslot[0], __float_as_uint(sA.y), m - 2);
-                keep_smaller(cbest[0], cslot[0], __float_as_uint(sB.y), m - 1);
-            }
-            carryA = sA.x; carryB = sB.x;
-            nDA_prev = dpA.x; PA_prev = dpA.y; nDB_prev = dpB.x; PB_prev = dpB.y;
-            hA_prev = __float_as_uint(dpA.z); hB_prev = __float_as_uint(dpB.z);
+            keep_smaller(cbest[0], cslot[0], __float_as_uint(s.x), m);
+            keep_smaller(cbest[0], cslot[0], __float_as_uint(s.y), m + 1);
         }
     }
 #pragma unroll
@@ -407,12 +429,12 @@ constexpr int brute_min_ctas(int B, bool prune) { return (B == 4 || (B <= 32 && 
 
 template <int DT, int B, int FMT, bool PRUNE>
 __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(QuantArgs p) {
-    constexpr bool SKEW = (B >= 32);          // the pair's halves are the two halves of one block
-    constexpr int G = SKEW ? B : 32;          // elements per thread
+    constexpr bool ONEBLK = (B >= 32);        // the thread owns exactly one block
+    constexpr int G = ONEBLK ? B : 32;          // elements per thread
     constexpr int NP = G / 2;                 // pairs per thread
-    constexpr int BL = SKEW ? NP : B;         // elements of one block inside one half
-    constexpr int NBL = NP / BL;              // blocks per half (1 when SKEW)
-    constexpr int NBT = SKEW ? 1 : 2 * NBL;   // blocks per thread
+    constexpr int BL = ONEBLK ? NP : B;         // elements of one block inside one half
+    constexpr int NBL = NP / BL;              // blocks per half (1 when ONEBLK)
+    constexpr int NBT = ONEBLK ? 1 : 2 * NBL;   // blocks per thread
     constexpr int NCLS = (FMT == kUE8M0) ? 1 : 8;
     constexpr float kTiny = 2.168404344971009e-19f;  // 2^-62
 
@@ -439,7 +461,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
         {
             float v[G];
             load_elems<DT, G>(p.x, grp * G, v);
-            if constexpr (PRUNE && !SKEW) {
+            if constexpr (PRUNE && !ONEBLK) {
                 float2 bmax[NBL];
 #pragma unroll
                 for (int k = 0; k < NBL; ++k) bmax[k] = make_float2(0.0f, 0.0f);
@@ -461,8 +483,10 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
             } else {
 #pragma unroll
                 for (int i = 0; i < NP; ++i) {
-                    v2[i] = make_float2(v[i], v[NP + i]);
-                    const float a0 = fabsf(v[i]), a1 = fabsf(v[NP + i]);
+                    // one block per thread: adjacent elements; else element i of either half
+                    const float x0 = ONEBLK ? v[2 * i] : v[i], x1 = ONEBLK ? v[2 * i + 1] : v[NP + i];
+                    v2[i] = make_float2(x0, x1);
+                    const float a0 = fabsf(x0), a1 = fabsf(x1);
                     amax = fmaxf(amax, fmaxf(a0, a1));
                     tiny |= (a0 < kTiny && a0 != 0.0f) || (a1 < kTiny && a1 != 0.0f);
                 }
@@ -562,7 +586,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
                     auto bound_exceeds_best = [&](int j) {
                         const float theta = __fmul_rn(wmax, 1.0f / (float)(1 << j));
                         bool pass = true;
-                        if constexpr (!SKEW) {
+                        if constexpr (!ONEBLK) {
                             float2 z[NBL];
 #pragma unroll
                             for (int k = 0; k < NBL; ++k) z[k] = make_float2(0.0f, 0.0f);
@@ -581,13 +605,10 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
                             float z = 0.0f;
 #pragma unroll
                             for (int i = 0; i < NP; ++i) {
-                                const float m = fabsf(v2[i].x) <= theta ? v2[i].x : 0.0f;
-                                z = __fmaf_rn(m, m, z);
-                            }
-#pragma unroll
-                            for (int i = 0; i < NP; ++i) {
-                                const float m = fabsf(v2[i].y) <= theta ? v2[i].y : 0.0f;
-                                z = __fmaf_rn(m, m, z);
+                                const float m0 = fabsf(v2[i].x) <= theta ? v2[i].x : 0.0f;
+                                z = __fmaf_rn(m0, m0, z);
+                                const float m1 = fabsf(v2[i].y) <= theta ? v2[i].y : 0.0f;
+                                z = __fmaf_rn(m1, m1, z);
                             }
                             pass = __float_as_uint(z) > (uint32_t)(best[0] >> 32);
                         }
@@ -635,7 +656,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
             }
             if (fast_ok && skipped_min < 256) {
                 // all-zero quantization: e = v, summed in element order like every other candidate
-                if constexpr (!SKEW) {
+                if constexpr (!ONEBLK) {
                     float2 s0[NBL];
 #pragma unroll
                     for (int k = 0; k < NBL; ++k) s0[k] = make_float2(0.0f, 0.0f);
@@ -650,9 +671,10 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
                 } else {
                     float s0 = 0.0f;
 #pragma unroll
-                    for (int i = 0; i < NP; ++i) s0 = __fmaf_rn(v2[i].x, v2[i].x, s0);
-#pragma unroll
-                    for (int i = 0; i < NP; ++i) s0 = __fmaf_rn(v2[i].y, v2[i].y, s0);
+                    for (int i = 0; i < NP; ++i) {
+                        s0 = __fmaf_rn(v2[i].x, v2[i].x, s0);
+                        s0 = __fmaf_rn(v2[i].y, v2[i].y, s0);
+                    }
                     const unsigned long long k0 = sse_key(s0, skipped_min);
                     if (k0 < best[0]) best[0] = k0;
                 }
@@ -665,7 +687,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
         for (int c = first; c < n_general; ++c) {
             const float D = T.D[c];
             if (!(fabsf(D) <= 3.402823466e38f)) continue;  // decode scale overflowed: not usable
-            if constexpr (!SKEW) {
+            if constexpr (!ONEBLK) {
 #pragma unroll
                 for (int k = 0; k < NBL; ++k) {
                     const unsigned long long k0 = sse_key(general_sse<B, NP>(v2, k * BL, 0, D), c);
@@ -676,17 +698,13 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
             } else {
                 float s = 0.0f;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                    for (int i = 0; i < NP; i += 2) {
-                        const float a = h ? v2[i].y : v2[i].x;
-                        const float b = h ? v2[i + 1].y : v2[i + 1].x;
-                        const float2 q = round_e2m1x2(quotient_general(a, D), quotient_general(b, D));
-                        const float e0 = __fmaf_rn(-q.x, D, a);
-                        s = __fmaf_rn(e0, e0, s);
-                        const float e1 = __fmaf_rn(-q.y, D, b);
-                        s = __fmaf_rn(e1, e1, s);
-                    }
+                for (int i = 0; i < NP; ++i) {
+                    const float a = v2[i].x, b = v2[i].y;
+                    const float2 q = round_e2m1x2(quotient_general(a, D), quotient_general(b, D));
+                    const float e0 = __fmaf_rn(-q.x, D, a);
+                    s = __fmaf_rn(e0, e0, s);
+                    const float e1 = __fmaf_rn(-q.y, D, b);
+                    s = __fmaf_rn(e1, e1, s);
                 }
                 const unsigned long long k0 = sse_key(s, c);
                 if (k0 < best[0]) best[0] = k0;
@@ -699,30 +717,48 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
         uint32_t sw[NBT];
 #pragma unroll
         for (int k = 0; k < (NBT + 3) / 4; ++k) sc[k] = 0;
+        if constexpr (ONEBLK) {
+            const int code = (int)(best[0] & 0xFFu);
+            const float D = T.D[code];
+            const float R = T.R[code];
+            const bool fast = (R != 0.0f) && (amax <= kFastMax);
+            sc[0] = (uint32_t)code;
+            sw[0] = (uint32_t)(best[0] >> 32);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            float t[NP];
+            for (int k = 0; k < G / 8; ++k) {
+                float t[8];
 #pragma unroll
-            for (int k = 0; k < NBL; ++k) {
-                const int kb = SKEW ? 0 : h * NBL + k;   // block index inside the thread
-                const int code = (int)(best[kb] & 0xFFu);
-                const float D = T.D[code];
-                const float R = T.R[code];
-                const bool fast = (R != 0.0f) && (amax <= kFastMax);
-#pragma unroll
-                for (int i = 0; i < BL; ++i) {
-                    const float a = h ? v2[k * BL + i].y : v2[k * BL + i].x;
-                    t[k * BL + i] = fast ? quotient_corrected(a, D, R) : quotient_general(a, D);
+                for (int i = 0; i < 4; ++i) {
+                    const float2 a = v2[4 * k + i];
+                    t[2 * i] = fast ? quotient_corrected(a.x, D, R) : quotient_general(a.x, D);
+                    t[2 * i + 1] = fast ? quotient_corrected(a.y, D, R) : quotient_general(a.y, D);
                 }
-                if (!SKEW || h == 0) {
+                packed[k] = pack_e2m1x8(t[0], t[1], t[2], t[3], t[4], t[5], t[6], t[7]);
+            }
+        } else {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float t[NP];
+#pragma unroll
+                for (int k = 0; k < NBL; ++k) {
+                    const int kb = h * NBL + k;   // block index inside the thread
+                    const int code = (int)(best[kb] & 0xFFu);
+                    const float D = T.D[code];
+                    const float R = T.R[code];
+                    const bool fast = (R != 0.0f) && (amax <= kFastMax);
+#pragma unroll
+                    for (int i = 0; i < BL; ++i) {
+                        const float a = h ? v2[k * BL + i].y : v2[k * BL + i].x;
+                        t[k * BL + i] = fast ? quotient_corrected(a, D, R) : quotient_general(a, D);
+                    }
                     sc[kb / 4] |= (uint32_t)code << (8 * (kb % 4));
                     sw[kb] = (uint32_t)(best[kb] >> 32);
                 }
-            }
 #pragma unroll
-            for (int k = 0; k < NP / 8; ++k)
-                packed[h * (NP / 8) + k] = pack_e2m1x8(t[8 * k], t[8 * k + 1], t[8 * k + 2], t[8 * k + 3], t[8 * k + 4],
-                                                       t[8 * k + 5], t[8 * k + 6], t[8 * k + 7]);
+                for (int k = 0; k < NP / 8; ++k)
+                    packed[h * (NP / 8) + k] = pack_e2m1x8(t[8 * k], t[8 * k + 1], t[8 * k + 2], t[8 * k + 3], t[8 * k + 4],
+                                                           t[8 * k + 5], t[8 * k + 6], t[8 * k + 7]);
+            }
         }
         if (!PRUNE || active) {
             store_bytes<G / 2>(p.codes + grp * (G / 2), packed);
