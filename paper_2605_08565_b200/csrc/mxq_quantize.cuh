@@ -197,6 +197,28 @@ __device__ __forceinline__ void pack_and_score(const float* v, const float* t, c
     }
 }
 
+// Quotients of one block by its decode scale, two elements per instruction (fma.rn.f32x2):
+// q = (-v) * (-R); r = q * D - v; q <- q - r * R, once (SHORTQ) or twice.  Same values as
+// quotient_short() / quotient_corrected(), including the sign of a zero quotient: every product and
+// sum has the signs of the scalar forms.
+template <int B, bool SHORTQ>
+__device__ __forceinline__ void block_quotients(const float* v, float D, float R, float* t) {
+    const float2 D2 = make_float2(D, D), nR2 = make_float2(-R, -R);
+#pragma unroll
+    for (int i = 0; i < B; i += 2) {
+        const float2 nv = make_float2(-v[i], -v[i + 1]);
+        float2 q = __fmul2_rn(nv, nR2);
+        float2 r = __ffma2_rn(q, D2, nv);
+        q = __ffma2_rn(r, nR2, q);
+        if constexpr (!SHORTQ) {
+            r = __ffma2_rn(q, D2, nv);
+            q = __ffma2_rn(r, nR2, q);
+        }
+        t[i] = q.x;
+        t[i + 1] = q.y;
+    }
+}
+
 // One candidate set of a group with the shortcuts (every entry has w != 0, magnitudes in range).
 template <int B, bool SHORTQ, bool HALF>
 __device__ __forceinline__ void encode_group_fast(const float* v, const float4* E, uint32_t* packed, float* sse) {
@@ -204,11 +226,58 @@ __device__ __forceinline__ void encode_group_fast(const float* v, const float4* 
     constexpr int NBG = GE / B;
     float t[GE];
 #pragma unroll
-    for (int j = 0; j < NBG; ++j)
-#pragma unroll
-        for (int i = 0; i < B; ++i)
-            t[j * B + i] = SHORTQ ? quotient_short(v[j * B + i], E[j].x, E[j].y) : quotient_corrected(v[j * B + i], E[j].x, E[j].y);
+    for (int j = 0; j < NBG; ++j) block_quotients<B, SHORTQ>(&v[j * B], E[j].x, E[j].y, &t[j * B]);
     pack_and_score<B, HALF>(v, t, E, packed, sse);
+}
+
+// Both 4-over-6 candidate sets of a group at once: quotients as above, FP4 pack / unpack per
+// candidate, and the two SSE chains of a block side by side in one fma.rn.f32x2 per element
+// (lane .x: the M = 6 candidate, lane .y: the M = 4 candidate; each lane sums its own residuals
+// in element order, exactly like the scalar chain).
+template <int B, bool SHORTQ, bool HALF>
+__device__ __forceinline__ void encode_group_fast_dual(const float* v, const float4* E6, const float4* E4, uint32_t* pk6,
+                                                       uint32_t* pk4, float* sse6, float* sse4) {
+    constexpr int GE = (B < 8) ? 8 : B;
+    constexpr int NBG = GE / B;
+    float t6[GE], t4[GE];
+#pragma unroll
+    for (int j = 0; j < NBG; ++j) {
+        block_quotients<B, SHORTQ>(&v[j * B], E6[j].x, E6[j].y, &t6[j * B]);
+        block_quotients<B, SHORTQ>(&v[j * B], E4[j].x, E4[j].y, &t4[j * B]);
+    }
+    uint32_t h6[GE / 2], h4[GE / 2];
+#pragma unroll
+    for (int k = 0; k < GE / 8; ++k) {
+        pk6[k] = quantize_e2m1x8_h(&t6[8 * k], &h6[4 * k]);
+        pk4[k] = quantize_e2m1x8_h(&t4[8 * k], &h4[4 * k]);
+    }
+#pragma unroll
+    for (int j = 0; j < NBG; ++j) {
+        float2 s = make_float2(0.0f, 0.0f);
+        const uint32_t nD6_16 = __float_as_uint(E6[j].z), nD4_16 = __float_as_uint(E4[j].z);
+        const float nD6 = -E6[j].x, nD4 = -E4[j].x;
+#pragma unroll
+        for (int i = 0; i < B; i += 2) {
+            const int e = j * B + i;
+            float a0, a1, b0, b1;   // residuals of elements e, e + 1 under candidate 6 (a) and 4 (b)
+            if constexpr (HALF) {
+                residual_pair_f16(h6[e / 2], nD6_16, v[e], v[e + 1], a0, a1);
+                residual_pair_f16(h4[e / 2], nD4_16, v[e], v[e + 1], b0, b1);
+            } else {
+                const float2 q6 = __half22float2(*reinterpret_cast<const __half2*>(&h6[e / 2]));
+                const float2 q4 = __half22float2(*reinterpret_cast<const __half2*>(&h4[e / 2]));
+                a0 = __fmaf_rn(q6.x, nD6, v[e]);
+                a1 = __fmaf_rn(q6.y, nD6, v[e + 1]);
+                b0 = __fmaf_rn(q4.x, nD4, v[e]);
+                b1 = __fmaf_rn(q4.y, nD4, v[e + 1]);
+            }
+            const float2 e0 = make_float2(a0, b0), e1 = make_float2(a1, b1);
+            s = __ffma2_rn(e0, e0, s);
+            s = __ffma2_rn(e1, e1, s);
+        }
+        sse6[j] = s.x;
+        sse4[j] = s.y;
+    }
 }
 
 // One candidate set of a group on the general path (IEEE division; zero scale -> signed zeros).
@@ -228,7 +297,8 @@ __device__ __forceinline__ void encode_group_general(const float* v, const float
 struct QuantConsts {
     float g, Rg;        // tensor scale and RN(1 / g)
     float m_lo, m_hi;   // a block maximum m takes the shortcuts when m == 0 or m_lo <= m <= m_hi
-    bool unit_g, need_lo, pz, all_short;
+    bool unit_g, need_lo, all_short;
+    int c_min;          // smallest admissible code: 1 under prevent-zero (FP8 formats), else 0
     int pow2_rule;      // kPow2Eq1 unless the format is UE8M0 and another rule was asked for
 };
 
@@ -270,13 +340,11 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             mmax = fmaxf(mmax, a);
             if (k.need_lo) mmin = fminf(mmin, a == 0.0f ? k.m_hi : a);
             u[j] = k.unit_g ? a : quotient_corrected(a, k.g, k.Rg);
-            c6[j] = target6_code<FMT, false>(u[j], k.pow2_rule);
-            if (k.pz) c6[j] = max(c6[j], 1);
+            c6[j] = max(target6_code<FMT, false>(u[j], k.pow2_rule), k.c_min);
+            if constexpr (DUAL) c4[j] = max(round_scale<FMT>(__fmul_rn(u[j], 0.25f)), k.c_min);
             E6[j] = T.E[c6[j]];
             wmin = fminf(wmin, E6[j].w);
             if constexpr (DUAL) {
-                c4[j] = round_scale<FMT>(__fmul_rn(u[j], 0.25f));
-                if (k.pz) c4[j] = max(c4[j], 1);
                 E4[j] = T.E[c4[j]];
                 wmin = fminf(wmin, E4[j].w);
             }
@@ -285,22 +353,22 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
         float sse[NBG], sse4[NBG];
         if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
             if (wmin >= 2.0f) {   // one decision for both candidates
-                encode_group_fast<B, SHORTQ, true>(v, E6, pk, sse);
-                if constexpr (DUAL) encode_group_fast<B, SHORTQ, true>(v, E4, pk4, sse4);
+                if constexpr (DUAL) encode_group_fast_dual<B, SHORTQ, true>(v, E6, E4, pk, pk4, sse, sse4);
+                else encode_group_fast<B, SHORTQ, true>(v, E6, pk, sse);
             } else {
-                encode_group_fast<B, SHORTQ, false>(v, E6, pk, sse);
-                if constexpr (DUAL) encode_group_fast<B, SHORTQ, false>(v, E4, pk4, sse4);
+                if constexpr (DUAL) encode_group_fast_dual<B, SHORTQ, false>(v, E6, E4, pk, pk4, sse, sse4);
+                else encode_group_fast<B, SHORTQ, false>(v, E6, pk, sse);
             }
         } else {
 #pragma unroll
             for (int j = 0; j < NBG; ++j) {
                 u[j] = __fdiv_rn(m[j], k.g);
                 c6[j] = target6_code<FMT, true>(u[j], k.pow2_rule);
-                if (k.pz) c6[j] = max(c6[j], 1);
+                c6[j] = max(c6[j], k.c_min);
                 E6[j] = T.E[c6[j]];
                 if constexpr (DUAL) {
                     c4[j] = round_scale<FMT>(__fmul_rn(u[j], 0.25f));
-                    if (k.pz) c4[j] = max(c4[j], 1);
+                    c4[j] = max(c4[j], k.c_min);
                     E4[j] = T.E[c4[j]];
                 }
             }
@@ -413,7 +481,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
     build_quant_tables<FMT>(T, k.g);
     k.unit_g = (k.g == 1.0f);
-    k.pz = p.prevent_zero && FMT != kUE8M0;
+    k.c_min = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     k.all_short = T.all_short != 0;
     k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;
     k.Rg = 1.0f;
