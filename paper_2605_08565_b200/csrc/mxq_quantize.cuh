@@ -160,8 +160,9 @@ __device__ __forceinline__ void widen(const uint32_t* w, float* v) {
     }
 }
 
-// Pack a group's quotients (GE / 8 code words) and accumulate the per-block SSE
-// (e = fma(-q, D, v); sse = fma(e, e, sse), in element order).
+// Pack a group's quotients (GE / 8 code words) and continue the per-block SSE chains from the
+// values in sse[] (e = fma(-q, D, v); sse = fma(e, e, sse), in element order): the caller starts
+// them at zero, and a block longer than a group is fed through in consecutive parts.
 template <int B, bool HALF>
 __device__ __forceinline__ void pack_and_score(const float* v, const float* t, const float4* E, uint32_t* packed,
                                                float* sse) {
@@ -172,7 +173,7 @@ __device__ __forceinline__ void pack_and_score(const float* v, const float* t, c
     for (int k = 0; k < GE / 8; ++k) packed[k] = quantize_e2m1x8_h(&t[8 * k], &h[4 * k]);
 #pragma unroll
     for (int j = 0; j < NBG; ++j) {
-        float s = 0.0f;
+        float s = sse[j];
         if constexpr (HALF) {
             const uint32_t nD16 = __float_as_uint(E[j].z);
 #pragma unroll
@@ -233,7 +234,7 @@ __device__ __forceinline__ void encode_group_fast(const float* v, const float4* 
 // Both 4-over-6 candidate sets of a group at once: quotients as above, FP4 pack / unpack per
 // candidate, and the two SSE chains of a block side by side in one fma.rn.f32x2 per element
 // (lane .x: the M = 6 candidate, lane .y: the M = 4 candidate; each lane sums its own residuals
-// in element order, exactly like the scalar chain).
+// in element order, exactly like the scalar chain).  The chains continue from sse6[] / sse4[].
 template <int B, bool SHORTQ, bool HALF>
 __device__ __forceinline__ void encode_group_fast_dual(const float* v, const float4* E6, const float4* E4, uint32_t* pk6,
                                                        uint32_t* pk4, float* sse6, float* sse4) {
@@ -253,7 +254,7 @@ __device__ __forceinline__ void encode_group_fast_dual(const float* v, const flo
     }
 #pragma unroll
     for (int j = 0; j < NBG; ++j) {
-        float2 s = make_float2(0.0f, 0.0f);
+        float2 s = make_float2(sse6[j], sse4[j]);
         const uint32_t nD6_16 = __float_as_uint(E6[j].z), nD4_16 = __float_as_uint(E4[j].z);
         const float nD6 = -E6[j].x, nD4 = -E4[j].x;
 #pragma unroll
@@ -351,6 +352,8 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
         }
         uint32_t pk[S::GE / 8], pk4[S::GE / 8];
         float sse[NBG], sse4[NBG];
+#pragma unroll
+        for (int j = 0; j < NBG; ++j) sse[j] = sse4[j] = 0.0f;
         if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
             if (wmin >= 2.0f) {   // one decision for both candidates
                 if constexpr (DUAL) encode_group_fast_dual<B, SHORTQ, true>(v, E6, E4, pk, pk4, sse, sse4);
@@ -439,6 +442,114 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
     if (p.block_sse) store_bytes<4 * S::NBC>(p.block_sse + chunk * S::NBC, sw);
 }
 
+// Blocks of 32 and 64 elements (chunk = one block).  The block is walked twice in parts of 16
+// elements read from the thread's ring slot, which stays valid until the next trip's request:
+// once for the block maximum, once for the encode with the SSE chains carried from part to part.
+// Only one part is live in registers at a time, which keeps as many CTAs resident as for B = 16.
+template <int DT, int B, int FMT, bool DUAL, bool SHORTQ, bool FAKE>
+__device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
+                                                    size_t chunk, const uint4* src) {
+    using S = QuantShape<DT, B>;
+    static_assert(S::C == B && S::NBC == 1, "one block per chunk");
+    constexpr int SG = 16;                        // elements per part
+    constexpr int NSG = B / SG;
+    constexpr int PPS = SG * S::EB / 16;          // 16-byte pieces per part
+    auto load_part = [&](int sg, float* v) {
+        uint32_t w[4 * PPS];
+#pragma unroll
+        for (int q = 0; q < PPS; ++q) {
+            const uint4 x = src[(sg * PPS + q) * kThreads];
+            w[4 * q + 0] = x.x; w[4 * q + 1] = x.y; w[4 * q + 2] = x.z; w[4 * q + 3] = x.w;
+        }
+        widen<DT, SG>(w, v);
+    };
+
+    float a = 0.0f;
+#pragma unroll
+    for (int sg = 0; sg < NSG; ++sg) {
+        float v[SG];
+        load_part(sg, v);
+#pragma unroll
+        for (int i = 0; i < SG; ++i) a = fmaxf(a, fabsf(v[i]));
+    }
+    float u = k.unit_g ? a : quotient_corrected(a, k.g, k.Rg);
+    int c6 = max(target6_code<FMT, false>(u, k.pow2_rule), k.c_min), c4 = 0;
+    float4 E6 = T.E[c6], E4 = E6;
+    float wmin = E6.w;
+    if constexpr (DUAL) {
+        c4 = max(round_scale<FMT>(__fmul_rn(u, 0.25f)), k.c_min);
+        E4 = T.E[c4];
+        wmin = fminf(wmin, E4.w);
+    }
+    const bool fast = wmin >= 1.0f && a <= k.m_hi && (a == 0.0f || a >= k.m_lo);
+    if (!fast) {
+        u = __fdiv_rn(a, k.g);
+        c6 = max(target6_code<FMT, true>(u, k.pow2_rule), k.c_min);
+        E6 = T.E[c6];
+        if constexpr (DUAL) {
+            c4 = max(round_scale<FMT>(__fmul_rn(u, 0.25f)), k.c_min);
+            E4 = T.E[c4];
+        }
+    }
+
+    uint32_t pk[B / 8], pk4[B / 8];
+    float sse = 0.0f, sse4 = 0.0f;
+#pragma unroll
+    for (int sg = 0; sg < NSG; ++sg) {
+        float v[SG];
+        load_part(sg, v);
+        uint32_t* o6 = &pk[sg * (SG / 8)];
+        uint32_t* o4 = &pk4[sg * (SG / 8)];
+        if (fast) {
+            if (wmin >= 2.0f) {
+                if constexpr (DUAL) encode_group_fast_dual<SG, SHORTQ, true>(v, &E6, &E4, o6, o4, &sse, &sse4);
+                else encode_group_fast<SG, SHORTQ, true>(v, &E6, o6, &sse);
+            } else {
+                if constexpr (DUAL) encode_group_fast_dual<SG, SHORTQ, false>(v, &E6, &E4, o6, o4, &sse, &sse4);
+                else encode_group_fast<SG, SHORTQ, false>(v, &E6, o6, &sse);
+            }
+        } else {
+            encode_group_general<SG>(v, &E6, o6, &sse);
+            if constexpr (DUAL) encode_group_general<SG>(v, &E4, o4, &sse4);
+        }
+    }
+    float Dw = E6.x;
+    if constexpr (DUAL) {
+        const bool take = sse4 < sse;
+        sse = take ? sse4 : sse;
+        c6 = take ? c4 : c6;
+        Dw = take ? E4.x : Dw;
+#pragma unroll
+        for (int i = 0; i < B / 8; ++i) pk[i] = take ? pk4[i] : pk[i];
+    }
+    if constexpr (FAKE) {   // fused fake-quantize: x_hat = fl32(grid(code) * D), optionally rounded to bf16
+        const size_t e0 = chunk * B;
+#pragma unroll
+        for (int w8 = 0; w8 < B / 8; ++w8) {
+            float q[8];
+            unpack_e2m1x8(pk[w8], q);
+            uint32_t o[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__fmul_rn(q[i], Dw));
+            if (p.xhat_dtype == kF32) {
+                store_bytes<32>(static_cast<float*>(p.xhat) + e0 + 8 * w8, o);
+            } else {
+                uint32_t h[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[2 * i]), __uint_as_float(o[2 * i + 1]));
+                    h[i] = *reinterpret_cast<const uint32_t*>(&b2);
+                }
+                store_bytes<16>(static_cast<__nv_bfloat16*>(p.xhat) + e0 + 8 * w8, h);
+            }
+        }
+        return;
+    }
+    store_bytes<B / 2>(p.codes + chunk * (B / 2), pk);
+    p.scales[chunk] = (uint8_t)c6;
+    if (p.block_sse) p.block_sse[chunk] = sse;
+}
+
 // Asynchronous copy of one chunk (PIECES x 16 bytes) from global memory into this thread's pieces
 // of a ring slot (piece k of thread t at ((slot * PIECES + k) * 256 + t) * 16), as one commit
 // group.  An empty group is committed when there is no chunk left, so that the group count per
@@ -510,21 +621,29 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     for (; chunk < p.n_items; chunk += stride) {
         // all but the DIST - 1 most recent groups are complete: this thread's copy of `chunk` has landed
         asm volatile("cp.async.wait_group %0;" ::"n"(DIST - 1) : "memory");
-        uint32_t raw[S::PIECES * 4];
         const uint4* src = ring + (size_t)slot * (S::PIECES * kThreads) + threadIdx.x;
-#pragma unroll
-        for (int q = 0; q < S::PIECES; ++q) {
-            const uint4 w = src[q * kThreads];
-            raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
-        }
         // the slot read one trip ago is free again (its words were consumed by the arithmetic of
-        // that trip): request the chunk DIST trips ahead into it
+        // that trip): request the chunk DIST trips ahead into it.  The slot of the current chunk
+        // is not requested into before the next trip, so it may be read throughout this one.
         stage_chunk<S::PIECES>(ring_base + fill * kSlotBytes, x + ahead * kChunkBytes, ahead < p.n_items);
         ahead += stride;
         slot = (slot + 1 == S::SLOTS) ? 0 : slot + 1;
         fill = (fill + 1 == S::SLOTS) ? 0 : fill + 1;
-        if (k.all_short) quantize_chunk<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, raw);
-        else quantize_chunk<DT, B, FMT, DUAL, false, FAKE>(p, T, k, chunk, raw);
+        // blocks longer than 16 elements go part by part, except 4-over-6 at B = 32, which measured
+        // slightly faster with the whole block in registers
+        if constexpr (B > 16 && !(DUAL && B == 32)) {
+            if (k.all_short) quantize_long_block<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, src);
+            else quantize_long_block<DT, B, FMT, DUAL, false, FAKE>(p, T, k, chunk, src);
+        } else {
+            uint32_t raw[S::PIECES * 4];
+#pragma unroll
+            for (int q = 0; q < S::PIECES; ++q) {
+                const uint4 w = src[q * kThreads];
+                raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
+            }
+            if (k.all_short) quantize_chunk<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, raw);
+            else quantize_chunk<DT, B, FMT, DUAL, false, FAKE>(p, T, k, chunk, raw);
+        }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
