@@ -135,6 +135,7 @@ struct QuantShape {
     static constexpr int NBC = C / B;                        // blocks per chunk
     static constexpr int PIECES = C * EB / 16;               // 16-byte pieces per chunk
     static constexpr int SLOTS = 2;                          // ring depth per thread
+    static constexpr bool COOP = PIECES > 4;                 // chunk above 64 bytes: the warp copies its chunks together
     static constexpr size_t RING_BYTES = (size_t)SLOTS * PIECES * 16 * kThreads;
 };
 
@@ -442,13 +443,22 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
     if (p.block_sse) store_bytes<4 * S::NBC>(p.block_sse + chunk * S::NBC, sw);
 }
 
+// Position (in 16-byte units, relative to the warp's first column of a ring slot) of piece k of
+// the chunk that lane `lane` works on.  Thread-private staging: row k, the thread's own column.
+// Cooperative staging: row k, column lane ^ k, so that both the warp's copies (which write many
+// rows of a few columns at once) and its later reads (one row, all columns) spread over all banks.
+template <bool COOP>
+__device__ __forceinline__ int ring_index(int k, int lane) {
+    return k * kThreads + (COOP ? (lane ^ k) : lane);
+}
+
 // Blocks of 32 and 64 elements (chunk = one block).  The block is walked twice in parts of 16
 // elements read from the thread's ring slot, which stays valid until the next trip's request:
 // once for the block maximum, once for the encode with the SSE chains carried from part to part.
 // Only one part is live in registers at a time, which keeps as many CTAs resident as for B = 16.
 template <int DT, int B, int FMT, bool DUAL, bool SHORTQ, bool FAKE>
 __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
-                                                    size_t chunk, const uint4* src) {
+                                                    size_t chunk, const uint4* slot_warp, int lane) {
     using S = QuantShape<DT, B>;
     static_assert(S::C == B && S::NBC == 1, "one block per chunk");
     constexpr int SG = 16;                        // elements per part
@@ -458,7 +468,7 @@ __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const Qu
         uint32_t w[4 * PPS];
 #pragma unroll
         for (int q = 0; q < PPS; ++q) {
-            const uint4 x = src[(sg * PPS + q) * kThreads];
+            const uint4 x = slot_warp[ring_index<S::COOP>(sg * PPS + q, lane)];
             w[4 * q + 0] = x.x; w[4 * q + 1] = x.y; w[4 * q + 2] = x.z; w[4 * q + 3] = x.w;
         }
         widen<DT, SG>(w, v);
@@ -550,6 +560,29 @@ __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const Qu
     if (p.block_sse) p.block_sse[chunk] = sse;
 }
 
+// Cooperative staging for chunks above 64 bytes.  With thread-private copies every 16-byte piece
+// of such a chunk lies in a cache line of its own lane, and one copy instruction of a warp touches
+// 32 lines for 512 bytes; the L1 tag rate then caps the kernel near two thirds of the HBM
+// bandwidth.  Here the warp copies its 32 consecutive chunks as one contiguous region instead:
+// instruction i moves pieces 32 i .. 32 i + 31 of the region (512 contiguous bytes, 4 lines), lane
+// l the piece 32 i + l, which is piece (32 i + l) % PIECES of the chunk of lane (32 i + l) / PIECES.
+// The data then crosses lanes, so the consumer waits for its own copies and joins a __syncwarp()
+// (every lane of the warp takes every trip of the loop).  wchunk: chunk of lane 0.
+template <int PIECES>
+__device__ __forceinline__ void stage_warp_chunks(uint32_t slot_warp_addr, const char* x, size_t chunk_bytes, size_t wchunk,
+                                                  size_t n_chunks, int lane) {
+#pragma unroll
+    for (int i = 0; i < PIECES; ++i) {
+        const int piece = i * 32 + lane;
+        const int owner = piece / PIECES, k = piece % PIECES;
+        if (wchunk + owner < n_chunks)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(slot_warp_addr + ring_index<true>(k, owner) * 16),
+                         "l"(x + wchunk * chunk_bytes + (size_t)piece * 16)
+                         : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
 // Asynchronous copy of one chunk (PIECES x 16 bytes) from global memory into this thread's pieces
 // of a ring slot (piece k of thread t at ((slot * PIECES + k) * 256 + t) * 16), as one commit
 // group.  An empty group is committed when there is no chunk left, so that the group count per
@@ -574,17 +607,22 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     wait_for_prior_grid();
     // request the first chunks before anything else: their latency hides behind the table build
     const size_t stride = (size_t)gridDim.x * kThreads;
+    const int lane = threadIdx.x & 31;
     size_t chunk = (size_t)blockIdx.x * kThreads + threadIdx.x;
+    const size_t wchunk0 = chunk - lane;   // chunk of the warp's lane 0
     constexpr size_t kChunkBytes = (size_t)S::C * S::EB;
     constexpr uint32_t kSlotBytes = S::PIECES * kThreads * 16;
     constexpr int DIST = S::SLOTS - 1;   // chunks requested ahead of the one being processed
-    const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(ring) + threadIdx.x * 16;
+    // first column of this warp in slot 0; a thread's own column is `lane` further
+    const uint32_t ring_warp = (uint32_t)__cvta_generic_to_shared(ring) + (threadIdx.x - lane) * 16;
+    const uint32_t ring_base = ring_warp + lane * 16;
     const char* x = static_cast<const char*>(p.x);
     {
-        size_t c = chunk;
+        size_t c = S::COOP ? wchunk0 : chunk;
 #pragma unroll
         for (int d = 0; d < DIST; ++d) {
-            stage_chunk<S::PIECES>(ring_base + d * kSlotBytes, x + c * kChunkBytes, c < p.n_items);
+            if constexpr (S::COOP) stage_warp_chunks<S::PIECES>(ring_warp + d * kSlotBytes, x, kChunkBytes, c, p.n_items, lane);
+            else stage_chunk<S::PIECES>(ring_base + d * kSlotBytes, x + c * kChunkBytes, c < p.n_items);
             c += stride;
         }
     }
@@ -614,31 +652,38 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
         k.m_lo = 0.0f;
     }
 
-    if (chunk >= p.n_items) return;   // no barrier follows
+    // Thread-private staging: a thread leaves when its chunks are done (no barrier follows).
+    // Cooperative staging: the warp stays together, lanes past the end only take part in the copies.
+    if ((S::COOP ? wchunk0 : chunk) >= p.n_items) return;
     int slot = 0;                      // slot holding `chunk`
     int fill = DIST % S::SLOTS;        // slot that the next request goes to
-    size_t ahead = chunk + (size_t)DIST * stride;
-    for (; chunk < p.n_items; chunk += stride) {
-        // all but the DIST - 1 most recent groups are complete: this thread's copy of `chunk` has landed
+    size_t ahead = (S::COOP ? wchunk0 : chunk) + (size_t)DIST * stride;
+    for (size_t lead = S::COOP ? wchunk0 : chunk; lead < p.n_items; lead += stride, chunk += stride) {
+        // all but the DIST - 1 most recent groups are complete: this thread's copies for `chunk` have landed
         asm volatile("cp.async.wait_group %0;" ::"n"(DIST - 1) : "memory");
-        const uint4* src = ring + (size_t)slot * (S::PIECES * kThreads) + threadIdx.x;
+        // cooperative staging: so have the other lanes' copies, and every lane is done reading the
+        // slot that the next request overwrites
+        if constexpr (S::COOP) __syncwarp();
+        const uint4* slot_warp = ring + (size_t)slot * (S::PIECES * kThreads) + (threadIdx.x - lane);
         // the slot read one trip ago is free again (its words were consumed by the arithmetic of
         // that trip): request the chunk DIST trips ahead into it.  The slot of the current chunk
         // is not requested into before the next trip, so it may be read throughout this one.
-        stage_chunk<S::PIECES>(ring_base + fill * kSlotBytes, x + ahead * kChunkBytes, ahead < p.n_items);
+        if constexpr (S::COOP) stage_warp_chunks<S::PIECES>(ring_warp + fill * kSlotBytes, x, kChunkBytes, ahead, p.n_items, lane);
+        else stage_chunk<S::PIECES>(ring_base + fill * kSlotBytes, x + ahead * kChunkBytes, ahead < p.n_items);
         ahead += stride;
         slot = (slot + 1 == S::SLOTS) ? 0 : slot + 1;
         fill = (fill + 1 == S::SLOTS) ? 0 : fill + 1;
+        if (S::COOP && chunk >= p.n_items) continue;   // a lane past the end (the warp's last trip)
         // blocks longer than 16 elements go part by part, except 4-over-6 at B = 32, which measured
         // slightly faster with the whole block in registers
         if constexpr (B > 16 && !(DUAL && B == 32)) {
-            if (k.all_short) quantize_long_block<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, src);
-            else quantize_long_block<DT, B, FMT, DUAL, false, FAKE>(p, T, k, chunk, src);
+            if (k.all_short) quantize_long_block<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, slot_warp, lane);
+            else quantize_long_block<DT, B, FMT, DUAL, false, FAKE>(p, T, k, chunk, slot_warp, lane);
         } else {
             uint32_t raw[S::PIECES * 4];
 #pragma unroll
             for (int q = 0; q < S::PIECES; ++q) {
-                const uint4 w = src[q * kThreads];
+                const uint4 w = slot_warp[ring_index<S::COOP>(q, lane)];
                 raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
             }
             if (k.all_short) quantize_chunk<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, raw);
