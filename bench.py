@@ -50,10 +50,10 @@ STREAM_ELEMS = 1 << 27            # tensor size of the streaming (HBM-bound) ker
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (same kernel build, same launch configuration); set an entry to None when its kernel changes.
 NCU_TRAFFIC_BYTES = {
-    "k_brute<bf16,B=16,UE4M3>@16Mi": 33.620480e6 + 11.776e3,
-    "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.498432e6 + 81.372672e6,
-    "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi": 268.504320e6 + 82.705408e6,
-    "k_quantize<f32,B=16,UE4M3,absmax>@128Mi": 536.908032e6 + 94.972672e6,
+    "k_brute<bf16,B=16,UE4M3>@16Mi": 33.620480e6 + 5.12e3,
+    "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.525568e6 + 80.861440e6,
+    "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi": 268.531712e6 + 83.055104e6,
+    "k_quantize<f32,B=16,UE4M3,absmax>@128Mi": 536.924672e6 + 96.008192e6,
 }
 
 
