@@ -5,26 +5,30 @@
 // Work layout.  One thread owns a chunk of consecutive elements (at least 64 bytes of input and
 // at least one block) and walks it in groups of max(B, 8) elements (one block, or 8/B small
 // blocks), so every per-block quantity lives in registers and the SSE is accumulated in element
-// order.  CTAs are persistent (grid = SMs x resident CTAs) and build the per-code table once.
+// order.  Blocks of 32 and 64 elements are walked in parts of 16 (quantize_long_block()).  CTAs
+// are persistent (grid = SMs x resident CTAs) and build the per-code table once.
 //
-// Input staging.  Every thread copies ITS OWN next chunk into ITS OWN slot of a two-slot
-// shared-memory ring with asynchronous 16-byte copies (cp.async.ca: the 128-byte line that the
-// first piece brings into L1 also serves the thread's other pieces and its neighbour) and waits
-// for it with cp.async.wait_group.  The data never crosses threads, so no barrier of any kind is
-// involved and nothing can wait forever.  One chunk (>= 64 bytes) per thread is in flight while
-// the current one is processed, independent of how many registers the arithmetic needs; a third
-// slot was measured and loses (the extra shared memory leaves too little L1 for fp32 input).
-// Slot layout: piece k of thread t sits at ((slot * PIECES + k) * 256 + t) * 16, so both the
-// asynchronous writes and the later 128-bit reads of a warp are contiguous (no bank conflict).
+// Input staging, chunks of 64 bytes.  Every thread copies ITS OWN next chunk into ITS OWN column
+// of a two-slot shared-memory ring with asynchronous 16-byte copies (cp.async.ca: the 128-byte
+// line that the first piece brings into L1 also serves the thread's other pieces and its
+// neighbour) and waits for it with cp.async.wait_group.  The data never crosses threads, so no
+// barrier of any kind is involved and nothing can wait forever.  One chunk per thread is in
+// flight while the current one is processed, independent of how many registers the arithmetic
+// needs; a third slot was measured and loses (the extra shared memory leaves too little L1 for
+// fp32 input).  Slot layout: piece k of thread t sits at ((slot * PIECES + k) * 256 + t) * 16, so
+// both the asynchronous writes and the later 128-bit reads of a warp are contiguous (no bank
+// conflict).  Chunks above 64 bytes are copied by the warp together (stage_warp_chunks()) and
+// handed over with a __syncwarp().
 //
-// Arithmetic per element (the instruction mix that the issue slots of an SM sub-partition bound):
-// bf16 -> binary32 by a mixed-precision add of -0 (FMA pipe), the exact quotient by the decode
-// scale (reciprocal multiply + one residual correction when every decode scale of the table has a
-// short significand, two corrections otherwise), half an FP4 pack, half an FP4 unpack, and the two
-// FMAs of the SSE -- the first being fma.rn.f32.f16 straight from the unpacked f16 grid value
-// whenever the decode scales of the group are exactly representable in f16 (always, for UE4M3
-// without a tensor scale), else an f16->f32 convert plus an FFMA.  Blocks whose numbers fall
-// outside the ranges these shortcuts need are redone with IEEE divisions (general path).
+// Arithmetic per element (kernel time follows the number of warp instructions): bf16 -> binary32
+// by a mixed-precision add of -0 (FMA pipe); the exact quotient by the decode scale, two elements
+// per instruction (reciprocal multiply + one residual correction when every decode scale of the
+// table has a short significand, two corrections otherwise); half an FP4 pack, half an FP4
+// unpack; the residual as fma.rn.f32.f16 straight from the unpacked f16 grid value whenever the
+// decode scales of the group are exactly representable in f16 (always, for UE4M3 without a tensor
+// scale), else an f16->f32 convert plus an FFMA; the square-accumulate FMA, for 4-over-6 one
+// fma.rn.f32x2 serving both candidates.  Blocks whose numbers fall outside the ranges these
+// shortcuts need are redone with IEEE divisions (general path).
 #pragma once
 
 #include <cuda_bf16.h>
