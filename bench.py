@@ -49,6 +49,8 @@ REFERENCE_BUDGET_S = 35.0        # wall-clock target of a whole --impl reference
 STREAM_ELEMS = 1 << 27            # tensor size of the streaming (HBM-bound) kernel measurements
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (same kernel build, same launch configuration); set an entry to None when its kernel changes.
+# smsp__issue_active.avg.pct_of_peak_sustained_active of the brute-force kernel in the same capture
+NCU_BRUTE_ISSUE_ACTIVE_PCT = 70.2
 NCU_TRAFFIC_BYTES = {
     "k_brute<bf16,B=16,UE4M3>@16Mi": 33.620480e6 + 5.12e3,
     "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.525568e6 + 80.861440e6,
@@ -429,7 +431,7 @@ def run_gpu(args) -> None:
                 "traffic": NCU_TRAFFIC_BYTES["k_brute<bf16,B=16,UE4M3>@16Mi"],
                 "peak_source": f"{n_sm} SMs x 128 lanes x {peaks['sm_max_mhz']:.0f} MHz (max SM clock, {peaks['source']})",
                 "frac_at_observed_clock": brute_ach / (n_sm * ALU_LANES_PER_SM * sm_mhz * 1e6 / 1e12),
-                "ms_per_launch": brute_ms}
+                "ms_per_launch": brute_ms, "ncu_issue_active_pct": NCU_BRUTE_ISSUE_ACTIVE_PCT}
     hbm = {}
     for name, key in (("absmax_B16", (16, ABSMAX)), ("4o6_B16", (16, R4O6))):
         ms = wl.kernel_ms(key)
