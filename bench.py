@@ -269,13 +269,8 @@ def streaming_rooflines(torch, mxq, device, peaks):
     from paper_2605_08565_b200 import inputs
     out = {}
     n = STREAM_ELEMS
-    codes, scales, sse = mxq.alloc_outputs(n, 16, device)
-    for name, dt, recipe, key in (
-            ("absmax_bf16_B16", torch.bfloat16, ABSMAX, "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi"),
-            ("4o6_bf16_B16", torch.bfloat16, R4O6, "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi"),
-            ("absmax_f32_B16", torch.float32, ABSMAX, "k_quantize<f32,B=16,UE4M3,absmax>@128Mi")):
-        x = inputs.student_t(n, 5, 0.02, 2, dt, device)
-        fn = lambda: mxq.mxq_quantize_ex(x, n, 16, UE4M3, recipe, 1.0, None, codes, scales, sse)
+
+    def entry(name, fn, nbytes, traffic):
         for _ in range(3):
             fn()
         times = []
@@ -288,12 +283,32 @@ def streaming_rooflines(torch, mxq, device, peaks):
             torch.cuda.synchronize()
             times.append(e0.elapsed_time(e1) / 10)
         ms = statistics.median(times)
-        ach = algorithmic_bytes(n, x.element_size(), 16) / (ms * 1e-3) / 1e9
+        ach = nbytes / (ms * 1e-3) / 1e9
         out[name] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0,
-                     "traffic": NCU_TRAFFIC_BYTES[key], "ms_per_launch": ms, "gelem_s": n / (ms * 1e-3) / 1e9,
-                     "elems": n, "peak_source": peaks["source"], "l2": "input larger than L2"}
+                     "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0, "traffic": traffic,
+                     "ms_per_launch": ms, "gelem_s": n / (ms * 1e-3) / 1e9, "elems": n,
+                     "peak_source": peaks["source"], "l2": "input larger than L2"}
+
+    for name, dt, recipe, B, key in (
+            ("absmax_bf16_B16", torch.bfloat16, ABSMAX, 16, "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi"),
+            ("4o6_bf16_B16", torch.bfloat16, R4O6, 16, "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi"),
+            ("absmax_f32_B16", torch.float32, ABSMAX, 16, "k_quantize<f32,B=16,UE4M3,absmax>@128Mi"),
+            ("4o6_f32_B16", torch.float32, R4O6, 16, None),
+            ("absmax_bf16_B64", torch.bfloat16, ABSMAX, 64, None),
+            ("absmax_f32_B64", torch.float32, ABSMAX, 64, None)):
+        codes, scales, sse = mxq.alloc_outputs(n, B, device)
+        x = inputs.student_t(n, 5, 0.02, 2, dt, device)
+        fn = lambda: mxq.mxq_quantize_ex(x, n, B, UE4M3, recipe, 1.0, None, codes, scales, sse)
+        entry(name, fn, algorithmic_bytes(n, x.element_size(), B), NCU_TRAFFIC_BYTES[key] if key else None)
         del x
+    # the other two kernels of the path: tensor abs-max (reads n elements) and de-quantization
+    x = inputs.student_t(n, 5, 0.02, 2, torch.bfloat16, device)
+    amax = torch.empty(1, dtype=torch.float32, device=device)
+    entry("tensor_amax_bf16", lambda: mxq.mxq_tensor_amax(x, n, amax), n * 2.0, None)
+    codes, scales, sse = mxq.alloc_outputs(n, 16, device)
+    mxq.mxq_quantize_ex(x, n, 16, UE4M3, ABSMAX, 1.0, None, codes, scales, sse)
+    xh = torch.empty(n, dtype=torch.float32, device=device)
+    entry("dequantize_B16_to_f32", lambda: mxq.mxq_dequantize(codes, scales, n, 16, UE4M3, 1.0, xh), n * (0.5 + 1.0 / 16 + 4.0), None)
     return out
 
 
