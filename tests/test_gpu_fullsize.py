@@ -200,3 +200,39 @@ def test_bulk_brute_force_16384x16384_fp32_laplace_with_tensor_scale(laplace_163
             assert prev <= m * (1 + 1e-6)
         prev = m
         del codes, scales, sse
+
+
+def test_more_than_two_to_the_32_elements():
+    """A tensor whose element index, byte offsets and block count need more than 32 bits where they
+    are formed (2^32 + 3 * 2^20 bf16 elements, 8.6 GB): one-pass recipes, brute force, tensor abs-max,
+    tensor MSE and de-quantization, compared with the oracle on the first and last blocks and on random ones."""
+    n = (1 << 32) + (3 << 20)
+    B, fmt = 16, mxq.MXQ_SF_UE4M3
+    x = inputs.student_t(n, 5, 0.02, 99, torch.bfloat16, "cuda")
+    x[-5] = 96.0                                       # the tensor maximum sits beyond element 2^32
+    amax = torch.empty(1, dtype=torch.float32, device="cuda")
+    mxq.mxq_tensor_amax(x, n, amax)
+    torch.cuda.synchronize()
+    assert float(amax.cpu()[0]) == 96.0 == float(x.abs().max().float().cpu())
+    codes, scales, sse = mxq.alloc_outputs(n, B, "cuda")
+    for recipe in (ABSMAX, R4O6):
+        mxq.mxq_quantize_ex(x, n, B, fmt, recipe, 1.0, None, codes, scales, sse)
+        torch.cuda.synchronize()
+        _check_sampled(x, B, fmt, recipe, 1.0, codes, scales, sse, 4000, 4242 + recipe)
+        got = float(mxq.tensor_mse(sse, n).cpu()[0])
+        want = sum(float(part.double().sum().cpu()) for part in sse.split(1 << 26)) / n
+        assert abs(got - want) <= 1e-6 * want
+    # brute force at this size, both sweeps
+    mxq.mxq_quantize_ex(x, n, B, fmt, BRUTE, 1.0, None, codes, scales, sse)
+    torch.cuda.synchronize()
+    _check_sampled(x, B, fmt, BRUTE, 1.0, codes, scales, sse, 1500, 4250)
+    _pruned_sweep_equals(x, B, fmt, BRUTE, 1.0, None, codes, scales, sse)
+    xh = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    mxq.mxq_dequantize(codes, scales, n, B, fmt, 1.0, xh)
+    torch.cuda.synchronize()
+    idx = _sample_blocks(n // B, 3000, 17)
+    t_idx = torch.from_numpy(idx).cuda()
+    want = orc.dequantize(codes.view(-1, B // 2)[t_idx].cpu().numpy().reshape(-1), scales[t_idx].cpu().numpy(), idx.size * B,
+                          B, orc.UE4M3, 1.0, orc.BF16)
+    got = inputs.to_numpy_bits(xh.view(-1, B)[t_idx].contiguous())
+    assert np.array_equal(got, want.view(np.uint16))
