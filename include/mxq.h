@@ -112,9 +112,8 @@ int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scal
 
 /*
  * mxq_fake_quantize -- quantize and de-quantize in one pass: out_i = fl32(grid(code_i) * D_b), the
- * values a model computes with when its MLP weights or activations are held in this format
- * (Results, downstream experiments: "applying these scaling methods to the weight and activation
- * quantization").  Bit-identical to mxq_quantize_ex followed by mxq_dequantize, without writing
+ * values a model computes with when its MLP weights or activations are held in this format (the
+ * setting of the downstream experiments in Results).  Bit-identical to mxq_quantize_ex followed by mxq_dequantize, without writing
  * codes, scales or SSE.
  *   x, dtype, n, block_size, scale_fmt, global_scale, d_global_scale, cuda_stream   as for mxq_quantize_ex.
  *   recipe     any recipe except the brute-force ones (MXQ_ERR_BAD_ENUM for those: run mxq_quantize_ex
@@ -126,8 +125,8 @@ int mxq_fake_quantize(const void* x, int dtype, size_t n, int block_size, int sc
                       float global_scale, const float* d_global_scale, void* d_out, int out_dtype, void* cuda_stream);
 
 /*
- * mxq_tensor_amax -- first stage of hierarchical scaling (Experimental Setup, "a per-tensor scale
- * is first identified using the abs-max across the entire tensor").
+ * mxq_tensor_amax -- first stage of hierarchical scaling (Experimental Setup): the largest magnitude
+ * of the whole tensor, from which the per-tensor scale is derived.
  *   d_out_amax  device, one float: max_i |x_i| (0 for an all-zero tensor).
  *   d_out_global_scale  device, one float, or NULL: receives g = amax / (6*448) computed in
  *               binary32 (1 if amax == 0), ready to be passed as d_global_scale.
@@ -176,7 +175,7 @@ int mxq_tensor_mse(const float* d_block_sse, size_t n_blocks, size_t n, double* 
 int mxq_tensor_mse_static(const float* d_block_sse, size_t n_blocks, size_t n, double* d_out_mse, void* cuda_stream);
 
 /*
- * mxq_dequantize -- "de-quantization simply multiplies by S" (Experimental Setup):
+ * mxq_dequantize -- de-quantization, a multiplication by the scale (Experimental Setup):
  * out_i = fl32(grid(code_i) * D_b), D_b = fl32(S_b * g); MXQ_BF16 output rounds that to bf16 (RNE).
  *   d_codes  n/2 bytes;  d_scales  n/block_size bytes;  d_out  n elements of out_dtype.
  * A scale byte that is not a finite code of the format decodes as NaN.
@@ -224,8 +223,8 @@ int mxq_segment_mse(const float* d_block_sse, size_t n_blocks, size_t blocks_per
                     double* d_out_mse, void* cuda_stream);
 
 /*
- * mxq_mask_interval -- the pre-quantization diagnostic of the appendix ("masking specific magnitude
- * intervals to zero" at full precision): out_i = 0 when lo <= |x_i| < hi, else x_i.
+ * mxq_mask_interval -- the pre-quantization diagnostic of the appendix (entries whose magnitude lies
+ * in a chosen interval are zeroed at full precision): out_i = 0 when lo <= |x_i| < hi, else x_i.
  *   x, d_out   device, n elements of dtype (MXQ_F32 or MXQ_BF16); d_out may be x (in place).
  *   lo, hi     0 <= lo <= hi, else MXQ_ERR_BAD_SCALE.  NaN entries pass unchanged.
  */

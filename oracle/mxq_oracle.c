@@ -186,8 +186,8 @@ float mxq_oracle_block_sse(const float *v, int B, int fmt, int code, float g, ui
 }
 
 /* Eq. 2 candidate for divisor M (6 = standard abs-max, 4 = the second 4-over-6 candidate), with
- * the optional Eq. 3 clamp.  Hierarchical scaling: the block target is found "after adjusting the
- * inputs using the global scale", i.e. from amax / g. */
+ * the optional Eq. 3 clamp.  Hierarchical scaling: the block scale is chosen for inputs already
+ * divided by the tensor scale, i.e. the target comes from amax / g. */
 static int absmax_code(float amax, float g, float M, int fmt, int prevent_zero)
 {
     float u = amax / g;
@@ -368,7 +368,7 @@ double mxq_oracle_tensor_mse(const float *block_sse, size_t n_blocks, size_t n)
     return s / (double)n;
 }
 
-/* De-quantization "simply multiplies by S": x_hat = fl32(grid(code) * D), D = fl32(S * g).
+/* De-quantization is a multiplication by the scale: x_hat = fl32(grid(code) * D), D = fl32(S * g).
  * out_dtype ORC_BF16 additionally rounds x_hat to bf16 (RNE). */
 int mxq_oracle_dequantize(const uint8_t *codes, const uint8_t *scales, size_t n, int B, int fmt, float g, void *out,
                           int out_dtype)

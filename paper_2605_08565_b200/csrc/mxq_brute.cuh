@@ -1,6 +1,6 @@
-// Brute-force scale search (Experimental Setup: "a brute-force search over possible scaling
-// factors to minimize the MSE"): every finite scale code of the format is tried on every block and
-// the code with the smallest SSE is kept (equal SSE: the smaller code).
+// Brute-force scale search (Experimental Setup: the optimal baseline, found by trying the possible
+// scale values and keeping the one with the least error): every finite scale code of the format
+// is tried on every block and the code with the smallest SSE is kept (equal SSE: the smaller code).
 //
 // Work layout.  A thread keeps its elements in registers as float pairs and the candidate loop
 // works on float pairs with the packed binary32 instructions of sm_100 (fma.rn.f32x2 /

@@ -93,7 +93,7 @@ def test_element_rounding_is_nearest_point_for_unit_global_scale():
 # Special cases with a closed form
 # ------------------------------------------------------------------------------------------------
 def test_zero_scale_sets_everything_to_zero():
-    # "all values are set to zero": magnitudes 0, signs kept, SSE = sum v^2 in element order
+    # a zero scale sends every value to zero: magnitudes 0, signs kept, SSE = sum v^2 in element order
     x = np.array([1e-3, -2e-3, 3e-4, -0.0, 5e-3, -4e-3, 1e-5, 2e-3], dtype=f32)
     codes, scales, sse = orc.quantize(x, 8, orc.UE4M3, orc.ABSMAX)
     assert scales[0] == 0
@@ -179,7 +179,7 @@ def test_prevent_zero_never_hurts_and_only_touches_zero_scales(fmt):
 
 def test_finer_is_better_for_the_brute_force_optimum():
     # Children may reuse the parent's scale, so the optimum cannot get worse when a block is split
-    # (Results: "the optimal MSE monotonically increases with larger block sizes").
+    # (Results: with the optimal scale the MSE grows monotonically with the block size).
     for seed, sigma in ((1, 0.004), (2, 0.02), (3, 1.0)):
         x = inputs.normal(2048, seed, sigma).numpy()
         prev = None
@@ -358,8 +358,8 @@ def test_elements_next_to_a_midpoint_follow_one_division_by_the_decode_scale(g):
 
 @pytest.mark.parametrize("g", [0.0371, 1.0 / 3.0, 0.7, 1.9e-3])
 def test_block_maxima_next_to_a_scale_midpoint_follow_two_divisions(g):
-    # Eq. 2 under a tensor scale: the target is fl(fl(amax / g) / M), "after adjusting the inputs using
-    # the global scale"; a single division by fl(g * M) picks the neighbouring scale code for some of
+    # Eq. 2 under a tensor scale: the target is fl(fl(amax / g) / M), the block scale being chosen for
+    # inputs already divided by the tensor scale; a single division by fl(g * M) picks the neighbouring scale code for some of
     # these maxima (the last assertion makes sure such maxima are among them).
     tab = ex.ue4m3_table()
     differ = 0

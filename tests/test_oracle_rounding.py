@@ -46,7 +46,7 @@ def test_e2m1_rounding_equals_ml_dtypes_cast():
 
 
 # ------------------------------------------------------------------------------------------------
-# Round_SF for the FP8 scale formats (Eq. 2: "rounding and clipping", round-to-nearest-even)
+# Round_SF for the FP8 scale formats (Eq. 2: rounded to nearest even and clipped to the format's range)
 # ------------------------------------------------------------------------------------------------
 def _boundary_points(fmt):
     tab = ex.TABLES[fmt]()
