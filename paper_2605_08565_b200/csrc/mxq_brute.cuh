@@ -5,8 +5,8 @@
 // Work layout.  A thread keeps its elements in registers as float pairs and the candidate loop
 // works on float pairs with the packed binary32 instructions of sm_100 (fma.rn.f32x2 /
 // mul.rn.f32x2, FP4 pack and unpack two at a time):
-//   B <= 16   the thread owns 32 consecutive elements, pair i = (element i, element 16 + i): the
-//             two halves of a pair belong to different blocks, so one instruction serves two
+//   B <= 16   the thread owns G = 32 consecutive elements (16 for B = 2), pair i = (element i,
+//             element G/2 + i): the two halves of a pair belong to different blocks, so one instruction serves two
 //             elements of one candidate and the two SSE chains are independent.  Two candidates
 //             per trip.
 //   B >= 32   the thread owns one block, pair i = (element 2i, element 2i + 1).  Its SSE is one
@@ -425,12 +425,17 @@ __device__ __forceinline__ void search_list(const BruteTables& T, int list, int 
 // Resident CTAs per SM asked of the register allocator: two where measurement showed that the
 // second CTA outweighs the few spills it costs (B = 4; every B up to 32 with the pruned sweep),
 // else no constraint beyond one CTA.
+// Elements a thread of k_brute owns: one block for B >= 32, else 32; 16 for B = 2, whose 16
+// running minima per 32 elements otherwise leave room for one CTA per SM only (measured: 496 -> 452 us;
+// B = 4 and B = 8 lose with 16).
+__host__ __device__ constexpr int brute_group_elems(int B) { return B >= 32 ? B : (B == 2 ? 16 : 32); }
+
 constexpr int brute_min_ctas(int B, bool prune) { return (B == 4 || (B <= 32 && prune)) ? 2 : 1; }
 
 template <int DT, int B, int FMT, bool PRUNE>
 __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(QuantArgs p) {
     constexpr bool ONEBLK = (B >= 32);        // the thread owns exactly one block
-    constexpr int G = ONEBLK ? B : 32;          // elements per thread
+    constexpr int G = brute_group_elems(B);     // elements per thread
     constexpr int NP = G / 2;                 // pairs per thread
     constexpr int BL = ONEBLK ? NP : B;         // elements of one block inside one half
     constexpr int NBL = NP / BL;              // blocks per half (1 when ONEBLK)
@@ -769,7 +774,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
 }
 
 // ------------------------------------------------------------------------------------------------
-// The blocks past the last whole 32-element group (block sizes up to 16 only): one block per
+// The blocks past the last whole per-thread group (block sizes up to 16 only): one block per
 // thread, general path.
 // ------------------------------------------------------------------------------------------------
 template <int DT, int B, int FMT>
@@ -823,7 +828,7 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
         if (err != cudaSuccess) return err;
         ctas_per_sm[dev] = n > 0 ? n : 1;
     }
-    constexpr size_t G = (B >= 32) ? B : 32;      // elements per thread of k_brute
+    constexpr size_t G = brute_group_elems(B);    // elements per thread of k_brute
     const size_t n_blocks = a.n_items;
     const size_t n_groups = n_blocks * B / G;
     if (n_groups > 0) {
