@@ -202,7 +202,18 @@ __device__ __forceinline__ float2 residual_pair(float2 tb, float2 P2, float2 v, 
             : "r"(h), "r"(nD16), "f"(v.x), "f"(v.y));
         return e;
     } else {
-        return __ffma2_rn(__half22float2(*reinterpret_cast<__half2*>(&h)), nD2, v);
+        // f16 -> binary32 as a mixed-precision add of -0 (exact, keeps the sign of zero): unlike a
+        // plain convert it takes its half straight out of the 32-bit register
+        float2 q;
+        asm("{\n"
+            " .reg .b16 qlo, qhi;\n"
+            " mov.b32 {qlo, qhi}, %2;\n"
+            " add.rn.f32.f16 %0, qlo, %3;\n"
+            " add.rn.f32.f16 %1, qhi, %3;\n"
+            "}"
+            : "=f"(q.x), "=f"(q.y)
+            : "r"(h), "f"(-0.0f));
+        return make_float2(__fmaf_rn(q.x, nD2.x, v.x), __fmaf_rn(q.y, nD2.y, v.y));
     }
 }
 
@@ -232,7 +243,15 @@ __device__ __forceinline__ float2 residual_two_candidates(float tA, float tB, fl
             : "=f"(e.x), "=f"(e.y)
             : "r"(h), "r"(nD16), "f"(v));
     } else {
-        const float2 q = __half22float2(*reinterpret_cast<__half2*>(&h));
+        float2 q;   // f16 -> binary32 as in residual_pair()
+        asm("{\n"
+            " .reg .b16 qlo, qhi;\n"
+            " mov.b32 {qlo, qhi}, %2;\n"
+            " add.rn.f32.f16 %0, qlo, %3;\n"
+            " add.rn.f32.f16 %1, qhi, %3;\n"
+            "}"
+            : "=f"(q.x), "=f"(q.y)
+            : "r"(h), "f"(-0.0f));
         e.x = __fmaf_rn(q.x, nDA, v);
         e.y = __fmaf_rn(q.y, nDB, v);
     }
