@@ -129,6 +129,21 @@ __device__ __forceinline__ void residual_pair_f16(uint32_t h, uint32_t nD16, flo
         : "r"(h), "r"(nD16), "f"(v0), "f"(v1));
 }
 
+// The two f16 grid values of a word as binary32: mixed-precision adds of -0 (exact, the sign of a
+// zero is kept), which read their half straight from the 32-bit register.
+__device__ __forceinline__ float2 widen_f16x2(uint32_t h) {
+    float2 q;
+    asm("{\n"
+        " .reg .b16 lo, hi;\n"
+        " mov.b32 {lo, hi}, %2;\n"
+        " add.rn.f32.f16 %0, lo, %3;\n"
+        " add.rn.f32.f16 %1, hi, %3;\n"
+        "}"
+        : "=f"(q.x), "=f"(q.y)
+        : "r"(h), "f"(-0.0f));
+    return q;
+}
+
 template <int DT, int B>
 struct QuantShape {
     static constexpr int EB = elem_bytes(DT);
@@ -192,7 +207,7 @@ __device__ __forceinline__ void pack_and_score(const float* v, const float* t, c
             const float nD = -E[j].x;
 #pragma unroll
             for (int i = 0; i < B; i += 2) {
-                const float2 q = __half22float2(*reinterpret_cast<const __half2*>(&h[(j * B + i) / 2]));
+                const float2 q = widen_f16x2(h[(j * B + i) / 2]);
                 const float e0 = __fmaf_rn(q.x, nD, v[j * B + i]);
                 s = __fmaf_rn(e0, e0, s);
                 const float e1 = __fmaf_rn(q.y, nD, v[j * B + i + 1]);
@@ -270,8 +285,8 @@ __device__ __forceinline__ void encode_group_fast_dual(const float* v, const flo
                 residual_pair_f16(h6[e / 2], nD6_16, v[e], v[e + 1], a0, a1);
                 residual_pair_f16(h4[e / 2], nD4_16, v[e], v[e + 1], b0, b1);
             } else {
-                const float2 q6 = __half22float2(*reinterpret_cast<const __half2*>(&h6[e / 2]));
-                const float2 q4 = __half22float2(*reinterpret_cast<const __half2*>(&h4[e / 2]));
+                const float2 q6 = widen_f16x2(h6[e / 2]);
+                const float2 q4 = widen_f16x2(h4[e / 2]);
                 a0 = __fmaf_rn(q6.x, nD6, v[e]);
                 a1 = __fmaf_rn(q6.y, nD6, v[e + 1]);
                 b0 = __fmaf_rn(q4.x, nD4, v[e]);
