@@ -326,3 +326,28 @@ def test_sse_output_is_optional_and_launches_are_counted():
     torch.cuda.synchronize()
     assert none is None and torch.equal(codes, c2) and torch.equal(scales, s2)
     assert mxq.mxq_launch_count() == before + 2
+
+
+@pytest.mark.parametrize("dtype,B,recipe", [
+    (torch.bfloat16, 16, mxq.MXQ_ABSMAX),        # thread-private staging
+    (torch.bfloat16, 64, mxq.MXQ_4O6),           # cooperative staging, block walked in parts
+    (torch.float32, 32, mxq.MXQ_4O6),            # cooperative staging, whole block in registers
+    (torch.float32, 64, mxq.MXQ_ABSMAX_PZ),      # cooperative staging, 16 pieces per chunk
+    (torch.bfloat16, 2, mxq.MXQ_BRUTE),
+    (torch.float32, 32, mxq.MXQ_BRUTE),
+])
+def test_repeated_launches_give_the_same_bytes(dtype, B, recipe, sweep_mode):
+    """The staging rings hand data from copies to readers (across lanes for the long chunks): a missing
+    wait would show as outputs that change from launch to launch.  Sixty launches over several trips of
+    the persistent grid, two streams' worth of back-to-back work, all compared with the first."""
+    n = 148 * 8 * 256 * max(B, 32) * 2 + 7 * 64          # more chunks than one wave of the grid holds
+    x = inputs.student_t(n, 5, 0.02, 321 + B, dtype, "cuda")
+    ref = [t.clone() for t in mxq.quantize(x, B, mxq.MXQ_SF_UE4M3, recipe)]
+    codes, scales, sse = mxq.alloc_outputs(n, B, "cuda")
+    for it in range(60):
+        mxq.mxq_quantize_ex(x, n, B, mxq.MXQ_SF_UE4M3, recipe, 1.0, None, codes, scales, sse)
+        if it % 20 == 19:
+            torch.cuda.synchronize()
+            assert torch.equal(codes, ref[0]) and torch.equal(scales, ref[1])
+            assert torch.equal(sse.view(torch.int32), ref[2].view(torch.int32))
+    check_parity(x[: 4096 * B].cpu(), B, mxq.MXQ_SF_UE4M3, recipe)
