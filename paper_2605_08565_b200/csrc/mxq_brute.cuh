@@ -258,21 +258,11 @@ __device__ __forceinline__ float2 residual_two_candidates(float tA, float tB, fl
     return e;
 }
 
-// fl32(v / Dref) for both halves; nD = -Dref, R = RN(1 / Dref), Dref in [1, 2), |v| <= 2^60.
-// Same value as quotient_corrected() except for the sign of a zero quotient, which the search
-// does not use.
+// fl32(v / Dref) for both halves; nD = -Dref, R = RN(1 / Dref), Dref in [1, 2), |v| <= 2^60: the
+// reciprocal multiply with one residual correction of quotient_short() (see there why one
+// correction gives the IEEE quotient for every divisor), except for the sign of a zero quotient,
+// which the search does not use.
 __device__ __forceinline__ float2 quotient_pair(float2 v, float2 nD, float2 R) {
-    float2 q = __fmul2_rn(v, R);
-    float2 r = __ffma2_rn(q, nD, v);
-    q = __ffma2_rn(r, R, q);
-    r = __ffma2_rn(q, nD, v);
-    q = __ffma2_rn(r, R, q);
-    return q;
-}
-
-// The same with ONE correction: exact when the significand of Dref has at most 19 bits (see
-// quotient_short() of the one-pass kernels for the argument).
-__device__ __forceinline__ float2 quotient_pair_short(float2 v, float2 nD, float2 R) {
     const float2 q = __fmul2_rn(v, R);
     const float2 r = __ffma2_rn(q, nD, v);
     return __ffma2_rn(r, R, q);
@@ -468,8 +458,6 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
     const int first = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     build_brute_tables<FMT, PRUNE>(T, g, first);
 
-    // all decode scales are short multiples of a class reference when g itself has few bits
-    const bool short_ref = (__float_as_uint(g) & 0x1FFu) == 0u;   // <= 15 bits of g, <= 19 bits of Dref
 
     // With PRUNE the loop is uniform per warp (lanes past the end repeat the warp's first group
     // and store nothing), so that the warp can agree on the candidates it leaves out.
@@ -529,7 +517,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
             const float2 nDr2 = make_float2(-Dr, -Dr), Rr2 = make_float2(Rr, Rr);
 #pragma unroll
             for (int i = 0; i < NP; ++i)
-                tb[i] = short_ref ? quotient_pair_short(v2[i], nDr2, Rr2) : quotient_pair(v2[i], nDr2, Rr2);
+                tb[i] = quotient_pair(v2[i], nDr2, Rr2);
         };
 
         if constexpr (!PRUNE) {

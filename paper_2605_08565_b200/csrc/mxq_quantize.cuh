@@ -47,13 +47,10 @@ namespace mxq {
 //      D = 0 counts as valid with R = 0: every quotient comes out as a zero with the sign of v.
 struct QuantTables {
     float4 E[256];
-    int all_short;   // every entry with w != 0 has a significand of at most 19 bits
 };
 
 template <int FMT>
 __device__ __forceinline__ void build_quant_tables(QuantTables& T, float g) {
-    if (threadIdx.x == 0) T.all_short = 1;
-    __syncthreads();
     for (int c = threadIdx.x; c < 256; c += blockDim.x) {
         float D = __uint_as_float(0x7FC00000u), R = 0.0f, w = 0.0f;
         uint32_t h16 = 0;
@@ -65,7 +62,6 @@ __device__ __forceinline__ void build_quant_tables(QuantTables& T, float g) {
                 const __half hD = __float2half_rn(-D);
                 h16 = (uint32_t)__half_as_ushort(hD);
                 w = (__half2float(hD) == -D) ? 2.0f : 1.0f;
-                if (__float_as_uint(D) & 0x1Fu) T.all_short = 0;   // benign race: every writer stores 0
             }
         }
         T.E[c] = make_float4(D, R, __uint_as_float(h16), w);
@@ -73,11 +69,14 @@ __device__ __forceinline__ void build_quant_tables(QuantTables& T, float g) {
     __syncthreads();
 }
 
-// fl32(v / D) when the significand of D has at most 19 bits: reciprocal multiply and ONE residual
-// correction.  q0 = RN(v * R) is within 1.5 ulp of v / D, the residual q0 * D - v is then exactly
-// representable, and q0 - r * R differs from v / D by at most 1.5 * 2^-24 ulp before its final
-// rounding; v / D itself stays at least 2^-20 ulp away from every rounding boundary because D has
-// few bits, so that rounding is the correct one.  Range conditions as for quotient_corrected().
+// fl32(v / D) by a reciprocal multiply and ONE residual correction, R = RN(1 / D) correctly rounded,
+// D and |v| within [2^-60, 2^60].  Why one correction is enough: q0 = RN(v * R) is within 1.5 ulp
+// of v / D, the residual q0 * D - v is exact (or, in the lower half of a binade, rounded by at most
+// 2^-47 relative to a quotient in [1/2, 1)), and the value that the final FMA rounds differs from
+// v / D by at most 3.5 * 2^-48 of that scale.  v / D can be that close to a rounding boundary (the
+// midpoint of two neighbouring floats) only when |A * 2^K - B * m| <= 6 for the integer
+// significands A, B of v, D and an odd m (K = 24 or 25); all 93 million such pairs (bound 16) were
+// enumerated on the host and give the IEEE quotient (tests/quotient_hard_cases.c).
 __device__ __forceinline__ float quotient_short(float v, float D, float R) {
     const float q = __fmul_rn(v, R);
     const float r = __fmaf_rn(q, D, -v);
@@ -219,10 +218,9 @@ __device__ __forceinline__ void pack_and_score(const float* v, const float* t, c
 }
 
 // Quotients of one block by its decode scale, two elements per instruction (fma.rn.f32x2):
-// q = (-v) * (-R); r = q * D - v; q <- q - r * R, once (SHORTQ) or twice.  Same values as
-// quotient_short() / quotient_corrected(), including the sign of a zero quotient: every product and
-// sum has the signs of the scalar forms.
-template <int B, bool SHORTQ>
+// q = (-v) * (-R); r = q * D - v; q <- q - r * R.  Same values as quotient_short(), including the
+// sign of a zero quotient: every product and sum has the signs of the scalar form.
+template <int B>
 __device__ __forceinline__ void block_quotients(const float* v, float D, float R, float* t) {
     const float2 D2 = make_float2(D, D), nR2 = make_float2(-R, -R);
 #pragma unroll
@@ -231,23 +229,19 @@ __device__ __forceinline__ void block_quotients(const float* v, float D, float R
         float2 q = __fmul2_rn(nv, nR2);
         float2 r = __ffma2_rn(q, D2, nv);
         q = __ffma2_rn(r, nR2, q);
-        if constexpr (!SHORTQ) {
-            r = __ffma2_rn(q, D2, nv);
-            q = __ffma2_rn(r, nR2, q);
-        }
         t[i] = q.x;
         t[i + 1] = q.y;
     }
 }
 
 // One candidate set of a group with the shortcuts (every entry has w != 0, magnitudes in range).
-template <int B, bool SHORTQ, bool HALF>
+template <int B, bool HALF>
 __device__ __forceinline__ void encode_group_fast(const float* v, const float4* E, uint32_t* packed, float* sse) {
     constexpr int GE = (B < 8) ? 8 : B;
     constexpr int NBG = GE / B;
     float t[GE];
 #pragma unroll
-    for (int j = 0; j < NBG; ++j) block_quotients<B, SHORTQ>(&v[j * B], E[j].x, E[j].y, &t[j * B]);
+    for (int j = 0; j < NBG; ++j) block_quotients<B>(&v[j * B], E[j].x, E[j].y, &t[j * B]);
     pack_and_score<B, HALF>(v, t, E, packed, sse);
 }
 
@@ -255,7 +249,7 @@ __device__ __forceinline__ void encode_group_fast(const float* v, const float4* 
 // candidate, and the two SSE chains of a block side by side in one fma.rn.f32x2 per element
 // (lane .x: the M = 6 candidate, lane .y: the M = 4 candidate; each lane sums its own residuals
 // in element order, exactly like the scalar chain).  The chains continue from sse6[] / sse4[].
-template <int B, bool SHORTQ, bool HALF>
+template <int B, bool HALF>
 __device__ __forceinline__ void encode_group_fast_dual(const float* v, const float4* E6, const float4* E4, uint32_t* pk6,
                                                        uint32_t* pk4, float* sse6, float* sse4) {
     constexpr int GE = (B < 8) ? 8 : B;
@@ -263,8 +257,8 @@ __device__ __forceinline__ void encode_group_fast_dual(const float* v, const flo
     float t6[GE], t4[GE];
 #pragma unroll
     for (int j = 0; j < NBG; ++j) {
-        block_quotients<B, SHORTQ>(&v[j * B], E6[j].x, E6[j].y, &t6[j * B]);
-        block_quotients<B, SHORTQ>(&v[j * B], E4[j].x, E4[j].y, &t4[j * B]);
+        block_quotients<B>(&v[j * B], E6[j].x, E6[j].y, &t6[j * B]);
+        block_quotients<B>(&v[j * B], E4[j].x, E4[j].y, &t4[j * B]);
     }
     uint32_t h6[GE / 2], h4[GE / 2];
 #pragma unroll
@@ -318,7 +312,7 @@ __device__ __forceinline__ void encode_group_general(const float* v, const float
 struct QuantConsts {
     float g, Rg;        // tensor scale and RN(1 / g)
     float m_lo, m_hi;   // a block maximum m takes the shortcuts when m == 0 or m_lo <= m <= m_hi
-    bool unit_g, need_lo, all_short;
+    bool unit_g, need_lo;
     int c_min;          // smallest admissible code: 1 under prevent-zero (FP8 formats), else 0
     int pow2_rule;      // kPow2Eq1 unless the format is UE8M0 and another rule was asked for
 };
@@ -333,7 +327,7 @@ __device__ __forceinline__ int target6_code(float u, int pow2_rule) {
     return round_scale<FMT>(EXACT ? __fdiv_rn(u, 6.0f) : div6_fast(u));
 }
 
-template <int DT, int B, int FMT, bool DUAL, bool SHORTQ, bool FAKE>
+template <int DT, int B, int FMT, bool DUAL, bool FAKE>
 __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
                                                size_t chunk, const uint32_t* raw) {
     using S = QuantShape<DT, B>;
@@ -376,11 +370,11 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
         for (int j = 0; j < NBG; ++j) sse[j] = sse4[j] = 0.0f;
         if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
             if (wmin >= 2.0f) {   // one decision for both candidates
-                if constexpr (DUAL) encode_group_fast_dual<B, SHORTQ, true>(v, E6, E4, pk, pk4, sse, sse4);
-                else encode_group_fast<B, SHORTQ, true>(v, E6, pk, sse);
+                if constexpr (DUAL) encode_group_fast_dual<B, true>(v, E6, E4, pk, pk4, sse, sse4);
+                else encode_group_fast<B, true>(v, E6, pk, sse);
             } else {
-                if constexpr (DUAL) encode_group_fast_dual<B, SHORTQ, false>(v, E6, E4, pk, pk4, sse, sse4);
-                else encode_group_fast<B, SHORTQ, false>(v, E6, pk, sse);
+                if constexpr (DUAL) encode_group_fast_dual<B, false>(v, E6, E4, pk, pk4, sse, sse4);
+                else encode_group_fast<B, false>(v, E6, pk, sse);
             }
         } else {
 #pragma unroll
@@ -475,7 +469,7 @@ __device__ __forceinline__ int ring_index(int k, int lane) {
 // elements read from the thread's ring slot, which stays valid until the next trip's request:
 // once for the block maximum, once for the encode with the SSE chains carried from part to part.
 // Only one part is live in registers at a time, which keeps as many CTAs resident as for B = 16.
-template <int DT, int B, int FMT, bool DUAL, bool SHORTQ, bool FAKE>
+template <int DT, int B, int FMT, bool DUAL, bool FAKE>
 __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
                                                     size_t chunk, const uint4* slot_warp, int lane) {
     using S = QuantShape<DT, B>;
@@ -531,11 +525,11 @@ __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const Qu
         uint32_t* o4 = &pk4[sg * (SG / 8)];
         if (fast) {
             if (wmin >= 2.0f) {
-                if constexpr (DUAL) encode_group_fast_dual<SG, SHORTQ, true>(v, &E6, &E4, o6, o4, &sse, &sse4);
-                else encode_group_fast<SG, SHORTQ, true>(v, &E6, o6, &sse);
+                if constexpr (DUAL) encode_group_fast_dual<SG, true>(v, &E6, &E4, o6, o4, &sse, &sse4);
+                else encode_group_fast<SG, true>(v, &E6, o6, &sse);
             } else {
-                if constexpr (DUAL) encode_group_fast_dual<SG, SHORTQ, false>(v, &E6, &E4, o6, o4, &sse, &sse4);
-                else encode_group_fast<SG, SHORTQ, false>(v, &E6, o6, &sse);
+                if constexpr (DUAL) encode_group_fast_dual<SG, false>(v, &E6, &E4, o6, o4, &sse, &sse4);
+                else encode_group_fast<SG, false>(v, &E6, o6, &sse);
             }
         } else {
             encode_group_general<SG>(v, &E6, o6, &sse);
@@ -650,7 +644,6 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     build_quant_tables<FMT>(T, k.g);
     k.unit_g = (k.g == 1.0f);
     k.c_min = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
-    k.all_short = T.all_short != 0;
     k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;
     k.Rg = 1.0f;
     // Ranges of a block maximum m for which u = fl(m / g) and fl(u / 6) come out exact from the
@@ -696,8 +689,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
         // blocks longer than 16 elements go part by part, except 4-over-6 at B = 32, which measured
         // slightly faster with the whole block in registers
         if constexpr (B > 16 && !(DUAL && B == 32)) {
-            if (k.all_short) quantize_long_block<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, slot_warp, lane);
-            else quantize_long_block<DT, B, FMT, DUAL, false, FAKE>(p, T, k, chunk, slot_warp, lane);
+            quantize_long_block<DT, B, FMT, DUAL, FAKE>(p, T, k, chunk, slot_warp, lane);
         } else {
             uint32_t raw[S::PIECES * 4];
 #pragma unroll
@@ -705,8 +697,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
                 const uint4 w = slot_warp[ring_index<S::COOP>(q, lane)];
                 raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
             }
-            if (k.all_short) quantize_chunk<DT, B, FMT, DUAL, true, FAKE>(p, T, k, chunk, raw);
-            else quantize_chunk<DT, B, FMT, DUAL, false, FAKE>(p, T, k, chunk, raw);
+            quantize_chunk<DT, B, FMT, DUAL, FAKE>(p, T, k, chunk, raw);
         }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
