@@ -95,18 +95,16 @@ __device__ __forceinline__ void build_scale_tables(float* tabD, float* tabR, flo
     __syncthreads();
 }
 
-// fl32(v / D) for kFastMin <= D <= kFastMax, |v| <= kFastMax, R = RN(1/D): a reciprocal
-// multiply followed by two residual corrections.  With a correctly rounded reciprocal the second
-// correction returns the correctly rounded quotient wherever |v/D| >= 2^-3; smaller quotients may
-// be off by rounding but stay far below the first FP4 decision point (0.25).  The residuals are
+// fl32(v / D) for kFastMin <= D <= kFastMax, |v| <= kFastMax, R = RN(1/D): a reciprocal multiply
+// followed by one residual correction, which is the IEEE quotient for every such pair (the
+// argument and the enumeration of the hard cases are with quotient_short() of the one-pass
+// kernels; magnitudes below 2^-62 may lose the residual to underflow, but their quotients stay far
+// below the first FP4 decision point, 0.25, or they are sent to the general path).  The residual is
 // formed as (q*D - v) so that a zero quotient keeps the sign of v.
 __device__ __forceinline__ float quotient_corrected(float v, float D, float R) {
-    float q = __fmul_rn(v, R);
-    float r = __fmaf_rn(q, D, -v);
-    q = __fmaf_rn(-r, R, q);
-    r = __fmaf_rn(q, D, -v);
-    q = __fmaf_rn(-r, R, q);
-    return q;
+    const float q = __fmul_rn(v, R);
+    const float r = __fmaf_rn(q, D, -v);
+    return __fmaf_rn(-r, R, q);
 }
 
 // General quotient: IEEE division; a zero scale sends every element to (signed) zero.
