@@ -2,18 +2,28 @@
 """Benchmark of the block-scaled FP4 quantize + scale-search + MSE hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mxq|reference]
+    python bench.py --config 1|2|3|4|5|all      one benchmark configuration, one recipe at a time
+    python bench.py --kernel absmax|4o6|brute|...   one kernel alone (sweeps, ncu captures)
 
-Workload (N = 1): the weight-shaped sweep -- 4096x4096 bf16, 0.02 * Student-t(nu=5), UE4M3 block
-scales, no tensor scale, block sizes {2,4,8,16,32,64}.  One STEP is one pass of the whole hot path
-over that batch: for every block size, quantize with abs-max, abs-max + prevent-zero, 4-over-6 and
-brute force, each followed by the tensor MSE reduction; plus the hierarchical leg (tensor abs-max ->
-device-resident global scale -> abs-max quantize at block 16 -> MSE) and one de-quantization.
-Successive passes read different tensors out of a rotating set larger than L2, so inputs come from
-HBM.  `value` = elements quantized per second over the whole job (all passes, all ranks).
+Workload of the default run (N = 1), one STEP = one pass of the whole hot path over one batch:
 
-With N > 1 (torchrun, one rank per GPU) every rank runs the same sweep on its own tensors: weak
-scaling, no data-path collective; the timed region is bracketed by barrier + synchronize and the
-time is the maximum over ranks.
+* bulk scale search: 16384 x 16384 fp32 Laplace(0,1), tensor abs-max -> device-resident tensor scale
+  g = amax / 2688, then the full brute-force sweep for every block size in {2,4,8,16,32} and every
+  scale format in {UE8M0, UE4M3, UE5M3}, each followed by the tensor MSE (15 sweeps);
+* weight leg: one matrix of each shape of an 8B-parameter Llama-style layer (4096x4096, 1024x4096,
+  14336x4096, 4096x14336; bf16, Student-t(4)/sqrt(fan_in)), block sizes {8,16} x {UE4M3, UE5M3} x
+  {abs-max, abs-max + prevent-zero, 4-over-6, 4-over-6 + prevent-zero}, tensor MSE after each;
+* activation leg: 8192 x 4096 bf16 with 1 % outlier columns, block 16: hierarchical scaling (tensor
+  abs-max -> g -> UE4M3 blocks) against UE5M3 blocks without a tensor scale, abs-max and 4-over-6,
+  tensor MSE after each, and one de-quantization.
+
+Inputs larger than L2 (the 1 GiB tensor), or visited so that no tensor is read twice within 126 MB of
+other traffic (the legs walk their matrices round-robin).  `value` = elements quantized per second
+over the whole job (all passes, all ranks).
+
+With N > 1 (one rank per GPU; `--gpus N` starts the ranks itself when it was not started by torchrun)
+every rank runs the same step on its own tensors: weak scaling, no data-path collective; the timed
+region is bracketed by barrier + synchronize and the time is the maximum over ranks.
 
 `--impl reference` times the CPU oracle (oracle/mxq_oracle.c) on the host cores on a bounded sample
 of the same workload and prints the same JSON line with "impl": "reference".
@@ -21,8 +31,12 @@ of the same workload and prints the same JSON line with "impl": "reference".
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
+import re
+import socket
 import statistics
 import subprocess
 import sys
@@ -35,32 +49,31 @@ if ROOT not in sys.path:
 
 METRIC = "GElem/s quantize+MSE per recipe (abs-max, 4/6, brute force); % HBM/ALU roofline"
 UNIT = "GElem/s"
-ROWS, COLS = 4096, 4096
-N_ELEM = ROWS * COLS
-BLOCKS = (2, 4, 8, 16, 32, 64)
-N_ROTATE = 8                      # 8 x 32 MiB inputs = 256 MiB > 126 MB L2
-UE4M3 = 1
-ABSMAX, ABSMAX_PZ, R4O6, BRUTE = 0, 1, 2, 4
-RECIPE_NAME = {ABSMAX: "absmax", ABSMAX_PZ: "absmax_pz", R4O6: "4o6", BRUTE: "brute"}
-N_CODES_UE4M3 = 127
+UE8M0, UE4M3, UE5M3 = 0, 1, 2
+ABSMAX, ABSMAX_PZ, R4O6, R4O6_PZ, BRUTE, BRUTE_PZ = 0, 1, 2, 3, 4, 5
+RECIPE_NAME = {ABSMAX: "absmax", ABSMAX_PZ: "absmax_pz", R4O6: "4o6", R4O6_PZ: "4o6_pz", BRUTE: "brute",
+               BRUTE_PZ: "brute_pz"}
+FMT_NAME = {UE8M0: "ue8m0", UE4M3: "ue4m3", UE5M3: "ue5m3"}
+N_CODES = {UE8M0: 255, UE4M3: 127, UE5M3: 255}
 ALU_LANES_PER_SM = 128            # 4 schedulers x 32 lanes, one instruction per scheduler per clock
-CPU_SAMPLE_ELEMS = 1 << 20
-REFERENCE_BUDGET_S = 35.0        # wall-clock target of a whole --impl reference run
+NOMINAL_HBM_GBS = 8000.0          # the bandwidth the targets are quoted against; the measured copy peak is lower
+
+# ---- the step's workload -------------------------------------------------------------------------
+SEARCH_ROWS = SEARCH_COLS = 16384
+SEARCH_N = SEARCH_ROWS * SEARCH_COLS
+SEARCH_BLOCKS = (2, 4, 8, 16, 32)
+SEARCH_FMTS = (UE8M0, UE4M3, UE5M3)
+WEIGHT_SHAPES = (("q", 4096, 4096, 0), ("k", 1024, 4096, 1), ("gate", 14336, 4096, 4), ("down", 4096, 14336, 6))
+WEIGHT_BLOCKS = (8, 16)
+WEIGHT_FMTS = (UE4M3, UE5M3)
+WEIGHT_RECIPES = (ABSMAX, ABSMAX_PZ, R4O6, R4O6_PZ)
+ACT_ROWS, ACT_COLS, ACT_ROTATE = 8192, 4096, 3
+ACT_N = ACT_ROWS * ACT_COLS
+ACT_PASSES = ((UE4M3, True, ABSMAX), (UE5M3, False, ABSMAX), (UE4M3, True, R4O6), (UE5M3, False, R4O6))
+
+CPU_SAMPLE_ELEMS = 1 << 20        # per tensor, cpu_baseline leg
+REFERENCE_BUDGET_S = 40.0         # wall-clock target of a whole --impl reference run
 STREAM_ELEMS = 1 << 27            # tensor size of the streaming (HBM-bound) kernel measurements
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (same kernel build, same launch configuration); set an entry to None when its kernel changes.
-# smsp__issue_active.avg.pct_of_peak_sustained_active of the brute-force kernel in the same capture
-NCU_BRUTE_ISSUE_ACTIVE_PCT = 70.8
-NCU_TRAFFIC_BYTES = {
-    "k_brute<bf16,B=16,UE4M3>@16Mi": 33.620224e6 + 0.016128e6,
-    "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi": 268.471552e6 + 82.490624e6,
-    "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi": 268.489216e6 + 83.071488e6,
-    "k_quantize<f32,B=16,UE4M3,absmax>@128Mi": 536.895488e6 + 95.571200e6,
-}
-
-
-def pass_list():
-    return [(B, r) for B in BLOCKS for r in (ABSMAX, ABSMAX_PZ, R4O6, BRUTE)]
 
 
 def measured_peaks():
@@ -70,6 +83,43 @@ def measured_peaks():
             p = json.load(f)
         return {"hbm_gbs": float(p["hbm_gbs"]), "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
     return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+def kernel_source_digest(*names) -> str:
+    """SHA-256 over the kernel sources a profile summary depends on (ties recorded ncu figures to the code)."""
+    h = hashlib.sha256()
+    for n in names:
+        with open(os.path.join(ROOT, "paper_2605_08565_b200", "csrc", n), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_profile(fname: str, sources) -> dict:
+    """Figures of a committed ncu summary (profiles/<fname>): returned only while the kernel sources still
+    hash to the digest written in that file; otherwise the figures are stale and reported as such."""
+    path = os.path.join(ROOT, "profiles", fname)
+    out = {"file": "profiles/" + fname, "stale": True, "dram_bytes": None, "issue_active_pct": None, "elems": None}
+    if not os.path.exists(path):
+        return out
+    txt = open(path).read()
+    m = re.search(r"kernel_source_digest:\s*([0-9a-f]+)", txt)
+    if not m or m.group(1) != kernel_source_digest(*sources):
+        return out
+
+    def num(key):
+        mm = re.search(re.escape(key) + r"\s+([0-9.eE+-]+)\s*(\S*)", txt)
+        if not mm:
+            return None
+        v = float(mm.group(1))
+        unit = mm.group(2).lower()
+        return v * {"kbyte": 1e3, "mbyte": 1e6, "gbyte": 1e9}.get(unit, 1.0)
+
+    rd, wr = num("dram__bytes_read.sum"), num("dram__bytes_write.sum")
+    me = re.search(r"elements_per_launch:\s*(\d+)", txt)
+    out.update(stale=False, dram_bytes=(rd + wr) if rd is not None and wr is not None else None,
+               issue_active_pct=num("smsp__issue_active.avg.pct_of_peak_sustained_active"),
+               elems=int(me.group(1)) if me else None)
+    return out
 
 
 class ClockSampler:
@@ -116,28 +166,6 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# ------------------------------------------------------------------------------------------------
-# CPU oracle legs (cpu_baseline of the normal run; the whole of --impl reference)
-# ------------------------------------------------------------------------------------------------
-def oracle_sample_run(sample_bits, threads: int) -> tuple[float, float]:
-    """One pass of the step's recipe mix over the sample with the oracle; returns (elements, seconds)."""
-    from oracle import mxq_oracle as orc
-    n = sample_bits.size
-    t0 = time.perf_counter()
-    elems = 0
-    for B, r in pass_list():
-        _, _, sse = orc.quantize(sample_bits, B, orc.UE4M3, r, 1.0, threads=threads)
-        orc.tensor_mse(sse, n)
-        elems += n
-    amax = orc.tensor_amax(sample_bits)
-    g = float(orc.global_scale_from_amax(amax))
-    codes, scales, sse = orc.quantize(sample_bits, 16, orc.UE4M3, orc.ABSMAX, g, threads=threads)
-    orc.tensor_mse(sse, n)
-    orc.dequantize(codes, scales, n, 16, orc.UE4M3, g, orc.BF16)
-    elems += n
-    return float(elems), time.perf_counter() - t0
-
-
 def host_threads() -> int:
     try:
         return max(1, len(os.sched_getaffinity(0)))
@@ -145,51 +173,120 @@ def host_threads() -> int:
         return os.cpu_count() or 1
 
 
-def host_sample(seed: int, n: int):
+def algorithmic_bytes(n: int, elem_bytes: int, B: int) -> float:
+    """Input + packed codes + scale bytes + block SSE of one fused quantize launch."""
+    return n * (elem_bytes + 0.5 + 5.0 / B)
+
+
+def pass_table():
+    """Every quantize pass of one step: (leg, tensor key, elements, block, format, recipe, tensor scale?)."""
+    rows = []
+    for B in SEARCH_BLOCKS:
+        for fmt in SEARCH_FMTS:
+            rows.append(("search", "search", SEARCH_N, B, fmt, BRUTE, True))
+    for B in WEIGHT_BLOCKS:
+        for fmt in WEIGHT_FMTS:
+            for r in WEIGHT_RECIPES:
+                for name, rr, cc, _ in WEIGHT_SHAPES:
+                    rows.append(("weight", "w_" + name, rr * cc, B, fmt, r, False))
+    for i, (fmt, hier, r) in enumerate(ACT_PASSES):
+        rows.append(("act", f"a_{i % ACT_ROTATE}", ACT_N, 16, fmt, r, hier))
+    return rows
+
+
+WORKLOAD_NAME = ("bulk scale search 16384x16384 fp32 Laplace, g=amax/2688, brute force full sweep, B in {2,4,8,16,32} x "
+                 "{UE8M0,UE4M3,UE5M3} + MSE each; + weight leg (Llama-8B layer shapes 4096x4096, 1024x4096, 14336x4096, "
+                 "4096x14336 bf16 t4/sqrt(fan_in), B in {8,16} x {UE4M3,UE5M3} x {abs-max, +pz, 4-over-6, +pz} + MSE each); "
+                 "+ activation leg (8192x4096 bf16 outlier columns, B=16, hierarchical UE4M3 vs UE5M3, abs-max and "
+                 "4-over-6 + MSE each, dequantize)")
+
+
+# ------------------------------------------------------------------------------------------------
+# Host-side inputs (the oracle legs and the end-to-end arm read these)
+# ------------------------------------------------------------------------------------------------
+def make_inputs(rank: int, device, n_limit: int | None = None):
+    """The step's tensors, keyed as in pass_table(); n_limit keeps only a prefix of each (oracle legs)."""
     import torch
-    from paper_2605_08565_b200 import inputs
-    return inputs.to_numpy_bits(inputs.student_t(n, 5, 0.02, seed, torch.bfloat16, "cpu"))
+    from paper_2605_08565_b200 import dist, inputs
+
+    def cut(n):
+        return n if n_limit is None else min(n, n_limit)
+
+    t = {"search": inputs.laplace(cut(SEARCH_N), dist.rank_seed(5, rank), torch.float32, device)}
+    for name, rr, cc, idx in WEIGHT_SHAPES:
+        t["w_" + name] = inputs.student_t(cut(rr * cc), 4, 1.0 / math.sqrt(cc), dist.rank_seed(4, rank, idx),
+                                          torch.bfloat16, device)
+    for i in range(ACT_ROTATE):
+        if n_limit is None:
+            t[f"a_{i}"] = inputs.outlier_columns(ACT_ROWS, ACT_COLS, dist.rank_seed(3, rank, i), dtype=torch.bfloat16,
+                                                 device=device)
+        else:
+            rows = max(1, n_limit // ACT_COLS)
+            t[f"a_{i}"] = inputs.outlier_columns(rows, ACT_COLS, dist.rank_seed(3, rank, i), dtype=torch.bfloat16,
+                                                 device=device)
+    return t
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs (cpu_baseline of the normal run; the whole of --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_step(samples: dict, threads: int, frac: float = 1.0) -> tuple[float, float]:
+    """One step's pass list over host samples with the oracle; returns (elements, seconds).
+    samples: key -> numpy bits (prefixes of the step's tensors); frac < 1 shortens every prefix."""
+    from oracle import mxq_oracle as orc
+    t0 = time.perf_counter()
+    elems = 0
+    g_of = {}
+    for leg, key, _, B, fmt, recipe, hier in pass_table():
+        x = samples[key]
+        n = max(64, int(x.size * frac) // 64 * 64)
+        x = x[:n]
+        g = 1.0
+        if hier:
+            if (key, n) not in g_of:
+                g_of[(key, n)] = float(orc.global_scale_from_amax(orc.tensor_amax(x)))
+            g = g_of[(key, n)]
+        codes, scales, sse = orc.quantize(x, B, fmt, recipe, g, threads=threads)
+        orc.tensor_mse(sse, n)
+        elems += n
+    orc.dequantize(codes, scales, n, 16, fmt, g, orc.BF16)
+    return float(elems), time.perf_counter() - t0
 
 
 def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    import torch
     from oracle import mxq_oracle as orc
+    from paper_2605_08565_b200 import inputs
     orc.build()
     threads = host_threads()
+    full = {k: inputs.to_numpy_bits(v) for k, v in make_inputs(0, "cpu", CPU_SAMPLE_ELEMS // 4).items()}
     # Size the per-step sample so that the whole run (warm-up + steps) stays near REFERENCE_BUDGET_S:
-    # probe the oracle's rate on 4096 elements, then give every step the same prefix of tensor 0.
-    full = host_sample(2, CPU_SAMPLE_ELEMS // 8)
-    pe, ps = oracle_sample_run(full[: 1 << 12], 1)
-    rate1 = pe / max(ps, 1e-6)                                  # elements of the recipe mix per second, one thread
-    passes = len(pass_list()) + 1
+    # probe the oracle's rate on a short prefix, then give every step the same prefix of every tensor.
+    probe_frac = 4096.0 / (CPU_SAMPLE_ELEMS // 4)
+    pe, ps = oracle_step(full, threads, probe_frac)
+    rate = pe / max(ps, 1e-6)                                    # elements of the pass mix per second
     trips = max(1, args.steps + args.warmup)
-    n_sample, use = 256, 1
-    for t in sorted({1, 2, 4, 8, threads}):                     # most threads that still get >= 2048 elements each
-        if t > threads:
-            continue
-        n_t = int(min(full.size, REFERENCE_BUDGET_S * rate1 * t / trips / passes)) // 64 * 64
-        if t == 1 or n_t >= 2048 * t:
-            n_sample, use = max(256, n_t), t
-    threads = use
-    sample = full[:n_sample]
+    per_step_elems = REFERENCE_BUDGET_S * rate / trips
+    frac = min(1.0, max(probe_frac / 8, per_step_elems / (len(pass_table()) * (CPU_SAMPLE_ELEMS // 4))))
     for _ in range(args.warmup):
-        oracle_sample_run(sample, threads)
+        oracle_step(full, threads, frac)
     elems, secs = 0.0, 0.0
     for _ in range(args.steps):
-        e, s = oracle_sample_run(sample, threads)
+        e, s = oracle_step(full, threads, frac)
         elems += e
         secs += s
     value = elems / secs / 1e9
-    sample_desc = (f"first {sample.size} elements of the 4096x4096 bf16 Student-t tensor, every pass of the step "
-                   f"(6 block sizes x abs-max, abs-max+pz, 4-over-6, brute force, + hierarchical leg)")
+    n_prefix = max(64, int((CPU_SAMPLE_ELEMS // 4) * frac) // 64 * 64)
+    sample_desc = (f"first {n_prefix} elements of every tensor of the step, every pass of the step "
+                   f"({len(pass_table())} quantize passes + MSE each, dequantize)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "weight sweep 4096x4096 bf16 Student-t(5)*0.02, UE4M3, B in {2..64} (bounded sample)",
-                   "sample_elems": int(sample.size)},
+        "config": {"workload": WORKLOAD_NAME + " (bounded sample)", "sample_elems_per_tensor": n_prefix},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample_desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -203,145 +300,228 @@ class Workload:
     def __init__(self, rank: int, device):
         import torch
         from paper_2605_08565_b200 import binding as mxq
-        from paper_2605_08565_b200 import dist, inputs
-        self.torch, self.mxq = torch, mxq
-        self.device = device
-        self.x = [inputs.student_t(N_ELEM, 5, 0.02, dist.rank_seed(2, rank, i), torch.bfloat16, device)
-                  for i in range(N_ROTATE)]
-        self.codes = torch.empty(N_ELEM // 2, dtype=torch.uint8, device=device)
-        self.scales = torch.empty(N_ELEM // 2, dtype=torch.uint8, device=device)
-        self.sse = torch.empty(N_ELEM // 2, dtype=torch.float32, device=device)
-        self.passes = pass_list()
-        self.mse = torch.zeros(len(self.passes) + 1, dtype=torch.float64, device=device)
-        self.ws = torch.empty(mxq.mxq_tensor_mse_workspace_bytes(N_ELEM // 2) // 8, dtype=torch.float64, device=device)
-        self.amax = torch.empty(1, dtype=torch.float32, device=device)
-        self.g = torch.empty(1, dtype=torch.float32, device=device)
-        self.xhat = torch.empty(N_ELEM, dtype=torch.bfloat16, device=device)
-        self.rot = 0
-        self.timers = {}          # (B, recipe) -> list of (start, stop) event pairs
-        self.elems_per_step = float(N_ELEM * (len(self.passes) + 1))
+        self.torch, self.mxq, self.device = torch, mxq, device
+        self.x = make_inputs(rank, device)
+        self.passes = pass_table()
+        nmax = SEARCH_N
+        self.codes = torch.empty(nmax // 2, dtype=torch.uint8, device=device)
+        self.scales = torch.empty(nmax // 2, dtype=torch.uint8, device=device)
+        self.sse = torch.empty(nmax // 2, dtype=torch.float32, device=device)
+        self.mse = torch.zeros(len(self.passes), dtype=torch.float64, device=device)
+        self.ws = torch.empty(mxq.mxq_tensor_mse_workspace_bytes(nmax // 2) // 8, dtype=torch.float64, device=device)
+        self.amax = torch.empty(4, dtype=torch.float32, device=device)
+        self.g = torch.empty(4, dtype=torch.float32, device=device)
+        self.xhat = torch.empty(ACT_N, dtype=torch.bfloat16, device=device)
+        self.search_events = {}   # (B, fmt) -> list of (start, stop)
+        self.leg_events = {}      # leg -> list of (start, stop)
+        self.elems_per_step = float(sum(p[2] for p in self.passes))
 
-    def _next_input(self):
-        x = self.x[self.rot % len(self.x)]
-        self.rot += 1
-        return x
+    def _ev(self):
+        return self.torch.cuda.Event(enable_timing=True)
 
-    def one_pass(self, x, B, recipe, slot, timed_keys=()):
-        mxq, torch = self.mxq, self.torch
-        key = (B, recipe)
-        ev = None
-        if key in timed_keys:
-            ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-            ev[0].record()
-        mxq.mxq_quantize_ex(x, N_ELEM, B, UE4M3, recipe, 1.0, None, self.codes, self.scales, self.sse)
-        if ev is not None:
-            ev[1].record()
-            self.timers.setdefault(key, []).append(ev)
-        mxq.mxq_tensor_mse(self.sse, N_ELEM // B, N_ELEM, self.mse[slot:slot + 1], self.ws)
-
-    def step(self, x_override=None, timed_keys=()):
+    def step(self, x=None, timed=False):
+        """One pass of the whole hot path.  x: the tensors to read (default: the resident set)."""
         mxq = self.mxq
-        for slot, (B, r) in enumerate(self.passes):
-            x = x_override if x_override is not None else self._next_input()
-            self.one_pass(x, B, r, slot, timed_keys)
-        # hierarchical leg + de-quantization
-        x = x_override if x_override is not None else self._next_input()
-        mxq.mxq_tensor_amax(x, N_ELEM, self.amax, self.g)
-        mxq.mxq_quantize_ex(x, N_ELEM, 16, UE4M3, ABSMAX, 1.0, self.g, self.codes, self.scales, self.sse)
-        slot = len(self.passes)
-        mxq.mxq_tensor_mse(self.sse, N_ELEM // 16, N_ELEM, self.mse[slot:slot + 1], self.ws)
-        mxq.mxq_dequantize(self.codes, self.scales, N_ELEM, 16, UE4M3, 1.0, self.xhat)
+        x = x or self.x
+        slot = 0
+        leg_start = {}
+        prev_leg = None
+        g_for = {}
+        for leg, key, n, B, fmt, recipe, hier in self.passes:
+            if timed and leg != prev_leg:
+                if prev_leg is not None:
+                    e = self._ev(); e.record()
+                    self.leg_events.setdefault(prev_leg, []).append((leg_start[prev_leg], e))
+                leg_start[leg] = self._ev(); leg_start[leg].record()
+            prev_leg = leg
+            t = x[key]
+            dg = None
+            if hier:
+                if key not in g_for:             # hierarchical scaling: tensor abs-max -> g, on the device
+                    i = len(g_for)
+                    mxq.mxq_tensor_amax(t, n, self.amax[i:i + 1], self.g[i:i + 1])
+                    g_for[key] = self.g[i:i + 1]
+                dg = g_for[key]
+            ev = None
+            if timed and leg == "search":
+                ev = (self._ev(), self._ev())
+                ev[0].record()
+            mxq.mxq_quantize_ex(t, n, B, fmt, recipe, 1.0, dg, self.codes, self.scales, self.sse)
+            if ev is not None:
+                ev[1].record()
+                self.search_events.setdefault((B, fmt), []).append(ev)
+            mxq.mxq_tensor_mse(self.sse, n // B, n, self.mse[slot:slot + 1], self.ws)
+            slot += 1
+        # the last pass left UE5M3 / 4-over-6 codes of an activation tensor: de-quantize them
+        mxq.mxq_dequantize(self.codes, self.scales, ACT_N, 16, UE5M3, 1.0, self.xhat)
+        if timed:
+            e = self._ev(); e.record()
+            self.leg_events.setdefault(prev_leg, []).append((leg_start[prev_leg], e))
 
-    def kernel_ms(self, key):
-        evs = self.timers.get(key, [])
-        return (sum(a.elapsed_time(b) for a, b in evs) / len(evs)) if evs else None
+    def mean_ms(self, evs):
+        return sum(a.elapsed_time(b) for a, b in evs) / len(evs)
 
 
-def algorithmic_bytes(n: int, elem_bytes: int, B: int) -> float:
-    """Input + packed codes + scale bytes + block SSE of one fused quantize launch."""
-    return n * (elem_bytes + 0.5 + 5.0 / B)
+def graph_timed(torch, body, launches: int, reps: int = 5):
+    """Average duration (ms) of one launch of `body`'s launch sequence when it is replayed from a CUDA
+    graph (host launch overhead excluded), median over reps; also the plain Python-loop figure."""
+    body()
+    torch.cuda.synchronize()
+    loop = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); body(); e1.record()
+        torch.cuda.synchronize()
+        loop.append(e0.elapsed_time(e1) / launches)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        body()
+    torch.cuda.current_stream().wait_stream(s)
+    gr = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gr):
+        body()
+    gr.replay()
+    torch.cuda.synchronize()
+    rep = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); gr.replay(); e1.record()
+        torch.cuda.synchronize()
+        rep.append(e0.elapsed_time(e1) / launches)
+    del gr
+    return statistics.median(rep), statistics.median(loop)
+
+
+def hbm_entry(n, elem_bytes, B, ms, ms_loop, peaks, extra=None):
+    ach = algorithmic_bytes(n, elem_bytes, B) / (ms * 1e-3) / 1e9
+    d = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+         "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "ms_per_launch": ms, "ms_per_launch_python_loop": ms_loop,
+         "gelem_s": n / (ms * 1e-3) / 1e9, "elems": n, "peak_source": peaks["source"]}
+    if extra:
+        d.update(extra)
+    return d
+
+
+def config_size_rooflines(torch, mxq, wl, peaks):
+    """The one-pass kernels at the sizes of the step's own tensors: launches back to back over copies
+    of the tensor that together exceed L2, replayed from a CUDA graph (and as a plain Python loop)."""
+    out = {}
+    cases = [("w_q", 4096 * 4096), ("w_k", 1024 * 4096), ("w_gate", 14336 * 4096), ("act", ACT_N)]
+    for key, n in cases:
+        src = wl.x["a_0"] if key == "act" else wl.x[key]
+        ncopies = max(3, min(48, (512 << 20) // (n * 2)))
+        xs = [src] + [src.clone() for _ in range(ncopies - 1)]
+        for recipe in (ABSMAX, R4O6):
+            for B in (16, 8):
+                if B == 8 and key not in ("w_q", "w_gate"):
+                    continue
+                codes, scales, sse = mxq.alloc_outputs(n, B, src.device)
+
+                def body():
+                    for x in xs:
+                        mxq.mxq_quantize_ex(x, n, B, UE4M3, recipe, 1.0, None, codes, scales, sse)
+                ms, ms_loop = graph_timed(torch, body, len(xs))
+                out[f"{RECIPE_NAME[recipe]}_bf16_B{B}_{key}"] = hbm_entry(
+                    n, 2, B, ms, ms_loop, peaks, {"l2": f"{len(xs)} copies of the tensor, {len(xs) * n * 2 >> 20} MiB, round-robin"})
+        del xs
+    return out
 
 
 def streaming_rooflines(torch, mxq, device, peaks):
-    """HBM-bound kernels on a tensor far larger than L2 (134M elements), ten launches back to back
-    per CUDA-event pair, outside the timed region of the step: the 16.8M-element launches of the
-    step itself last 8-20 us and are dominated by launch ramp."""
+    """HBM-bound kernels on a tensor far larger than L2 (134M elements), launches back to back."""
     from paper_2605_08565_b200 import inputs
     out = {}
     n = STREAM_ELEMS
-
-    def entry(name, fn, nbytes, traffic):
-        for _ in range(3):
-            fn()
-        times = []
-        for _ in range(5):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(10):
-                fn()
-            e1.record()
-            torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1) / 10)
-        ms = statistics.median(times)
-        ach = nbytes / (ms * 1e-3) / 1e9
-        out[name] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0, "traffic": traffic,
-                     "ms_per_launch": ms, "gelem_s": n / (ms * 1e-3) / 1e9, "elems": n,
-                     "peak_source": peaks["source"], "l2": "input larger than L2"}
-
-    for name, dt, recipe, B, key in (
-            ("absmax_bf16_B16", torch.bfloat16, ABSMAX, 16, "k_quantize<bf16,B=16,UE4M3,absmax>@128Mi"),
-            ("4o6_bf16_B16", torch.bfloat16, R4O6, 16, "k_quantize<bf16,B=16,UE4M3,4o6>@128Mi"),
-            ("absmax_f32_B16", torch.float32, ABSMAX, 16, "k_quantize<f32,B=16,UE4M3,absmax>@128Mi"),
-            ("4o6_f32_B16", torch.float32, R4O6, 16, None),
-            ("absmax_bf16_B64", torch.bfloat16, ABSMAX, 64, None),
-            ("absmax_f32_B64", torch.float32, ABSMAX, 64, None)):
+    prof = {("bf16", ABSMAX): "k_quantize_absmax_bf16_B16_128Mi.txt", ("bf16", R4O6): "k_quantize_4o6_bf16_B16_128Mi.txt",
+            ("f32", ABSMAX): "k_quantize_absmax_f32_B16_128Mi.txt"}
+    for name, dt, recipe, B in (
+            ("absmax_bf16_B16", torch.bfloat16, ABSMAX, 16), ("4o6_bf16_B16", torch.bfloat16, R4O6, 16),
+            ("absmax_f32_B16", torch.float32, ABSMAX, 16), ("4o6_f32_B16", torch.float32, R4O6, 16),
+            ("absmax_bf16_B64", torch.bfloat16, ABSMAX, 64), ("4o6_bf16_B8", torch.bfloat16, R4O6, 8)):
         codes, scales, sse = mxq.alloc_outputs(n, B, device)
-        x = inputs.student_t(n, 5, 0.02, 2, dt, device)
-        fn = lambda: mxq.mxq_quantize_ex(x, n, B, UE4M3, recipe, 1.0, None, codes, scales, sse)
-        entry(name, fn, algorithmic_bytes(n, x.element_size(), B), NCU_TRAFFIC_BYTES[key] if key else None)
-        del x
-    # the other two kernels of the path: tensor abs-max (reads n elements) and de-quantization
+        xs = [inputs.student_t(n, 5, 0.02, 2 + i, dt, device) for i in range(2)]
+
+        def body():
+            for _ in range(3):
+                for x in xs:
+                    mxq.mxq_quantize_ex(x, n, B, UE4M3, recipe, 1.0, None, codes, scales, sse)
+        ms, ms_loop = graph_timed(torch, body, 6)
+        rec = recorded_profile(prof.get(("bf16" if dt == torch.bfloat16 else "f32", recipe), "-"),
+                               ("mxq_quantize.cuh", "mxq_device.cuh")) if B == 16 else None
+        extra = {"l2": "input larger than L2"}
+        if rec is not None:
+            extra.update(traffic=rec["dram_bytes"], traffic_source=rec["file"], traffic_stale=rec["stale"])
+        out[name] = hbm_entry(n, xs[0].element_size(), B, ms, ms_loop, peaks, extra)
+        del xs
     x = inputs.student_t(n, 5, 0.02, 2, torch.bfloat16, device)
     amax = torch.empty(1, dtype=torch.float32, device=device)
-    entry("tensor_amax_bf16", lambda: mxq.mxq_tensor_amax(x, n, amax), n * 2.0, None)
+
+    def body_amax():
+        for _ in range(6):
+            mxq.mxq_tensor_amax(x, n, amax)
+    ms, ms_loop = graph_timed(torch, body_amax, 6)
+    ach = n * 2.0 / (ms * 1e-3) / 1e9
+    out["tensor_amax_bf16"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
+                               "ms_per_launch": ms, "ms_per_launch_python_loop": ms_loop, "elems": n}
     codes, scales, sse = mxq.alloc_outputs(n, 16, device)
     mxq.mxq_quantize_ex(x, n, 16, UE4M3, ABSMAX, 1.0, None, codes, scales, sse)
     xh = torch.empty(n, dtype=torch.float32, device=device)
-    entry("dequantize_B16_to_f32", lambda: mxq.mxq_dequantize(codes, scales, n, 16, UE4M3, 1.0, xh), n * (0.5 + 1.0 / 16 + 4.0), None)
+
+    def body_deq():
+        for _ in range(6):
+            mxq.mxq_dequantize(codes, scales, n, 16, UE4M3, 1.0, xh)
+    ms, ms_loop = graph_timed(torch, body_deq, 6)
+    ach = n * (0.5 + 1.0 / 16 + 4.0) / (ms * 1e-3) / 1e9
+    out["dequantize_B16_to_f32"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                    "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
+                                    "ms_per_launch": ms, "ms_per_launch_python_loop": ms_loop, "elems": n}
     return out
 
 
 def pruned_sweep_report(torch, mxq, wl):
-    """The brute-force passes of the step once more with the pruned sweep switched on (outside the
-    timed region; `value` and `roofline` are always the full sweep): per block size the time of both
-    sweeps over the rotating tensors, launches back to back, and whether the outputs are identical."""
+    """The 15 brute-force sweeps of the step once more with the pruned sweep switched on (outside the timed
+    region; `value` and `roofline` are always the full sweep): per sweep the time of both modes on the same
+    tensor and whether every output byte is identical."""
     out = {}
-    x0 = wl.x[0]
-    n = x0.numel()
+    x = wl.x["search"]
+    n = x.numel()
+    dg = wl.g[0:1]
+    mxq.mxq_tensor_amax(x, n, wl.amax[0:1], dg)
     try:
-        for B in BLOCKS:
-            bufs = {}
-            ms = {}
-            for mode in (0, 1):
-                mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, mode)
-                codes, scales, sse = mxq.alloc_outputs(n, B, x0.device)
-                fn = lambda x: mxq.mxq_quantize_ex(x, n, B, UE4M3, BRUTE, 1.0, None, codes, scales, sse)
-                fn(x0)
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                for x in wl.x:
-                    fn(x)
-                e1.record()
-                fn(x0)
-                torch.cuda.synchronize()
-                ms[mode] = e0.elapsed_time(e1) / len(wl.x)
-                bufs[mode] = (codes, scales, sse)
-            same = all(torch.equal(a.view(torch.uint8), b.view(torch.uint8)) for a, b in zip(bufs[0], bufs[1]))
-            out[f"B{B}"] = {"full_ms": ms[0], "pruned_ms": ms[1], "speedup": ms[0] / ms[1], "outputs_identical": bool(same)}
+        for B in SEARCH_BLOCKS:
+            for fmt in SEARCH_FMTS:
+                res = {}
+                ms = {}
+                for mode in (0, 1):
+                    mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, mode)
+                    codes, scales, sse = mxq.alloc_outputs(n, B, x.device)
+                    mxq.mxq_quantize_ex(x, n, B, fmt, BRUTE, 1.0, dg, codes, scales, sse)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    mxq.mxq_quantize_ex(x, n, B, fmt, BRUTE, 1.0, dg, codes, scales, sse)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ms[mode] = e0.elapsed_time(e1)
+                    res[mode] = (codes, scales, sse)
+                same = all(torch.equal(a.view(torch.uint8), b.view(torch.uint8)) for a, b in zip(res[0], res[1]))
+                out[f"B{B}_{FMT_NAME[fmt]}"] = {"full_ms": ms[0], "pruned_ms": ms[1], "speedup": ms[0] / ms[1],
+                                               "outputs_identical": bool(same)}
+                del res
     finally:
         mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 0)
     return out
+
+
+def spawn_ranks(args) -> int:
+    """`--gpus N` without a torchrun environment: start the N ranks on this node and relay their output."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def run_gpu(args) -> None:
@@ -358,12 +538,9 @@ def run_gpu(args) -> None:
     peaks = measured_peaks()
 
     wl = Workload(rank, device)
-    hot = {(16, BRUTE), (16, ABSMAX), (16, R4O6)}   # kernels timed live for the roofline entries
-
     for _ in range(args.warmup):
         wl.step()
     torch.cuda.synchronize()
-    wl.timers.clear()
 
     # ---- device-resident timing ---------------------------------------------------------------
     try:
@@ -379,7 +556,7 @@ def run_gpu(args) -> None:
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
-        wl.step(timed_keys=hot)
+        wl.step(timed=True)
     e1.record()
     torch.cuda.synchronize()
     dist.barrier()
@@ -389,13 +566,14 @@ def run_gpu(args) -> None:
     value, t_max = dist.whole_job_throughput(wl.elems_per_step * args.steps, local_s)
     mse_host = wl.mse.cpu().numpy().copy()
 
-    # ---- end to end: host buffers, H2D of the step's input and D2H of its results every step ----
-    # The input of step i + 1 is copied on a second stream into the other of two device buffers while
+    # ---- end to end: host buffers, H2D of the step's inputs and D2H of its results every step ----
+    # The inputs of step i + 1 are copied on a second stream into the other of two device sets while
     # step i computes; every copy is awaited by the compute stream, so all of them lie inside the
     # timed region.
-    host_in = wl.x[0].cpu().pin_memory()
+    host_in = {k: v.cpu().pin_memory() for k, v in wl.x.items()}
+    h2d_bytes = sum(v.numel() * v.element_size() for v in host_in.values())
     host_out = torch.empty(wl.mse.numel(), dtype=torch.float64).pin_memory()
-    dev_in = [torch.empty_like(wl.x[0]), torch.empty_like(wl.x[0])]
+    dev_in = [{k: torch.empty_like(v) for k, v in wl.x.items()} for _ in range(2)]
     copy_stream = torch.cuda.Stream(device=device)
     main_stream = torch.cuda.current_stream(device)
 
@@ -408,7 +586,8 @@ def run_gpu(args) -> None:
         def enqueue_copy(i):
             with torch.cuda.stream(copy_stream):
                 copy_stream.wait_event(free[i % 2])
-                dev_in[i % 2].copy_(host_in, non_blocking=True)
+                for k, v in host_in.items():
+                    dev_in[i % 2][k].copy_(v, non_blocking=True)
                 ready[i % 2].record(copy_stream)
 
         enqueue_copy(0)
@@ -416,78 +595,323 @@ def run_gpu(args) -> None:
             if i + 1 < n_steps:
                 enqueue_copy(i + 1)
             main_stream.wait_event(ready[i % 2])
-            wl.step(x_override=dev_in[i % 2])
+            wl.step(x=dev_in[i % 2])
             free[i % 2].record(main_stream)
             host_out.copy_(wl.mse, non_blocking=True)
 
+    e2e_steps = max(2, min(args.steps, 10))
     e2e_loop(2)
     torch.cuda.synchronize()
     dist.barrier()
     e0.record()
-    e2e_loop(args.steps)
+    e2e_loop(e2e_steps)
     e1.record()
     torch.cuda.synchronize()
     dist.barrier()
-    e2e_value, _ = dist.whole_job_throughput(wl.elems_per_step * args.steps, e0.elapsed_time(e1) / 1e3)
+    e2e_value, _ = dist.whole_job_throughput(wl.elems_per_step * e2e_steps, e0.elapsed_time(e1) / 1e3)
+    del dev_in
+
+    # ---- end to end, second form: one abs-max pass whose codes and scale bytes go back to the host ----
+    nq = 14336 * 4096
+    hq_in = host_in["w_gate"]
+    dq_in = torch.empty_like(wl.x["w_gate"])
+    cq, sq, _ = mxq.alloc_outputs(nq, 16, device, with_sse=False)
+    hq_codes = torch.empty(nq // 2, dtype=torch.uint8).pin_memory()
+    hq_scales = torch.empty(nq // 16, dtype=torch.uint8).pin_memory()
+
+    def to_host_loop(k):
+        for _ in range(k):
+            dq_in.copy_(hq_in, non_blocking=True)
+            mxq.mxq_quantize_ex(dq_in, nq, 16, UE4M3, ABSMAX, 1.0, None, cq, sq, None)
+            hq_codes.copy_(cq, non_blocking=True)
+            hq_scales.copy_(sq, non_blocking=True)
+    to_host_loop(2)
+    torch.cuda.synchronize()
+    dist.barrier()
+    e0.record()
+    to_host_loop(10)
+    e1.record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    q2h_value, _ = dist.whole_job_throughput(float(nq) * 10, e0.elapsed_time(e1) / 1e3)
 
     if rank != 0:
         dist.shutdown()
         return
 
-    # ---- rooflines of the kernels timed live --------------------------------------------------
+    # ---- roofline of the dominant kernel: every brute-force launch of the step, time-weighted ----
     sm_mhz = (clocks or {}).get("sm_mhz") or peaks["sm_max_mhz"]
     n_sm = torch.cuda.get_device_properties(device).multi_processor_count
-    alu_peak_max = n_sm * ALU_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12          # Tlaneop/s at max clock
-    brute_ms = wl.kernel_ms((16, BRUTE))
-    brute_ops = N_ELEM * N_CODES_UE4M3 * 4.0                                            # 4 lane-ops per element-code
-    brute_ach = brute_ops / (brute_ms * 1e-3) / 1e12
-    roofline = {"kernel": "k_brute<bf16,B=16,UE4M3>", "bound": "alu", "achieved": brute_ach, "peak": alu_peak_max,
-                "unit": "Tlaneop/s", "frac": brute_ach / alu_peak_max,
-                "traffic": NCU_TRAFFIC_BYTES["k_brute<bf16,B=16,UE4M3>@16Mi"],
+    alu_peak = n_sm * ALU_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12          # Tlaneop/s at the maximum SM clock
+    per_inst, tot_ops, tot_ms = {}, 0.0, 0.0
+    for (B, fmt), evs in wl.search_events.items():
+        ms = wl.mean_ms(evs)
+        ops = SEARCH_N * N_CODES[fmt] * 4.0                                        # 4 lane-ops per (element, code)
+        per_inst[f"B{B}_{FMT_NAME[fmt]}"] = {"ms_per_launch": ms, "achieved": ops / (ms * 1e-3) / 1e12,
+                                             "frac": ops / (ms * 1e-3) / 1e12 / alu_peak,
+                                             "gelem_s": SEARCH_N / (ms * 1e-3) / 1e9}
+        tot_ops += ops
+        tot_ms += ms
+    step_ms = t_max / args.steps * 1e3
+    largest = max(per_inst, key=lambda k: per_inst[k]["ms_per_launch"])
+    rec = recorded_profile("k_brute_f32_B16_ue4m3_tensor_scale_16Mi.txt", ("mxq_brute.cuh", "mxq_device.cuh"))
+    traffic = None
+    if rec["dram_bytes"] is not None and rec["elems"]:
+        traffic = rec["dram_bytes"] * SEARCH_N / rec["elems"]      # input and outputs grow in proportion to the elements
+    roofline = {"kernel": "k_brute<f32, B, fmt> full sweep, tensor scale: the 15 launches of a step, time-weighted",
+                "bound": "alu", "achieved": tot_ops / (tot_ms * 1e-3) / 1e12, "peak": alu_peak, "unit": "Tlaneop/s",
+                "frac": tot_ops / (tot_ms * 1e-3) / 1e12 / alu_peak,
+                "frac_at_observed_clock": tot_ops / (tot_ms * 1e-3) / 1e12 / (n_sm * ALU_LANES_PER_SM * sm_mhz * 1e6 / 1e12),
+                "traffic": traffic, "traffic_source": rec["file"] + " (16.8M-element capture scaled to 268M elements)",
+                "traffic_stale": rec["stale"], "ncu_issue_active_pct_recorded": rec["issue_active_pct"],
                 "peak_source": f"{n_sm} SMs x 128 lanes x {peaks['sm_max_mhz']:.0f} MHz (max SM clock, {peaks['source']})",
-                "frac_at_observed_clock": brute_ach / (n_sm * ALU_LANES_PER_SM * sm_mhz * 1e6 / 1e12),
-                "ms_per_launch": brute_ms, "ncu_issue_active_pct": NCU_BRUTE_ISSUE_ACTIVE_PCT}
-    hbm = {}
-    for name, key in (("absmax_B16", (16, ABSMAX)), ("4o6_B16", (16, R4O6))):
-        ms = wl.kernel_ms(key)
-        ach = algorithmic_bytes(N_ELEM, 2, 16) / (ms * 1e-3) / 1e9
-        hbm[name] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": ach / 8000.0, "traffic": None,
-                     "ms_per_launch": ms, "gelem_s": N_ELEM / (ms * 1e-3) / 1e9, "peak_source": peaks["source"]}
-    streaming = None if args.skip_streaming else streaming_rooflines(torch, mxq, device, peaks)
-    pruned = None if args.skip_streaming else pruned_sweep_report(torch, mxq, wl)
-    per_recipe = {"brute_B16": N_ELEM / (brute_ms * 1e-3) / 1e9, "absmax_B16": hbm["absmax_B16"]["gelem_s"],
-                  "4o6_B16": hbm["4o6_B16"]["gelem_s"]}
+                "launches_per_step": len(per_inst), "ms_per_launch": tot_ms / len(per_inst),
+                "ms_all_launches_per_step": tot_ms, "share_of_step_time": tot_ms / step_ms,
+                "largest_share": largest, "per_instantiation": per_inst}
+    legs = {leg: {"ms_per_step": wl.mean_ms(evs),
+                  "gelem_s": sum(p[2] for p in wl.passes if p[0] == leg) / (wl.mean_ms(evs) * 1e-3) / 1e9}
+            for leg, evs in wl.leg_events.items()}
+
+    hbm = None if args.skip_extras else config_size_rooflines(torch, mxq, wl, peaks)
+    streaming = None if args.skip_extras else streaming_rooflines(torch, mxq, device, peaks)
+    pruned = None if args.skip_extras else pruned_sweep_report(torch, mxq, wl)
 
     # ---- CPU oracle on a bounded sample of the same workload ------------------------------------
     from oracle import mxq_oracle as orc
+    from paper_2605_08565_b200 import inputs
     orc.build()
     threads = host_threads()
-    sample = host_sample(dist.rank_seed(2, 0, 0), CPU_SAMPLE_ELEMS)
-    oracle_sample_run(sample[: 1 << 12], threads)
-    c_elems, c_secs = oracle_sample_run(sample, threads)
-    cpu_baseline = {"value": c_elems / c_secs / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
-                    "seconds": c_secs,
-                    "sample": f"first {CPU_SAMPLE_ELEMS} elements of tensor 0, every pass of one step"}
+    samples = {k: inputs.to_numpy_bits(v[:CPU_SAMPLE_ELEMS]) for k, v in wl.x.items()}
+    oracle_step(samples, threads, 4096.0 / CPU_SAMPLE_ELEMS)
+    c_elems, c_secs = oracle_step(samples, threads)
+    cpu_baseline = {"value": c_elems / c_secs / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": c_secs,
+                    "sample": f"first {CPU_SAMPLE_ELEMS} elements of every tensor of the step, every pass of one step"}
 
+    names = [f"{leg}:{key}:B{B}:{FMT_NAME[fmt]}:{RECIPE_NAME[r]}" + (":g" if hier else "")
+             for leg, key, _, B, fmt, r, hier in wl.passes]
     print(json.dumps({
         "metric": METRIC, "value": value / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": t_max / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "weight sweep: 4096x4096 bf16 0.02*Student-t(5), UE4M3 block scales, g=1, "
-                               "B in {2,4,8,16,32,64} x {abs-max, abs-max+pz, 4-over-6, brute force} + MSE each; "
-                               "+ hierarchical leg (amax, g, abs-max B=16, MSE) + dequantize",
-                   "elements_per_step": wl.elems_per_step, "passes_per_step": len(wl.passes) + 1,
-                   "l2": f"inputs rotate over {N_ROTATE} tensors (256 MiB) > 126 MB L2"},
-        "roofline": roofline, "roofline_hbm": hbm, "roofline_hbm_streaming": streaming,
-        "per_recipe_gelem_s": per_recipe, "brute_pruned_sweep": pruned,
-        "cpu_baseline": cpu_baseline,
-        "e2e": {"value": e2e_value / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(host_in.numel() * 2),
-                "d2h_bytes_per_step": int(host_out.numel() * 8)},
+        "config": {"workload": WORKLOAD_NAME, "elements_per_step": wl.elems_per_step, "passes_per_step": len(wl.passes),
+                   "l2": "search tensor 1 GiB > 126 MB L2; the legs walk their tensors round-robin (277 MB and 201 MB sets)"},
+        "roofline": roofline, "legs": legs, "roofline_hbm": hbm, "roofline_hbm_streaming": streaming,
+        "brute_pruned_sweep": pruned, "cpu_baseline": cpu_baseline,
+        "e2e": {"value": e2e_value / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(h2d_bytes),
+                "d2h_bytes_per_step": int(host_out.numel() * 8), "steps": e2e_steps,
+                "what": "the same step with all inputs copied from pinned host memory every step (overlapped with the "
+                        "previous step) and the per-pass MSE values copied back"},
+        "e2e_quantize_to_host": {"value": q2h_value / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(nq * 2),
+                                 "d2h_bytes_per_step": int(nq // 2 + nq // 16),
+                                 "what": "one abs-max pass (14336x4096 bf16, B=16, UE4M3): input from pinned host memory, "
+                                         "codes and scale bytes back to pinned host memory, one stream, no overlap"},
         "gpu_launches": int(launches), "clocks": clocks,
-        "mse_by_block_size": {RECIPE_NAME[r] + f"_B{B}": float(mse_host[i]) for i, (B, r) in enumerate(wl.passes)},
+        "mse": {nm: float(mse_host[i]) for i, nm in enumerate(names)},
     }))
     dist.shutdown()
+
+
+# ------------------------------------------------------------------------------------------------
+# --config: the five benchmark configurations, one recipe at a time
+# ------------------------------------------------------------------------------------------------
+class _Acc:
+    """CUDA-event time and elements per (B, fmt, recipe, tensor-scale) key.  A key's tensors are quantized
+    back to back inside one event pair (after one untimed launch), `rounds` times over; the tensor MSE is
+    taken afterwards, untimed."""
+
+    def __init__(self, torch, mxq):
+        self.torch, self.mxq = torch, mxq
+        self.ms, self.elems, self.mse = {}, {}, {}
+
+    def run(self, key, xs, B, fmt, recipe, g, dgs, bufs, rounds=1):
+        self._run(key, xs, B, fmt, recipe, g, dgs, bufs, rounds)
+        if recipe in (BRUTE, BRUTE_PZ):   # the same pass with the pruned sweep, as a row of its own
+            self.mxq.mxq_set_option(self.mxq.MXQ_OPT_BRUTE_PRUNE, 1)
+            try:
+                self._run(key + ("pruned",), xs, B, fmt, recipe, g, dgs, bufs, rounds)
+            finally:
+                self.mxq.mxq_set_option(self.mxq.MXQ_OPT_BRUTE_PRUNE, 0)
+
+    def _run(self, key, xs, B, fmt, recipe, g, dgs, bufs, rounds):
+        torch, mxq = self.torch, self.mxq
+        codes, scales, sse, mse_out, ws = bufs
+        dgs = dgs if dgs is not None else [None] * len(xs)
+        mxq.mxq_quantize_ex(xs[0], xs[0].numel(), B, fmt, recipe, g, dgs[0], codes, scales, sse)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(rounds):
+            for x, dg in zip(xs, dgs):
+                mxq.mxq_quantize_ex(x, x.numel(), B, fmt, recipe, g, dg, codes, scales, sse)
+        e1.record()
+        tot, cnt = 0.0, 0
+        for x, dg in zip(xs, dgs):
+            mxq.mxq_quantize_ex(x, x.numel(), B, fmt, recipe, g, dg, codes, scales, sse)
+            mxq.mxq_tensor_mse(sse, x.numel() // B, x.numel(), mse_out, ws)
+            tot += float(mse_out.cpu()[0]) * x.numel()
+            cnt += x.numel()
+        torch.cuda.synchronize()
+        self.ms[key] = self.ms.get(key, 0.0) + e0.elapsed_time(e1)
+        self.elems[key] = self.elems.get(key, 0) + cnt * rounds
+        m = self.mse.setdefault(key, [0.0, 0])
+        m[0] += tot
+        m[1] += cnt
+
+    def rows(self, cfg, elem_bytes, hbm_gbs, alu_peak):
+        out = []
+        for key, ms in self.ms.items():
+            B, fmt, recipe, gk = key[:4]
+            pruned = len(key) > 4
+            n = self.elems[key]
+            ge = n / ms / 1e6
+            row = {"config": cfg, "block": B, "scale_fmt": FMT_NAME[fmt],
+                   "recipe": RECIPE_NAME[recipe] + ("+prune" if pruned else ""), "tensor_scale": gk,
+                   "elements": n, "ms": ms, "gelem_s": ge, "mse": self.mse[key][0] / self.mse[key][1]}
+            if pruned:
+                # codes left out are not work done: no roofline fraction, only the speed-up over the full sweep
+                full = self.elems[key[:4]] / self.ms[key[:4]] / 1e6
+                row.update(bound="alu", speedup_over_full_sweep=ge / full, frac=None)
+            elif recipe in (BRUTE, BRUTE_PZ):
+                ach = ge * 1e9 * N_CODES[fmt] * 4 / 1e12
+                row.update(bound="alu", achieved_tlaneop_s=ach, frac=ach / alu_peak)
+            else:
+                ach = ge * (elem_bytes + 0.5 + 5.0 / B)
+                row.update(bound="hbm", achieved_gb_s=ach, frac=ach / hbm_gbs, frac_of_8tbs=ach / NOMINAL_HBM_GBS)
+            out.append(row)
+        return out
+
+
+class _InputDigest:
+    """SHA-256 over the bytes of a configuration's input tensors, in generation order (so that a run
+    can be tied to the exact inputs it quantized); computed on the host, only when asked for."""
+
+    def __init__(self, enabled):
+        self.h = hashlib.sha256() if enabled else None
+        self.tensors, self.elements = 0, 0
+
+    def add(self, x):
+        import torch
+        self.tensors += 1
+        self.elements += x.numel()
+        if self.h is not None:
+            self.h.update(x.view(torch.uint8).cpu().numpy().tobytes())
+
+    def result(self):
+        return {"tensors": self.tensors, "elements": self.elements,
+                "sha256": self.h.hexdigest() if self.h is not None else None}
+
+
+def run_configs(configs, hash_inputs=False):
+    """Times every (configuration, block size, scale format, recipe) of the five benchmark configurations
+    at full size: the quantize pass with CUDA events as it is called from Python (launches back to back;
+    tensors larger than L2 or rotated so that inputs come from HBM), the tensor MSE afterwards."""
+    import torch
+    from paper_2605_08565_b200 import binding as mxq
+    from paper_2605_08565_b200 import inputs
+    if not torch.cuda.is_available():
+        raise mxq.MxqError("needs a CUDA device (no CPU fallback)")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    hbm, mhz = peaks["hbm_gbs"], peaks["sm_max_mhz"]
+    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+    alu_peak = n_sm * ALU_LANES_PER_SM * mhz * 1e6 / 1e12
+    A, P, R4, R4P, BR, BRP = ABSMAX, ABSMAX_PZ, R4O6, R4O6_PZ, BRUTE, BRUTE_PZ
+    rows, digests = [], {}
+
+    def bufs(n, B):
+        codes, scales, sse = mxq.alloc_outputs(n, B, dev)
+        return (codes, scales, sse, torch.empty(1, dtype=torch.float64, device=dev),
+                torch.empty(mxq.mxq_tensor_mse_workspace_bytes(n // B) // 8, dtype=torch.float64, device=dev))
+
+    def tensor_scale(x):
+        amax = torch.empty(1, dtype=torch.float32, device=dev)
+        dg = torch.empty(1, dtype=torch.float32, device=dev)
+        mxq.mxq_tensor_amax(x, x.numel(), amax, dg)
+        return dg
+
+    warm = inputs.normal(1 << 20, 0, 1.0, torch.float32, dev)          # first-launch costs out of the way
+    for r in (A, R4, BR):
+        mxq.quantize(warm, 16, UE4M3, r)
+
+    if 1 in configs:   # 1024 x 1024 fp32 N(0,1), B=16, UE4M3 + tensor scale; 4 MB: L2-resident, launch-bound
+        x = inputs.normal(1024 * 1024, 1, 1.0, torch.float32, dev)
+        digests["C1"] = _InputDigest(hash_inputs)
+        digests["C1"].add(x)
+        dg = tensor_scale(x)
+        acc, b = _Acc(torch, mxq), bufs(x.numel(), 16)
+        for r in (A, R4, BR):
+            acc.run((16, UE4M3, r, "amax/2688"), [x], 16, UE4M3, r, 1.0, [dg], b, rounds=50)
+        rows += acc.rows("C1 1024x1024 fp32 N(0,1)", 4, hbm, alu_peak)
+
+    if 2 in configs:   # 4096 x 4096 bf16 0.02 * t5, all block sizes, UE4M3, no tensor scale; 8 rotating tensors
+        xs = [inputs.student_t(4096 * 4096, 5, 0.02, 2 * 1_000_003 + i, torch.bfloat16, dev) for i in range(8)]
+        digests["C2"] = _InputDigest(hash_inputs)
+        for x in xs:
+            digests["C2"].add(x)
+        acc = _Acc(torch, mxq)
+        for B in (2, 4, 8, 16, 32, 64):
+            b = bufs(xs[0].numel(), B)
+            for r in (A, P, R4, BR):
+                acc.run((B, UE4M3, r, "none"), xs, B, UE4M3, r, 1.0, None, b, rounds=4 if r != BR else 1)
+        rows += acc.rows("C2 4096x4096 bf16 0.02*t5", 2, hbm, alu_peak)
+        del xs
+
+    if 3 in configs:   # 8192 x 4096 bf16 N(0,1) with 1 % outlier columns x50, B=16; 4 rotating tensors
+        xs = [inputs.outlier_columns(8192, 4096, 3 + i, dtype=torch.bfloat16, device=dev) for i in range(4)]
+        digests["C3"] = _InputDigest(hash_inputs)
+        for x in xs:
+            digests["C3"].add(x)
+        dgs = [tensor_scale(x) for x in xs]
+        acc, b = _Acc(torch, mxq), bufs(xs[0].numel(), 16)
+        for r in (A, R4):
+            acc.run((16, UE4M3, r, "amax/2688"), xs, 16, UE4M3, r, 1.0, dgs, b, rounds=4)
+            acc.run((16, UE5M3, r, "none"), xs, 16, UE5M3, r, 1.0, None, b, rounds=4)
+        rows += acc.rows("C3 8192x4096 bf16 outlier columns", 2, hbm, alu_peak)
+        del xs
+
+    if 4 in configs:   # Llama-3-8B-shaped weight set, 224 matrices, one at a time
+        acc = _Acc(torch, mxq)
+        digests["C4"] = _InputDigest(hash_inputs)
+        for layer in range(inputs.LLAMA8B_LAYERS):
+            for idx, (name, rows_, cols) in enumerate(inputs.LLAMA8B_LAYER_SHAPES):
+                x = inputs.student_t(rows_ * cols, 4, 1.0 / math.sqrt(cols), 4 + layer * 7 + idx, torch.bfloat16, dev)
+                digests["C4"].add(x)
+                for B in (8, 16):
+                    b = bufs(x.numel(), B)
+                    for fmt in (UE4M3, UE5M3):
+                        for r in (A, P, R4, R4P, BR, BRP):
+                            acc.run((B, fmt, r, "none"), [x], B, fmt, r, 1.0, None, b)
+                del x
+        rows += acc.rows("C4 Llama-3-8B-shaped set (224 matrices, 6.98 G elements)", 2, hbm, alu_peak)
+
+    if 5 in configs:   # 16384 x 16384 fp32 Laplace, brute force, tensor scale
+        x = inputs.laplace(16384 * 16384, 5, torch.float32, dev)
+        digests["C5"] = _InputDigest(hash_inputs)
+        digests["C5"].add(x)
+        dg = tensor_scale(x)
+        acc = _Acc(torch, mxq)
+        for B in (2, 4, 8, 16, 32):
+            b = bufs(x.numel(), B)
+            for fmt in (UE8M0, UE4M3, UE5M3):
+                acc.run((B, fmt, BR, "amax/2688"), [x], B, fmt, BR, 1.0, [dg], b)
+        rows += acc.rows("C5 16384x16384 fp32 Laplace", 4, hbm, alu_peak)
+    return {"hbm_gbs": hbm, "alu_peak_tlaneop_s": alu_peak, "peak_source": peaks["source"], "rows": rows,
+            "inputs": {k: d.result() for k, d in digests.items()}}
+
+
+def run_config_mode(args) -> None:
+    configs = (1, 2, 3, 4, 5) if args.config == "all" else tuple(int(c) for c in args.config.split(","))
+    res = run_configs(configs, hash_inputs=args.hash_inputs)
+    for r in res["rows"]:
+        head = (f'{r["config"][:28]:28s} B={r["block"]:<2d} {r["scale_fmt"]:5s} {r["recipe"]:14s} g={r["tensor_scale"]:9s} '
+                f'{r["gelem_s"]:9.1f} GElem/s  ')
+        if r["frac"] is None:
+            print(head + f'{r["speedup_over_full_sweep"]:8.2f} x the full sweep{"":14s}  mse={r["mse"]:.4e}', file=sys.stderr)
+            continue
+        ach = r.get("achieved_gb_s", r.get("achieved_tlaneop_s"))
+        unit = "GB/s" if r["bound"] == "hbm" else "Tlop/s"
+        print(head + f'{ach:8.1f} {unit:6s} {100 * r["frac"]:5.1f}% of {r["bound"]}  mse={r["mse"]:.4e}', file=sys.stderr)
+    print(json.dumps(res))
 
 
 def run_single_kernel(args) -> None:
@@ -525,6 +949,12 @@ def run_single_kernel(args) -> None:
         mxq.mxq_quantize_ex(x, n, B, fmt, 0, g, None, codes, scales, sse)
         fn = lambda: mxq.mxq_dequantize(codes, scales, n, B, fmt, g, out)
         nbytes = n * (eb + 0.5 + 1.0 / B)
+    elif args.kernel == "hist":
+        mxq.mxq_quantize_ex(x, n, B, fmt, 0, g, None, codes, scales, sse)
+        ch = torch.zeros(16, dtype=torch.int64, device=dev)
+        sh = torch.zeros(256, dtype=torch.int64, device=dev)
+        fn = lambda: mxq.mxq_histograms(codes, scales, n, B, ch, sh)
+        nbytes = n * (0.5 + 1.0 / B)
     else:
         raise SystemExit(f"unknown --kernel {args.kernel}")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if n * eb < (256 << 20) else None
@@ -543,14 +973,15 @@ def run_single_kernel(args) -> None:
            "gelem_s": n / ms / 1e6, "algorithmic_gb_s": nbytes / ms / 1e6,
            "l2": "flushed between iterations" if flush is not None else "input larger than L2"}
     if recipe in (4, 5):
-        ncodes = 127 if fmt == 1 else 255
-        res["tlaneop_s"] = n * ncodes * 4.0 / (ms * 1e-3) / 1e12
+        res["tlaneop_s"] = n * N_CODES[fmt] * 4.0 / (ms * 1e-3) / 1e12
     print(json.dumps(res))
 
 
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default=None, help="time one kernel alone: absmax|absmax_pz|4o6|4o6_pz|brute|brute_pz|amax|mse|dequant")
+    ap.add_argument("--kernel", default=None, help="time one kernel alone: absmax|absmax_pz|4o6|4o6_pz|brute|brute_pz|amax|mse|dequant|hist")
+    ap.add_argument("--config", default=None, help="time one benchmark configuration (1..5, comma list, or all), one recipe at a time")
+    ap.add_argument("--hash-inputs", action="store_true", help="with --config: record the SHA-256 of every configuration's input bytes")
     ap.add_argument("--block", type=int, default=16)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--fmt", default="ue4m3", choices=["ue8m0", "ue4m3", "ue5m3"])
@@ -559,22 +990,27 @@ def main() -> None:
     ap.add_argument("--global-scale", type=float, default=1.0)
     ap.add_argument("--prune", action="store_true", help="with --kernel brute|brute_pz: the pruned sweep")
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--skip-streaming", action="store_true",
-                    help="leave out the measurements taken outside the timed step: the 134M-element streaming "
-                         "launches and the pruned brute-force sweep (roofline_hbm_streaming, brute_pruned_sweep = null)")
+    ap.add_argument("--skip-extras", action="store_true",
+                    help="leave out the measurements taken outside the timed step (roofline_hbm, roofline_hbm_streaming, "
+                         "brute_pruned_sweep = null)")
     ap.add_argument("--impl", default="mxq", choices=["mxq", "reference"])
     args = ap.parse_args()
     if args.kernel:
         run_single_kernel(args)
         return
+    if args.config:
+        run_config_mode(args)
+        return
     if args.warmup < 3 and args.impl == "mxq":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_gpu(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
+    run_gpu(args)
 
 
 if __name__ == "__main__":

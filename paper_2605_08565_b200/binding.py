@@ -12,7 +12,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmxq.so")
+# MXQ_LIB: load another build of the library (kernel experiments); the default is the in-tree build
+LIB_PATH = os.environ.get("MXQ_LIB") or os.path.join(_HERE, "libmxq.so")
 
 MXQ_F32, MXQ_BF16 = 0, 1
 MXQ_SF_UE8M0, MXQ_SF_UE4M3, MXQ_SF_UE5M3 = 0, 1, 2

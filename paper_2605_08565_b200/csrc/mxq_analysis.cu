@@ -18,6 +18,7 @@ template <int DT, int B>
 __global__ void __launch_bounds__(kThreads) k_block_clip_sse(const void* x, size_t n_blocks, int fmt, float g,
                                                              const float* d_g, const uint8_t* scales, float* out) {
     wait_for_prior_grid();
+    release_dependents();
     const float gs = d_g ? *d_g : g;
     const size_t stride = (size_t)gridDim.x * kThreads;
     for (size_t b = (size_t)blockIdx.x * kThreads + threadIdx.x; b < n_blocks; b += stride) {

@@ -454,6 +454,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
 
     __shared__ BruteTables T;
     wait_for_prior_grid();
+    release_dependents();
     const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
     const int first = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     build_brute_tables<FMT, PRUNE>(T, g, first);

@@ -19,6 +19,18 @@ constexpr int kThreads = 256;
 // has completed and its writes are visible.
 __device__ __forceinline__ void wait_for_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Lets the next kernel of the stream (if it was launched with programmatic stream serialization) be
+// staged onto SM resources as they become free, so that its launch latency and prologue overlap
+// this kernel's tail.  It still blocks in its own wait_for_prior_grid() until this grid has
+// completed and flushed its writes, so the ordering of a plain stream is kept.  The dependent grid
+// is released only after EVERY CTA of this grid has executed this instruction (or exited), i.e.
+// when all of them are resident or done: the staged CTAs can never keep this grid off the SMs.
+__device__ __forceinline__ void release_dependents() {
+#ifndef MXQ_NO_EARLY_RELEASE
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#endif
+}
+
 __host__ __device__ constexpr int num_codes(int fmt) { return fmt == kUE4M3 ? 127 : 255; }
 __host__ __device__ constexpr int elem_bytes(int dt) { return dt == kF32 ? 4 : 2; }
 

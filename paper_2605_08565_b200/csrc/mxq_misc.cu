@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(kThreads) k_tensor_amax(const void* x, size_t 
 // g = amax / (6 * 448): the tensor maximum maps to the top of FP4 times the top of E4M3.
 __global__ void k_global_scale(const float* amax, float* g) {
     wait_for_prior_grid();
+    release_dependents();
     const float a = *amax;
     *g = (a > 0.0f && a <= 3.402823466e38f) ? __fdiv_rn(a, 2688.0f) : 1.0f;
 }
@@ -119,6 +120,7 @@ __device__ __forceinline__ double cta_tree_sum(double v, double* sh) {
 __global__ void __launch_bounds__(kThreads) k_mse_partial(const float* sse, size_t nb, size_t slice, double* partials) {
     __shared__ double sh[kThreads];
     wait_for_prior_grid();
+    release_dependents();
     const size_t lo = (size_t)blockIdx.x * slice;
     const size_t hi = (lo + slice < nb) ? lo + slice : nb;
     double acc = 0.0;
@@ -130,6 +132,7 @@ __global__ void __launch_bounds__(kThreads) k_mse_partial(const float* sse, size
 __global__ void __launch_bounds__(kMsePartials) k_mse_final(const double* partials, int n_partials, double n, double* out) {
     __shared__ double sh[kMsePartials];
     wait_for_prior_grid();
+    release_dependents();
     const double v = (int)threadIdx.x < n_partials ? partials[threadIdx.x] : 0.0;
     const double total = cta_tree_sum<kMsePartials>(v, sh);
     if (threadIdx.x == 0) *out = __ddiv_rn(total, n);
@@ -164,6 +167,7 @@ template <int ODT>
 __global__ void __launch_bounds__(kThreads) k_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n,
                                                          int log2B, int fmt, float g, void* out) {
     wait_for_prior_grid();
+    release_dependents();
     constexpr int E = (ODT == kF32) ? 4 : 8;      // elements per unit
     constexpr int LOG2E = (ODT == kF32) ? 2 : 3;
     constexpr int U = 4;

@@ -22,8 +22,8 @@
 //
 // Arithmetic per element (kernel time follows the number of warp instructions): bf16 -> binary32
 // by a mixed-precision add of -0 (FMA pipe); the exact quotient by the decode scale, two elements
-// per instruction (reciprocal multiply + one residual correction when every decode scale of the
-// table has a short significand, two corrections otherwise); half an FP4 pack, half an FP4
+// per instruction (reciprocal multiply + one residual correction; for bf16 input and decode scales
+// of at most four significant bits a single multiply rounded toward zero); half an FP4 pack, half an FP4
 // unpack; the residual as fma.rn.f32.f16 straight from the unpacked f16 grid value whenever the
 // decode scales of the group are exactly representable in f16 (always, for UE4M3 without a tensor
 // scale), else an f16->f32 convert plus an FFMA; the square-accumulate FMA, for 4-over-6 one
@@ -43,7 +43,9 @@ namespace mxq {
 //   x  D = fl32(value(c) * g); NaN for codes that do not exist
 //   y  R = RN(1 / D) when 2^-60 <= D <= 2^60, else 0
 //   z  bits: f16(-D) in the low half
-//   w  0: general path only; 1: shortcuts valid; 2: shortcuts valid and -D exact in f16.
+//   w  0: general path only; 1: shortcuts valid; 2: shortcuts valid and -D exact in f16; 3: as 2,
+//      and D has at most four significant bits (every decode scale of the FP8 and power-of-two
+//      formats when the tensor scale is a power of two).
 //      D = 0 counts as valid with R = 0: every quotient comes out as a zero with the sign of v.
 struct QuantTables {
     float4 E[256];
@@ -62,6 +64,7 @@ __device__ __forceinline__ void build_quant_tables(QuantTables& T, float g) {
                 const __half hD = __float2half_rn(-D);
                 h16 = (uint32_t)__half_as_ushort(hD);
                 w = (__half2float(hD) == -D) ? 2.0f : 1.0f;
+                if (w == 2.0f && (__float_as_uint(D) & 0x000FFFFFu) == 0u) w = 3.0f;
             }
         }
         T.E[c] = make_float4(D, R, __uint_as_float(h16), w);
@@ -220,8 +223,28 @@ __device__ __forceinline__ void pack_and_score(const float* v, const float* t, c
 // Quotients of one block by its decode scale, two elements per instruction (fma.rn.f32x2):
 // q = (-v) * (-R); r = q * D - v; q <- q - r * R.  Same values as quotient_short(), including the
 // sign of a zero quotient: every product and sum has the signs of the scalar form.
-template <int B>
+//
+// SHORT: the elements have at most 8 significant bits (bf16 input) and D at most 4.  Then the FP4
+// code of fl(v / D) is the FP4 code of RZ(v * R), one multiply rounded toward zero: the quotient is a
+// ratio of small integers times a power of two, so it either IS an FP4 rounding midpoint or lies
+// more than 2^-9 (relative) away from every one of them, far more than the error of the product;
+// and RN(1 / D) is never below 1 / D for these eight significands (it exceeds it by at most
+// 0.875 * 2^-24 relative), so that at a midpoint M the exact product lies in [M, M + ulp) and the
+// truncation returns M itself, which the FP4 rounding then sends to the even neighbour exactly as it
+// does for the true quotient.  Checked on the host for every bf16 value and
+// every significand (tests/test_quotient_hard_cases.py).  The sign of a zero product is that of v.
+template <int B, bool SHORT>
 __device__ __forceinline__ void block_quotients(const float* v, float D, float R, float* t) {
+    if constexpr (SHORT) {
+        const float2 R2 = make_float2(R, R);
+#pragma unroll
+        for (int i = 0; i < B; i += 2) {
+            const float2 q = __fmul2_rz(make_float2(v[i], v[i + 1]), R2);
+            t[i] = q.x;
+            t[i + 1] = q.y;
+        }
+        return;
+    }
     const float2 D2 = make_float2(D, D), nR2 = make_float2(-R, -R);
 #pragma unroll
     for (int i = 0; i < B; i += 2) {
@@ -235,13 +258,13 @@ __device__ __forceinline__ void block_quotients(const float* v, float D, float R
 }
 
 // One candidate set of a group with the shortcuts (every entry has w != 0, magnitudes in range).
-template <int B, bool HALF>
+template <int B, bool HALF, bool SHORT>
 __device__ __forceinline__ void encode_group_fast(const float* v, const float4* E, uint32_t* packed, float* sse) {
     constexpr int GE = (B < 8) ? 8 : B;
     constexpr int NBG = GE / B;
     float t[GE];
 #pragma unroll
-    for (int j = 0; j < NBG; ++j) block_quotients<B>(&v[j * B], E[j].x, E[j].y, &t[j * B]);
+    for (int j = 0; j < NBG; ++j) block_quotients<B, SHORT>(&v[j * B], E[j].x, E[j].y, &t[j * B]);
     pack_and_score<B, HALF>(v, t, E, packed, sse);
 }
 
@@ -249,7 +272,7 @@ __device__ __forceinline__ void encode_group_fast(const float* v, const float4* 
 // candidate, and the two SSE chains of a block side by side in one fma.rn.f32x2 per element
 // (lane .x: the M = 6 candidate, lane .y: the M = 4 candidate; each lane sums its own residuals
 // in element order, exactly like the scalar chain).  The chains continue from sse6[] / sse4[].
-template <int B, bool HALF>
+template <int B, bool HALF, bool SHORT>
 __device__ __forceinline__ void encode_group_fast_dual(const float* v, const float4* E6, const float4* E4, uint32_t* pk6,
                                                        uint32_t* pk4, float* sse6, float* sse4) {
     constexpr int GE = (B < 8) ? 8 : B;
@@ -257,8 +280,8 @@ __device__ __forceinline__ void encode_group_fast_dual(const float* v, const flo
     float t6[GE], t4[GE];
 #pragma unroll
     for (int j = 0; j < NBG; ++j) {
-        block_quotients<B>(&v[j * B], E6[j].x, E6[j].y, &t6[j * B]);
-        block_quotients<B>(&v[j * B], E4[j].x, E4[j].y, &t4[j * B]);
+        block_quotients<B, SHORT>(&v[j * B], E6[j].x, E6[j].y, &t6[j * B]);
+        block_quotients<B, SHORT>(&v[j * B], E4[j].x, E4[j].y, &t4[j * B]);
     }
     uint32_t h6[GE / 2], h4[GE / 2];
 #pragma unroll
@@ -345,7 +368,7 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
         float m[NBG], u[NBG];
         int c6[NBG], c4[NBG];
         float4 E6[NBG], E4[NBG];
-        float wmin = 2.0f, mmax = 0.0f, mmin = k.m_hi;
+        float wmin = 3.0f, mmax = 0.0f, mmin = k.m_hi;
 #pragma unroll
         for (int j = 0; j < NBG; ++j) {
             float a = 0.0f;
@@ -369,12 +392,15 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
 #pragma unroll
         for (int j = 0; j < NBG; ++j) sse[j] = sse4[j] = 0.0f;
         if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
-            if (wmin >= 2.0f) {   // one decision for both candidates
-                if constexpr (DUAL) encode_group_fast_dual<B, true>(v, E6, E4, pk, pk4, sse, sse4);
-                else encode_group_fast<B, true>(v, E6, pk, sse);
+            // one decision for both candidates.  bf16 input: the one-multiply quotient with the f16
+            // residual when every decode scale of the group is short, else the general shortcuts.
+            constexpr bool SH = (DT == kBF16);
+            if (wmin >= (SH ? 3.0f : 2.0f)) {
+                if constexpr (DUAL) encode_group_fast_dual<B, true, SH>(v, E6, E4, pk, pk4, sse, sse4);
+                else encode_group_fast<B, true, SH>(v, E6, pk, sse);
             } else {
-                if constexpr (DUAL) encode_group_fast_dual<B, false>(v, E6, E4, pk, pk4, sse, sse4);
-                else encode_group_fast<B, false>(v, E6, pk, sse);
+                if constexpr (DUAL) encode_group_fast_dual<B, false, false>(v, E6, E4, pk, pk4, sse, sse4);
+                else encode_group_fast<B, false, false>(v, E6, pk, sse);
             }
         } else {
 #pragma unroll
@@ -524,12 +550,13 @@ __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const Qu
         uint32_t* o6 = &pk[sg * (SG / 8)];
         uint32_t* o4 = &pk4[sg * (SG / 8)];
         if (fast) {
-            if (wmin >= 2.0f) {
-                if constexpr (DUAL) encode_group_fast_dual<SG, true>(v, &E6, &E4, o6, o4, &sse, &sse4);
-                else encode_group_fast<SG, true>(v, &E6, o6, &sse);
+            constexpr bool SH = (DT == kBF16);
+            if (wmin >= (SH ? 3.0f : 2.0f)) {
+                if constexpr (DUAL) encode_group_fast_dual<SG, true, SH>(v, &E6, &E4, o6, o4, &sse, &sse4);
+                else encode_group_fast<SG, true, SH>(v, &E6, o6, &sse);
             } else {
-                if constexpr (DUAL) encode_group_fast_dual<SG, false>(v, &E6, &E4, o6, o4, &sse, &sse4);
-                else encode_group_fast<SG, false>(v, &E6, o6, &sse);
+                if constexpr (DUAL) encode_group_fast_dual<SG, false, false>(v, &E6, &E4, o6, o4, &sse, &sse4);
+                else encode_group_fast<SG, false, false>(v, &E6, o6, &sse);
             }
         } else {
             encode_group_general<SG>(v, &E6, o6, &sse);
@@ -618,6 +645,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     extern __shared__ uint4 ring[];
     __shared__ QuantTables T;
     wait_for_prior_grid();
+    release_dependents();
     // request the first chunks before anything else: their latency hides behind the table build
     const size_t stride = (size_t)gridDim.x * kThreads;
     const int lane = threadIdx.x & 31;

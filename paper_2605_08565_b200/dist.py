@@ -81,40 +81,63 @@ def row_shard(n_rows: int, rank: int, world: int) -> tuple[int, int]:
     return n_rows * rank // world, n_rows * (rank + 1) // world
 
 
+def _all_reduce_max(t: torch.Tensor) -> None:
+    """In-place MAX all-reduce; a CUDA tensor under the gloo backend goes through a host copy."""
+    if dist.get_backend() == "gloo" and t.is_cuda:
+        h = t.cpu()
+        dist.all_reduce(h, op=dist.ReduceOp.MAX)
+        t.copy_(h)
+    else:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+
+
 def global_amax(local_amax: torch.Tensor) -> torch.Tensor:
-    """MAX all-reduce of a one-element float32 tensor holding this rank's abs-max (in place)."""
+    """MAX all-reduce of a one-element float32 tensor holding this rank's abs-max (in place).  The
+    maximum is exact and order-free, so every rank ends with the same bits."""
     if dist.is_initialized():
-        dist.all_reduce(local_amax, op=dist.ReduceOp.MAX)
+        _all_reduce_max(local_amax)
     return local_amax
 
 
-def global_mse(local_sse_sum: float, n_total: int) -> float:
-    """Tensor MSE from the per-rank sums of block SSE: gathered, then added in rank order."""
+def global_mse(local_sse_sum, n_total: int) -> float:
+    """Tensor MSE from the per-rank sums of block SSE (a float, or a one-element float64 tensor on any
+    device): the sums are gathered and added in rank order in binary64, then divided once by the
+    element count of the whole tensor, so the result does not depend on arrival order."""
+    mine = torch.as_tensor(local_sse_sum, dtype=torch.float64).reshape(1)
     if not dist.is_initialized():
-        return float(local_sse_sum) / n_total
-    mine = torch.tensor([float(local_sse_sum)], dtype=torch.float64, device=_device())
+        return float(mine.item()) / n_total
+    if dist.get_backend() == "gloo":
+        mine = mine.cpu()
     parts = [torch.zeros_like(mine) for _ in range(dist.get_world_size())]
     dist.all_gather(parts, mine)
     total = 0.0
-    for p in parts:
-        total += float(p.item())
+    for v in torch.cat(parts).cpu().tolist():     # rank order
+        total += v
     return total / n_total
 
 
 def sharded_hierarchical_quantize(x_local: torch.Tensor, n_total: int, block_size: int, scale_fmt: int, recipe: int):
     """Quantize this rank's rows of a tensor that is sharded by rows, with ONE tensor scale
     g = amax_of_the_whole_tensor / (6 * 448) shared by all ranks.  Returns (codes, scales, block_sse,
-    g tensor on the device, tensor MSE of the whole tensor).  Every rank reads only its own memory."""
+    g tensor on the device, tensor MSE of the whole tensor).  Every rank reads only its own memory.
+
+    Only argument marshalling and the two exchanges happen here: the abs-max, g, the quantization and
+    this rank's binary64 sum of block SSEs (the library's fixed tree, called with the divisor 1, so
+    that the quotient is the sum itself) are computed by the library on the device; the only host
+    read is the final one of the gathered sums."""
     from . import binding as mxq
     n = x_local.numel()
-    amax = torch.empty(1, dtype=torch.float32, device=x_local.device)
+    dev = x_local.device
+    amax = torch.empty(1, dtype=torch.float32, device=dev)
     mxq.mxq_tensor_amax(x_local, n, amax)
     global_amax(amax)
-    g = mxq.mxq_global_scale_from_amax(float(amax.item()))
-    dg = torch.tensor([g], dtype=torch.float32, device=x_local.device)
+    # g from the all-reduced abs-max, on the device: the abs-max of the one-element tensor `amax` is itself
+    amax_all = torch.empty(1, dtype=torch.float32, device=dev)
+    dg = torch.empty(1, dtype=torch.float32, device=dev)
+    mxq.mxq_tensor_amax(amax, 1, amax_all, dg)
     codes, scales, sse = mxq.quantize(x_local, block_size, scale_fmt, recipe, 1.0, dg)
-    local_mse = mxq.tensor_mse(sse, n)                      # deterministic local tree
-    mse = global_mse(float(local_mse.item()) * n, n_total)
+    local_sum = mxq.tensor_mse(sse, 1)
+    mse = global_mse(local_sum, n_total)
     return codes, scales, sse, dg, mse
 
 
