@@ -15,6 +15,14 @@
  *   - Return value: MXQ_OK (0) or a positive mxq_status.  Nothing throws, aborts or prints.
  *   - Results are deterministic from run to run (no floating-point atomics).
  *   - Inputs must be finite.  NaN or Inf elements give unspecified (but memory-safe) outputs.
+ *   - Threads.  Entry points may be called from several host threads at once (on the same or on
+ *     different devices and streams): the library keeps no per-call host state, its first-use caches
+ *     (SM count, resident CTAs per kernel) are atomics whose racing writers store equal values, and
+ *     mxq_last_cuda_error() is per thread.  Two things are process-wide and therefore shared by all
+ *     threads: the options of mxq_set_option() (a call reads the option once, when it is made; changing
+ *     it while another thread is inside mxq_quantize_ex affects only calls made afterwards), and the
+ *     scratch array of mxq_tensor_mse_static() (see there).  As with any CUDA library, the device that
+ *     owns the pointers must be the calling thread's current device.
  *
  * Data layout
  *   x            n elements, contiguous; a block is B consecutive elements of the flat array
@@ -182,6 +190,16 @@ int mxq_tensor_mse_static(const float* d_block_sse, size_t n_blocks, size_t n, d
  */
 int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
                    float global_scale, void* d_out, int out_dtype, void* cuda_stream);
+
+/*
+ * mxq_dequantize_ex -- mxq_dequantize with an optional device-resident tensor scale, so that the
+ * hierarchical flow (mxq_tensor_amax -> g on the device -> mxq_quantize_ex -> ... -> de-quantize) never
+ * has to read g back to the host (Experimental Setup, hierarchical scaling).
+ *   d_global_scale  device pointer to one float holding g, or NULL.  When non-NULL it overrides
+ *                   `global_scale` (which is then not checked) and is read by the kernel at run time.
+ */
+int mxq_dequantize_ex(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
+                      float global_scale, const float* d_global_scale, void* d_out, int out_dtype, void* cuda_stream);
 
 /*
  * mxq_block_clip_sse -- the clipping part of the block SSE (Appendix, "Clipping only MSE": the MSE

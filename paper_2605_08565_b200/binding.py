@@ -22,7 +22,8 @@ MXQ_OPT_BRUTE_PRUNE = 1
 
 EXPORTS = (
     "mxq_quantize", "mxq_quantize_ex", "mxq_fake_quantize", "mxq_tensor_amax", "mxq_global_scale_from_amax",
-    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_mask_interval", "mxq_set_option", "mxq_get_option", "mxq_launch_count",
+    "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_dequantize_ex",
+    "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_mask_interval", "mxq_set_option", "mxq_get_option", "mxq_launch_count",
     "mxq_status_string", "mxq_last_cuda_error", "mxq_version",
 )
 
@@ -63,6 +64,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_tensor_mse_static.argtypes = [vp, sz, sz, vp, vp]
     L.mxq_dequantize.restype = i32
     L.mxq_dequantize.argtypes = [vp, vp, sz, i32, i32, f32, vp, i32, vp]
+    L.mxq_dequantize_ex.restype = i32
+    L.mxq_dequantize_ex.argtypes = [vp, vp, sz, i32, i32, f32, vp, vp, i32, vp]
     L.mxq_block_clip_sse.restype = i32
     L.mxq_block_clip_sse.argtypes = [vp, i32, sz, i32, i32, f32, vp, vp, vp, vp]
     L.mxq_histograms.restype = i32
@@ -173,6 +176,11 @@ def mxq_tensor_mse_static(d_block_sse, n_blocks, n, d_out_mse, stream=None) -> N
 def mxq_dequantize(d_codes, d_scales, n, block_size, scale_fmt, global_scale, d_out, stream=None) -> None:
     _check(load_library().mxq_dequantize(_ptr(d_codes), _ptr(d_scales), n, block_size, scale_fmt, global_scale,
                                          _ptr(d_out), _dtype_id(d_out), _stream(stream, d_out)))
+
+
+def mxq_dequantize_ex(d_codes, d_scales, n, block_size, scale_fmt, global_scale, d_global_scale, d_out, stream=None) -> None:
+    _check(load_library().mxq_dequantize_ex(_ptr(d_codes), _ptr(d_scales), n, block_size, scale_fmt, global_scale,
+                                            _ptr(d_global_scale), _ptr(d_out), _dtype_id(d_out), _stream(stream, d_out)))
 
 
 def mxq_block_clip_sse(x, n, block_size, scale_fmt, global_scale, d_global_scale, d_scales, out_clip_sse,

@@ -15,14 +15,15 @@ static thread_local int tl_cuda_error = 0;
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 int sm_count(int device) {
-    static int cached[kMaxDevices] = {0};
+    // first-use cache; two threads that race here both store the same value
+    static std::atomic<int> cached[kMaxDevices];
     if (device < 0 || device >= kMaxDevices) return 1;
-    if (cached[device] == 0) {
-        int n = 0;
+    int n = cached[device].load(std::memory_order_relaxed);
+    if (n == 0) {
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = 1;
-        cached[device] = n;
+        cached[device].store(n, std::memory_order_relaxed);
     }
-    return cached[device];
+    return n;
 }
 
 static int cuda_fail(cudaError_t e) {
@@ -36,10 +37,6 @@ static bool valid_block(int b) { return b == 2 || b == 4 || b == 8 || b == 16 ||
 }  // namespace mxq
 
 using namespace mxq;
-
-extern "C" {
-
-}  // extern "C"
 
 // Shared by mxq_quantize_ex (codes + scales, optional SSE) and mxq_fake_quantize (x_hat only).
 static int quantize_common(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe,
@@ -163,17 +160,25 @@ int mxq_tensor_mse_static(const float* d_block_sse, size_t n_blocks, size_t n, d
     return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
 }
 
-int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
-                   float global_scale, void* d_out, int out_dtype, void* cuda_stream) {
+int mxq_dequantize_ex(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
+                      float global_scale, const float* d_global_scale, void* d_out, int out_dtype, void* cuda_stream) {
     if (!d_codes || !d_scales || !d_out) return MXQ_ERR_NULL;
     if (out_dtype != MXQ_F32 && out_dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
     if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
     if (!valid_block(block_size) || n == 0 || n % (size_t)block_size != 0) return MXQ_ERR_BAD_SHAPE;
-    if (!(global_scale > 0.0f && std::isfinite(global_scale))) return MXQ_ERR_BAD_SCALE;
-    if (!aligned16(d_codes) || !aligned16(d_out) || (reinterpret_cast<uintptr_t>(d_scales) & 3u)) return MXQ_ERR_ALIGN;
-    cudaError_t err = launch_dequantize(d_codes, d_scales, n, block_size, scale_fmt, global_scale, d_out, out_dtype,
-                                        static_cast<cudaStream_t>(cuda_stream));
+    if (!d_global_scale && !(global_scale > 0.0f && std::isfinite(global_scale))) return MXQ_ERR_BAD_SCALE;
+    if (!aligned16(d_codes) || !aligned16(d_out) || (reinterpret_cast<uintptr_t>(d_scales) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_global_scale) & 3u))
+        return MXQ_ERR_ALIGN;
+    cudaError_t err = launch_dequantize(d_codes, d_scales, n, block_size, scale_fmt, d_global_scale ? 1.0f : global_scale,
+                                        d_global_scale, d_out, out_dtype, static_cast<cudaStream_t>(cuda_stream));
     return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+int mxq_dequantize(const uint8_t* d_codes, const uint8_t* d_scales, size_t n, int block_size, int scale_fmt,
+                   float global_scale, void* d_out, int out_dtype, void* cuda_stream) {
+    return mxq_dequantize_ex(d_codes, d_scales, n, block_size, scale_fmt, global_scale, nullptr, d_out, out_dtype,
+                             cuda_stream);
 }
 
 int mxq_block_clip_sse(const void* x, int dtype, size_t n, int block_size, int scale_fmt, float global_scale,

@@ -31,6 +31,8 @@
 // is the smaller code); class winners are merged as 64-bit keys (SSE bits << 32 | code).
 #pragma once
 
+#include <atomic>
+
 #include "mxq_device.cuh"
 #include "mxq_internal.h"
 
@@ -825,16 +827,18 @@ __global__ void k_brute_tail(QuantArgs p) {
 
 template <int DT, int B, int FMT, bool PRUNE>
 static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
-    static int ctas_per_sm[kMaxDevices] = {0};
+    static std::atomic<int> ctas_per_sm[kMaxDevices];   // first-use cache; racing threads store the same value
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (ctas_per_sm[dev] == 0) {
+    int resident = ctas_per_sm[dev].load(std::memory_order_relaxed);
+    if (resident == 0) {
         int n = 0;
         err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_brute<DT, B, FMT, PRUNE>, kThreads, 0);
         if (err != cudaSuccess) return err;
-        ctas_per_sm[dev] = n > 0 ? n : 1;
+        resident = n > 0 ? n : 1;
+        ctas_per_sm[dev].store(resident, std::memory_order_relaxed);
     }
     constexpr size_t G = brute_group_elems(B);    // elements per thread of k_brute
     const size_t n_blocks = a.n_items;
@@ -843,7 +847,7 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
         QuantArgs m = a;
         m.n_items = n_groups;
         const size_t want = (n_groups + kThreads - 1) / kThreads;
-        const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
+        const size_t cap = (size_t)sm_count(dev) * (size_t)resident;
         const unsigned grid = (unsigned)(want < cap ? want : cap);
         err = launch_pdl(k_brute<DT, B, FMT, PRUNE>, grid, kThreads, 0, stream, m);
         count_launch();

@@ -68,8 +68,8 @@ cudaError_t launch_tensor_mse(const float* d_sse, size_t n_blocks, size_t n, dou
                               cudaStream_t s);
 // Same reduction with the first-level partials in a library-owned device array (no workspace).
 cudaError_t launch_tensor_mse_static(const float* d_sse, size_t n_blocks, size_t n, double* d_out, cudaStream_t s);
-cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n, int B, int fmt, float g, void* out,
-                              int out_dtype, cudaStream_t s);
+cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n, int B, int fmt, float g,
+                              const float* d_g, void* out, int out_dtype, cudaStream_t s);
 
 cudaError_t launch_block_clip_sse(const void* x, int dtype, size_t n, int B, int fmt, float g, const float* d_g,
                                   const uint8_t* scales, float* out, cudaStream_t s);

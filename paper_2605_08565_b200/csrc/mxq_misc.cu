@@ -165,9 +165,10 @@ __device__ __forceinline__ float decode_scale(int fmt, int c, float g) {
 // units per thread and trip keep four independent loads in flight.
 template <int ODT>
 __global__ void __launch_bounds__(kThreads) k_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n,
-                                                         int log2B, int fmt, float g, void* out) {
+                                                         int log2B, int fmt, float g_host, const float* d_g, void* out) {
     wait_for_prior_grid();
     release_dependents();
+    const float g = d_g ? *d_g : g_host;   // device-resident tensor scale (written by an earlier kernel of the stream)
     constexpr int E = (ODT == kF32) ? 4 : 8;      // elements per unit
     constexpr int LOG2E = (ODT == kF32) ? 2 : 3;
     constexpr int U = 4;
@@ -230,8 +231,8 @@ __global__ void __launch_bounds__(kThreads) k_dequantize(const uint8_t* codes, c
     }
 }
 
-cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n, int B, int fmt, float g, void* out,
-                              int out_dtype, cudaStream_t s) {
+cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_t n, int B, int fmt, float g,
+                              const float* d_g, void* out, int out_dtype, cudaStream_t s) {
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
@@ -241,8 +242,8 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* scales, size_
     if (want == 0) want = 1;
     const size_t cap = (size_t)sm_count(dev) * 8;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
-    if (out_dtype == kF32) err = launch_pdl(k_dequantize<kF32>, grid, kThreads, 0, s, codes, scales, n, log2B, fmt, g, out);
-    else err = launch_pdl(k_dequantize<kBF16>, grid, kThreads, 0, s, codes, scales, n, log2B, fmt, g, out);
+    if (out_dtype == kF32) err = launch_pdl(k_dequantize<kF32>, grid, kThreads, 0, s, codes, scales, n, log2B, fmt, g, d_g, out);
+    else err = launch_pdl(k_dequantize<kBF16>, grid, kThreads, 0, s, codes, scales, n, log2B, fmt, g, d_g, out);
     count_launch();
     return err;
 }

@@ -34,6 +34,9 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <atomic>
+#include <type_traits>
+
 #include "mxq_device.cuh"
 #include "mxq_internal.h"
 
@@ -51,8 +54,11 @@ struct QuantTables {
     float4 E[256];
 };
 
+// Returns whether EVERY code of the format got class 3 (CTA-uniform).
 template <int FMT>
-__device__ __forceinline__ void build_quant_tables(QuantTables& T, float g) {
+__device__ __forceinline__ bool build_quant_tables(QuantTables& T, float g) {
+    static_assert(kThreads == 256, "one thread per table entry");
+    bool all_short = true;
     for (int c = threadIdx.x; c < 256; c += blockDim.x) {
         float D = __uint_as_float(0x7FC00000u), R = 0.0f, w = 0.0f;
         uint32_t h16 = 0;
@@ -68,8 +74,9 @@ __device__ __forceinline__ void build_quant_tables(QuantTables& T, float g) {
             }
         }
         T.E[c] = make_float4(D, R, __uint_as_float(h16), w);
+        all_short = all_short && (c >= num_codes(FMT) || w == 3.0f);
     }
-    __syncthreads();
+    return __syncthreads_and(all_short) != 0;
 }
 
 // fl32(v / D) by a reciprocal multiply and ONE residual correction, R = RN(1 / D) correctly rounded,
@@ -338,7 +345,16 @@ struct QuantConsts {
     bool unit_g, need_lo;
     int c_min;          // smallest admissible code: 1 under prevent-zero (FP8 formats), else 0
     int pow2_rule;      // kPow2Eq1 unless the format is UE8M0 and another rule was asked for
+    float u_floor;      // lean path: prevent-zero as a floor on amax / g, 4 * value(code 1), else 0
 };
+
+// Both 4-over-6 scale codes of a block from one conversion (UE4M3): the code for w6 in bits 0..7,
+// the code for w4 in bits 8..15.
+__device__ __forceinline__ uint32_t round_scale_pair_ue4m3(float w4, float w6) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(w4), "f"(w6));
+    return r;
+}
 
 // Scale code for the M = 6 target from u = amax / g: Eq. 2 (Eq. 1 for UE8M0), or one of the
 // alternative power-of-two rules.
@@ -350,9 +366,20 @@ __device__ __forceinline__ int target6_code(float u, int pow2_rule) {
     return round_scale<FMT>(EXACT ? __fdiv_rn(u, 6.0f) : div6_fast(u));
 }
 
-template <int DT, int B, int FMT, bool DUAL, bool FAKE>
+// LEAN (launch-uniform; bf16 input, FP8 scale format, no tensor scale, every decode scale of the
+// table of class 3): nothing of a block can leave the shortcuts, so the per-block class and range
+// tests, the tensor-scale quotient and the general path are left out.  Why no magnitude test is
+// needed: the one-multiply quotient neither forms a residual nor divides (a product that
+// overflows or underflows still rounds to the FP4 code of the true quotient, 6 or 0 with the sign
+// of the element); amax / 6 by multiply-and-correct is exact from 1e-30 to 1e30, below that every
+// FP8 format gives code 0 (the prevent-zero floor keeps the argument far above it anyway) and
+// above it both formats saturate.  Prevent-zero is a floor on the block maximum: for both
+// formats max(code_M(u), 1) = code_M(max(u, 4 eps)) for M = 6 and M = 4, eps = value(code 1)
+// (4 eps / 6 and 4 eps / 4 round to code 1; anything below rounds to 0 or 1, anything above to >= 1).
+template <int DT, int B, int FMT, bool DUAL, bool FAKE, bool LEAN>
 __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
                                                size_t chunk, const uint32_t* raw) {
+    static_assert(!LEAN || (DT == kBF16 && FMT != kUE8M0), "lean path: bf16 input, FP8 scale formats");
     using S = QuantShape<DT, B>;
     constexpr int NBG = S::NBG;
     uint32_t packed[S::C / 8];
@@ -374,6 +401,21 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             float a = 0.0f;
 #pragma unroll
             for (int i = 0; i < B; ++i) a = fmaxf(a, fabsf(v[j * B + i]));
+            if constexpr (LEAN) {
+                const float uf = fmaxf(a, k.u_floor);
+                const float w6 = div6_fast(uf);
+                if constexpr (DUAL && FMT == kUE4M3) {
+                    const uint32_t r = round_scale_pair_ue4m3(__fmul_rn(uf, 0.25f), w6);
+                    c6[j] = (int)(r & 0xFFu);
+                    c4[j] = (int)(r >> 8);
+                } else {
+                    c6[j] = round_scale<FMT>(w6);
+                    if constexpr (DUAL) c4[j] = round_scale<FMT>(__fmul_rn(uf, 0.25f));
+                }
+                E6[j] = T.E[c6[j]];
+                if constexpr (DUAL) E4[j] = T.E[c4[j]];
+                continue;
+            }
             m[j] = a;
             mmax = fmaxf(mmax, a);
             if (k.need_lo) mmin = fminf(mmin, a == 0.0f ? k.m_hi : a);
@@ -391,7 +433,10 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
         float sse[NBG], sse4[NBG];
 #pragma unroll
         for (int j = 0; j < NBG; ++j) sse[j] = sse4[j] = 0.0f;
-        if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
+        if constexpr (LEAN) {
+            if constexpr (DUAL) encode_group_fast_dual<B, true, true>(v, E6, E4, pk, pk4, sse, sse4);
+            else encode_group_fast<B, true, true>(v, E6, pk, sse);
+        } else if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
             // one decision for both candidates.  bf16 input: the one-multiply quotient with the f16
             // residual when every decode scale of the group is short, else the general shortcuts.
             constexpr bool SH = (DT == kBF16);
@@ -669,10 +714,11 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     }
     QuantConsts k;
     k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    build_quant_tables<FMT>(T, k.g);
+    const bool all_short = build_quant_tables<FMT>(T, k.g);
     k.unit_g = (k.g == 1.0f);
     k.c_min = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;
+    k.u_floor = k.c_min ? __fmul_rn(4.0f, scale_value(FMT, 1)) : 0.0f;
     k.Rg = 1.0f;
     // Ranges of a block maximum m for which u = fl(m / g) and fl(u / 6) come out exact from the
     // multiply-and-correct forms.  The FP8 formats round every u below 2^-20 to code 0, so an
@@ -695,38 +741,50 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     // Thread-private staging: a thread leaves when its chunks are done (no barrier follows).
     // Cooperative staging: the warp stays together, lanes past the end only take part in the copies.
     if ((S::COOP ? wchunk0 : chunk) >= p.n_items) return;
-    int slot = 0;                      // slot holding `chunk`
-    int fill = DIST % S::SLOTS;        // slot that the next request goes to
-    size_t ahead = (S::COOP ? wchunk0 : chunk) + (size_t)DIST * stride;
-    for (size_t lead = S::COOP ? wchunk0 : chunk; lead < p.n_items; lead += stride, chunk += stride) {
-        // all but the DIST - 1 most recent groups are complete: this thread's copies for `chunk` have landed
-        asm volatile("cp.async.wait_group %0;" ::"n"(DIST - 1) : "memory");
-        // cooperative staging: so have the other lanes' copies, and every lane is done reading the
-        // slot that the next request overwrites
-        if constexpr (S::COOP) __syncwarp();
-        const uint4* slot_warp = ring + (size_t)slot * (S::PIECES * kThreads) + (threadIdx.x - lane);
-        // the slot read one trip ago is free again (its words were consumed by the arithmetic of
-        // that trip): request the chunk DIST trips ahead into it.  The slot of the current chunk
-        // is not requested into before the next trip, so it may be read throughout this one.
-        if constexpr (S::COOP) stage_warp_chunks<S::PIECES>(ring_warp + fill * kSlotBytes, x, kChunkBytes, ahead, p.n_items, lane);
-        else stage_chunk<S::PIECES>(ring_base + fill * kSlotBytes, x + ahead * kChunkBytes, ahead < p.n_items);
-        ahead += stride;
-        slot = (slot + 1 == S::SLOTS) ? 0 : slot + 1;
-        fill = (fill + 1 == S::SLOTS) ? 0 : fill + 1;
-        if (S::COOP && chunk >= p.n_items) continue;   // a lane past the end (the warp's last trip)
-        // blocks longer than 16 elements go part by part, except 4-over-6 at B = 32, which measured
-        // slightly faster with the whole block in registers
-        if constexpr (B > 16 && !(DUAL && B == 32)) {
-            quantize_long_block<DT, B, FMT, DUAL, FAKE>(p, T, k, chunk, slot_warp, lane);
-        } else {
-            uint32_t raw[S::PIECES * 4];
+    // The chunk loop, instantiated with and without the lean per-block path (see quantize_chunk);
+    // which one runs is the same for every thread of the launch.
+    auto chunk_loop = [&](auto lean_tag) {
+        constexpr bool LEAN = decltype(lean_tag)::value;
+        int slot = 0;                      // slot holding `chunk`
+        int fill = DIST % S::SLOTS;        // slot that the next request goes to
+        size_t ahead = (S::COOP ? wchunk0 : chunk) + (size_t)DIST * stride;
+        for (size_t lead = S::COOP ? wchunk0 : chunk; lead < p.n_items; lead += stride, chunk += stride) {
+            // all but the DIST - 1 most recent groups are complete: this thread's copies for `chunk` have landed
+            asm volatile("cp.async.wait_group %0;" ::"n"(DIST - 1) : "memory");
+            // cooperative staging: so have the other lanes' copies, and every lane is done reading the
+            // slot that the next request overwrites
+            if constexpr (S::COOP) __syncwarp();
+            const uint4* slot_warp = ring + (size_t)slot * (S::PIECES * kThreads) + (threadIdx.x - lane);
+            // the slot read one trip ago is free again (its words were consumed by the arithmetic of
+            // that trip): request the chunk DIST trips ahead into it.  The slot of the current chunk
+            // is not requested into before the next trip, so it may be read throughout this one.
+            if constexpr (S::COOP) stage_warp_chunks<S::PIECES>(ring_warp + fill * kSlotBytes, x, kChunkBytes, ahead, p.n_items, lane);
+            else stage_chunk<S::PIECES>(ring_base + fill * kSlotBytes, x + ahead * kChunkBytes, ahead < p.n_items);
+            ahead += stride;
+            slot = (slot + 1 == S::SLOTS) ? 0 : slot + 1;
+            fill = (fill + 1 == S::SLOTS) ? 0 : fill + 1;
+            if (S::COOP && chunk >= p.n_items) continue;   // a lane past the end (the warp's last trip)
+            // blocks longer than 16 elements go part by part, except 4-over-6 at B = 32, which measured
+            // slightly faster with the whole block in registers
+            if constexpr (B > 16 && !(DUAL && B == 32)) {
+                quantize_long_block<DT, B, FMT, DUAL, FAKE>(p, T, k, chunk, slot_warp, lane);
+            } else {
+                uint32_t raw[S::PIECES * 4];
 #pragma unroll
-            for (int q = 0; q < S::PIECES; ++q) {
-                const uint4 w = slot_warp[ring_index<S::COOP>(q, lane)];
-                raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
+                for (int q = 0; q < S::PIECES; ++q) {
+                    const uint4 w = slot_warp[ring_index<S::COOP>(q, lane)];
+                    raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
+                }
+                quantize_chunk<DT, B, FMT, DUAL, FAKE, LEAN>(p, T, k, chunk, raw);
             }
-            quantize_chunk<DT, B, FMT, DUAL, FAKE>(p, T, k, chunk, raw);
         }
+    };
+    constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
+    if constexpr (CAN_LEAN) {
+        if (all_short && k.unit_g) chunk_loop(std::true_type{});
+        else chunk_loop(std::false_type{});
+    } else {
+        chunk_loop(std::false_type{});
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
@@ -736,19 +794,21 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
 template <int DT, int B, int FMT, bool DUAL, bool FAKE>
 static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream) {
     using S = QuantShape<DT, B>;
-    static int ctas_per_sm[kMaxDevices] = {0};
+    static std::atomic<int> ctas_per_sm[kMaxDevices];   // first-use cache; racing threads store the same value
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (ctas_per_sm[dev] == 0) {
+    int resident = ctas_per_sm[dev].load(std::memory_order_relaxed);
+    if (resident == 0) {
         err = cudaFuncSetAttribute(k_quantize<DT, B, FMT, DUAL, FAKE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)S::RING_BYTES);
         if (err != cudaSuccess) return err;
         int n = 0;
         err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_quantize<DT, B, FMT, DUAL, FAKE>, kThreads, S::RING_BYTES);
         if (err != cudaSuccess) return err;
-        ctas_per_sm[dev] = n > 0 ? n : 1;
+        resident = n > 0 ? n : 1;
+        ctas_per_sm[dev].store(resident, std::memory_order_relaxed);
     }
     const size_t n_blocks = a.n_items;
     const size_t n_chunks = n_blocks / S::NBC;
@@ -756,7 +816,7 @@ static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream)
         QuantArgs m = a;
         m.n_items = n_chunks;
         const size_t want = (n_chunks + kThreads - 1) / kThreads;
-        const size_t cap = (size_t)sm_count(dev) * (size_t)ctas_per_sm[dev];
+        const size_t cap = (size_t)sm_count(dev) * (size_t)resident;
         const unsigned grid = (unsigned)(want < cap ? want : cap);
         err = launch_pdl(k_quantize<DT, B, FMT, DUAL, FAKE>, grid, kThreads, S::RING_BYTES, stream, m);
         count_launch();

@@ -30,11 +30,13 @@ BLOCK_SIZES = (4, 8, 16, 32)
 
 def run(block_sizes=BLOCK_SIZES, n_sigma: int = 151, sigma_lo: float = 0.0005, sigma_hi: float = 0.05,
         blocks_per_sigma: int = 50_000, scale_fmt: int = mxq.MXQ_SF_UE4M3, seed: int = 0, device="cuda",
-        recipes=RECIPES, histogram_sigmas=()):
+        recipes=RECIPES, histogram_sigmas=(), keep_block_sse: bool = False):
     """Returns {"sigma": [...], "mse": {recipe: {B: [...]}}, "clip_mse": {...}, "hist": {...}, "seconds": ...}.
 
     histogram_sigmas: indices into the sigma grid for which the 16-bin entry histogram and the
     256-bin scale histogram are collected per recipe and block size.
+    keep_block_sse: also return the per-block SSE tensors (device, one row of blocks_per_sigma values
+    per sigma) under "block_sse", for callers that want more than the mean (e.g. its sampling error).
     """
     if not torch.cuda.is_available():
         raise mxq.MxqError("the numerical study needs a CUDA device (no CPU fallback)")
@@ -42,6 +44,8 @@ def run(block_sizes=BLOCK_SIZES, n_sigma: int = 151, sigma_lo: float = 0.0005, s
     sig = inputs.sigma_grid(n_sigma, sigma_lo, sigma_hi)
     res = {"sigma": [float(s) for s in sig], "blocks_per_sigma": blocks_per_sigma, "scale_fmt": scale_fmt,
            "mse": {r: {} for r in recipes}, "clip_mse": {r: {} for r in recipes}, "hist": {}, "elements": 0}
+    if keep_block_sse:
+        res["block_sse"] = {r: {} for r in recipes}
     torch.cuda.synchronize(dev)
     t0 = time.perf_counter()
     gpu_s = 0.0
@@ -62,6 +66,8 @@ def run(block_sizes=BLOCK_SIZES, n_sigma: int = 151, sigma_lo: float = 0.0005, s
             mxq.mxq_block_clip_sse(x, n, B, scale_fmt, 1.0, None, scales, clip)
             mxq.mxq_segment_mse(clip, nb, blocks_per_sigma, per_sigma, cmse)
             res["mse"][name][B] = mse.cpu().tolist()
+            if keep_block_sse:
+                res["block_sse"][name][B] = sse.view(n_sigma, blocks_per_sigma).clone()
             res["clip_mse"][name][B] = cmse.cpu().tolist()
             for k in histogram_sigmas:
                 ch = torch.zeros(16, dtype=torch.int64, device=dev)

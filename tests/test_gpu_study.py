@@ -148,3 +148,58 @@ def test_mask_interval_matches_definition(dtype):
                        out.view(torch.int16 if dtype == torch.bfloat16 else torch.int32))
     with pytest.raises(mxq.MxqError):
         mxq.mxq_mask_interval(xg, n, 0.02, 0.01, out)
+
+
+def test_numerical_study_at_the_papers_size_shows_the_papers_findings():
+    """The full protocol of the numerical study (Results, "Numerical Study" and its MSE-versus-sigma
+    figure): N(0, sigma^2) samples, 151 sigmas evenly spaced in [0.0005, 0.05], 50,000 blocks per sigma,
+    block sizes 4, 8, 16, 32, FP4 entries, UE4M3 scales.  Asserted, with the sampling error of every MSE
+    estimate taken into account (mean of 50,000 block SSEs; different block sizes see different samples):
+      * Region A: where every abs-max scale underflows to zero the MSE is the signal power itself, the
+        abs-max curve peaks far above prevent-zero's at small sigma, and prevent-zero is never worse;
+      * Region B: with abs-max + prevent-zero the smallest block is significantly WORSE than the largest
+        over a range of sigmas (the inversion), and most of that error is clipping;
+      * 4-over-6 + prevent-zero and brute force show no significant inversion at any sigma, and the
+        brute-force optimum never gets significantly worse when blocks get finer."""
+    res = study.run(keep_block_sse=True)
+    sig = np.array(res["sigma"])
+    assert len(sig) == 151 and res["blocks_per_sigma"] == 50_000
+    bs = (4, 8, 16, 32)
+    mean, se = {}, {}
+    for name in study.RECIPES:
+        for B in bs:
+            s = res["block_sse"][name][B].double()
+            mean[name, B] = (s.mean(dim=1) / B).cpu().numpy()
+            se[name, B] = (s.std(dim=1) / (s.shape[1] ** 0.5) / B).cpu().numpy()
+            got = np.array(res["mse"][name][B])
+            assert np.all(np.abs(got - mean[name, B]) <= 1e-9 * mean[name, B] + 1e-300)   # the library's tree = the plain mean
+
+    def worse(name, b_small, b_large, z=5.0):
+        """sigmas at which b_small's MSE exceeds b_large's by more than z combined standard errors"""
+        d = mean[name, b_small] - mean[name, b_large]
+        return np.flatnonzero(d > z * np.sqrt(se[name, b_small] ** 2 + se[name, b_large] ** 2))
+
+    # Region A
+    k0 = 0                                                       # sigma = 0.0005: every block maximum / 6 rounds to scale 0
+    assert abs(mean["absmax", 4][k0] / sig[k0] ** 2 - 1.0) < 0.02
+    ratio = mean["absmax", 4] / mean["absmax_pz", 4]
+    kpk = int(np.argmax(ratio))
+    assert ratio[kpk] > 10.0 and sig[kpk] < 0.005
+    for B in bs:
+        assert np.all(mean["absmax_pz", B] <= mean["absmax", B])
+        assert np.all(mean["4o6_pz", B] <= mean["4o6", B])
+    # Region B
+    inv = worse("absmax_pz", 4, 32)
+    assert inv.size >= 20 and 0.004 < sig[inv].min() < 0.01 and sig[inv].max() < 0.03
+    mid = inv[inv.size // 2]
+    clip_share = np.array(res["clip_mse"]["absmax_pz"][4])[mid] / mean["absmax_pz", 4][mid]
+    assert clip_share > 0.4
+    # no inversion for 4-over-6 + prevent-zero beyond the zero-scale region, none at all for brute force
+    assert np.all(sig[worse("4o6_pz", 4, 32)] < 0.004)
+    assert worse("brute", 4, 32).size == 0
+    for a, b in ((4, 8), (8, 16), (16, 32)):
+        assert worse("brute", a, b).size == 0
+    # the recipes order as the paper has them, at every sigma and block size
+    for B in bs:
+        assert np.all(mean["brute", B] <= mean["4o6_pz", B] * (1 + 1e-12))
+        assert np.all(mean["4o6_pz", B] <= mean["absmax_pz", B] * (1 + 1e-12))
