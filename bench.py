@@ -9,7 +9,8 @@ Workload of the default run (N = 1), one STEP = one pass of the whole hot path o
 
 * bulk scale search: 16384 x 16384 fp32 Laplace(0,1), tensor abs-max -> device-resident tensor scale
   g = amax / 2688, then the full brute-force sweep for every block size in {2,4,8,16,32} and every
-  scale format in {UE8M0, UE4M3, UE5M3}, each followed by the tensor MSE (15 sweeps);
+  scale format in {UE8M0, UE4M3, UE5M3}, each scored by the tensor MSE (15 sweeps; quantization and MSE
+  are one call, ``mxq_quantize_mse``);
 * weight leg: one matrix of each shape of an 8B-parameter Llama-style layer (4096x4096, 1024x4096,
   14336x4096, 4096x14336; bf16, Student-t(4)/sqrt(fan_in)), block sizes {8,16} x {UE4M3, UE5M3} x
   {abs-max, abs-max + prevent-zero, 4-over-6, 4-over-6 + prevent-zero}, tensor MSE after each;
@@ -346,11 +347,12 @@ class Workload:
             if timed and leg == "search":
                 ev = (self._ev(), self._ev())
                 ev[0].record()
-            mxq.mxq_quantize_ex(t, n, B, fmt, recipe, 1.0, dg, self.codes, self.scales, self.sse)
+            # quantize + tensor MSE in one call: the kernel sums its own block SSEs, a one-CTA kernel finishes
+            mxq.mxq_quantize_mse(t, n, B, fmt, recipe, 1.0, dg, self.codes, self.scales, self.sse,
+                                 self.mse[slot:slot + 1], self.ws)
             if ev is not None:
                 ev[1].record()
                 self.search_events.setdefault((B, fmt), []).append(ev)
-            mxq.mxq_tensor_mse(self.sse, n // B, n, self.mse[slot:slot + 1], self.ws)
             slot += 1
         # the last pass left UE5M3 / 4-over-6 codes of an activation tensor: de-quantize them
         mxq.mxq_dequantize(self.codes, self.scales, ACT_N, 16, UE5M3, 1.0, self.xhat)
@@ -480,6 +482,39 @@ def streaming_rooflines(torch, mxq, device, peaks):
     return out
 
 
+def weight_set_report(torch, mxq, device, peaks, layers: int = 8):
+    """A quarter of the Llama-3-8B-shaped weight set (8 layers x 7 matrices, 1.74 G bf16 elements) quantized
+    three ways: one launch per matrix from a Python loop, the same launches replayed from a CUDA graph, and
+    ONE multi-tensor launch (mxq_quantize_batch); abs-max and 4-over-6, B = 16, UE4M3."""
+    from paper_2605_08565_b200 import inputs
+    xs = []
+    for layer in range(layers):
+        for idx, (name, rows_, cols) in enumerate(inputs.LLAMA8B_LAYER_SHAPES):
+            xs.append(inputs.student_t(rows_ * cols, 4, 1.0 / math.sqrt(cols), 4 + layer * 7 + idx, torch.bfloat16, device))
+    outs = [mxq.alloc_outputs(x.numel(), 16, device) for x in xs]
+    h, d = mxq.make_tensor_descs([(x, c, s_, e) for x, (c, s_, e) in zip(xs, outs)])
+    n_total = sum(x.numel() for x in xs)
+    res = {"matrices": len(xs), "elements": n_total}
+    for recipe in (ABSMAX, R4O6):
+        def per_matrix():
+            for x, (c, s_, e) in zip(xs, outs):
+                mxq.mxq_quantize_ex(x, x.numel(), 16, UE4M3, recipe, 1.0, None, c, s_, e)
+
+        def batched():
+            mxq.mxq_quantize_batch(h, d, len(xs), mxq.MXQ_BF16, 16, UE4M3, recipe, 1.0)
+        ms_graph, ms_loop = graph_timed(torch, per_matrix, 1, reps=3)
+        ms_batch_graph, ms_batch = graph_timed(torch, batched, 1, reps=3)
+        nbytes = algorithmic_bytes(n_total, 2, 16)
+        res[RECIPE_NAME[recipe]] = {
+            "per_matrix_python_loop_ms": ms_loop, "per_matrix_graph_ms": ms_graph, "one_batch_launch_ms": ms_batch,
+            "gelem_s": {"per_matrix_python_loop": n_total / ms_loop / 1e6, "per_matrix_graph": n_total / ms_graph / 1e6,
+                        "one_batch_launch": n_total / ms_batch / 1e6},
+            "frac_of_measured_hbm": {"per_matrix_python_loop": nbytes / ms_loop / 1e6 / peaks["hbm_gbs"],
+                                     "per_matrix_graph": nbytes / ms_graph / 1e6 / peaks["hbm_gbs"],
+                                     "one_batch_launch": nbytes / ms_batch / 1e6 / peaks["hbm_gbs"]}}
+    return res
+
+
 def pruned_sweep_report(torch, mxq, wl):
     """The 15 brute-force sweeps of the step once more with the pruned sweep switched on (outside the timed
     region; `value` and `roofline` are always the full sweep): per sweep the time of both modes on the same
@@ -514,14 +549,15 @@ def pruned_sweep_report(torch, mxq, wl):
     return out
 
 
-def spawn_ranks(args) -> int:
-    """`--gpus N` without a torchrun environment: start the N ranks on this node and relay their output."""
+def spawn_ranks(n_ranks: int, script: str | None = None, argv=None) -> int:
+    """`--gpus N` without a torchrun environment: start the N ranks on this node (one process per GPU,
+    rendezvous on 127.0.0.1) with the same command line; their output goes to this process's stdout."""
     with socket.socket() as s:
         s.bind(("127.0.0.1", 0))
         port = s.getsockname()[1]
-    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
-           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
-    return subprocess.call(cmd)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), script or os.path.abspath(__file__)]
+    return subprocess.call(cmd + list(sys.argv[1:] if argv is None else argv))
 
 
 def run_gpu(args) -> None:
@@ -675,6 +711,7 @@ def run_gpu(args) -> None:
     hbm = None if args.skip_extras else config_size_rooflines(torch, mxq, wl, peaks)
     streaming = None if args.skip_extras else streaming_rooflines(torch, mxq, device, peaks)
     pruned = None if args.skip_extras else pruned_sweep_report(torch, mxq, wl)
+    weight_set = None if args.skip_extras else weight_set_report(torch, mxq, device, peaks)
 
     # ---- CPU oracle on a bounded sample of the same workload ------------------------------------
     from oracle import mxq_oracle as orc
@@ -696,7 +733,7 @@ def run_gpu(args) -> None:
         "config": {"workload": WORKLOAD_NAME, "elements_per_step": wl.elems_per_step, "passes_per_step": len(wl.passes),
                    "l2": "search tensor 1 GiB > 126 MB L2; the legs walk their tensors round-robin (277 MB and 201 MB sets)"},
         "roofline": roofline, "legs": legs, "roofline_hbm": hbm, "roofline_hbm_streaming": streaming,
-        "brute_pruned_sweep": pruned, "cpu_baseline": cpu_baseline,
+        "brute_pruned_sweep": pruned, "weight_set_8_layers": weight_set, "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(h2d_bytes),
                 "d2h_bytes_per_step": int(host_out.numel() * 8), "steps": e2e_steps,
                 "what": "the same step with all inputs copied from pinned host memory every step (overlapped with the "
@@ -1009,7 +1046,7 @@ def main() -> None:
         run_reference(args)
         return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
-        sys.exit(spawn_ranks(args))
+        sys.exit(spawn_ranks(args.gpus))
     run_gpu(args)
 
 

@@ -119,6 +119,32 @@ int mxq_quantize_ex(const void* x, int dtype, size_t n, int block_size, int scal
                     float* out_block_sse, void* cuda_stream);
 
 /*
+ * mxq_quantize_batch -- mxq_quantize_ex over a LIST of tensors in one launch: the weight matrices of a
+ * model, say, which the experiments of the paper quantize one recipe at a time (Results, downstream
+ * evaluation: every MLP weight matrix).  One persistent grid walks all tensors, so the launch overhead,
+ * the ramp at the start and the drain at the end are paid once for the whole list instead of once per
+ * tensor.  Outputs are those of mxq_quantize_ex on each tensor, bit for bit.
+ *   h_descs     HOST array of n_tensors descriptors (read during the call: validation, grid size).
+ *   d_descs     DEVICE copy of the same array, made by the caller (it owns the memory; the kernel reads it,
+ *               so it must stay unchanged until the launch has run).  16-byte aligned.
+ *   n_tensors   1 .. 1024 (MXQ_ERR_TOO_LARGE beyond).
+ *   dtype, block_size, scale_fmt, global_scale, d_global_scale   common to all tensors, as for mxq_quantize_ex.
+ *   recipe      any recipe except the brute-force ones (their launches last milliseconds; MXQ_ERR_BAD_ENUM).
+ * Every tensor: x, out_codes, out_scales non-NULL, out_block_sse optional, all 16-byte aligned; n a
+ * positive multiple of 64 (MXQ_ERR_BAD_SHAPE otherwise).
+ */
+typedef struct {
+    const void* x;        /* device, n elements of the call's dtype */
+    uint8_t* out_codes;   /* device, n / 2 bytes */
+    uint8_t* out_scales;  /* device, n / block_size bytes */
+    float* out_block_sse; /* device, n / block_size floats, or NULL */
+    size_t n;             /* element count */
+} mxq_tensor_desc;
+int mxq_quantize_batch(const mxq_tensor_desc* h_descs, const mxq_tensor_desc* d_descs, size_t n_tensors, int dtype,
+                       int block_size, int scale_fmt, int recipe, float global_scale, const float* d_global_scale,
+                       void* cuda_stream);
+
+/*
  * mxq_fake_quantize -- quantize and de-quantize in one pass: out_i = fl32(grid(code_i) * D_b), the
  * values a model computes with when its MLP weights or activations are held in this format (the
  * setting of the downstream experiments in Results).  Bit-identical to mxq_quantize_ex followed by mxq_dequantize, without writing
@@ -158,6 +184,25 @@ float mxq_global_scale_from_amax(float amax);
 size_t mxq_tensor_mse_workspace_bytes(size_t n_blocks);
 int mxq_tensor_mse(const float* d_block_sse, size_t n_blocks, size_t n, double* d_out_mse, void* d_workspace,
                    size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * mxq_quantize_mse -- mxq_quantize_ex and the tensor MSE of its result in one call (Eq. 4 text, "MSE(v, S)";
+ * Results, numerical study: every quantization is scored by its MSE).  The quantization kernel adds up
+ * the block SSEs it produces -- binary64, a fixed order per thread, a fixed tree per CTA -- and a one-CTA
+ * kernel adds the per-CTA sums with the second level of mxq_tensor_mse's tree and divides by n: the
+ * block SSEs are not read back from memory, and out_block_sse may be NULL when only the MSE is wanted.
+ *   x .. out_block_sse, cuda_stream   as for mxq_quantize_ex (every recipe, brute force included).
+ *   d_out_mse     device, one double: (sum of all block SSEs) / n.
+ *   d_workspace   device scratch of at least mxq_tensor_mse_workspace_bytes(n / block_size) bytes;
+ *                 contents are overwritten; no need to clear it.
+ * Codes, scale bytes and block SSEs are those of mxq_quantize_ex bit for bit.  The MSE is deterministic
+ * (same device, same arguments: same bits) and agrees with mxq_tensor_mse on the same SSEs to within the
+ * rounding of binary64 sums taken in a different order (about 1e-15 relative).
+ */
+int mxq_quantize_mse(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe,
+                     float global_scale, const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales,
+                     float* out_block_sse, double* d_out_mse, void* d_workspace, size_t workspace_bytes,
+                     void* cuda_stream);
 
 /*
  * mxq_tensor_mse_static -- mxq_tensor_mse for callers that have no device memory to lend as a

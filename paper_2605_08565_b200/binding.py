@@ -21,7 +21,7 @@ MXQ_ABSMAX, MXQ_ABSMAX_PZ, MXQ_4O6, MXQ_4O6_PZ, MXQ_BRUTE, MXQ_BRUTE_PZ, MXQ_ABS
 MXQ_OPT_BRUTE_PRUNE = 1
 
 EXPORTS = (
-    "mxq_quantize", "mxq_quantize_ex", "mxq_fake_quantize", "mxq_tensor_amax", "mxq_global_scale_from_amax",
+    "mxq_quantize", "mxq_quantize_ex", "mxq_quantize_mse", "mxq_quantize_batch", "mxq_fake_quantize", "mxq_tensor_amax", "mxq_global_scale_from_amax",
     "mxq_tensor_mse_workspace_bytes", "mxq_tensor_mse", "mxq_tensor_mse_static", "mxq_dequantize", "mxq_dequantize_ex",
     "mxq_block_clip_sse", "mxq_histograms", "mxq_segment_mse", "mxq_mask_interval", "mxq_set_option", "mxq_get_option", "mxq_launch_count",
     "mxq_status_string", "mxq_last_cuda_error", "mxq_version",
@@ -30,6 +30,12 @@ EXPORTS = (
 
 class MxqError(RuntimeError):
     pass
+
+
+class TensorDesc(ctypes.Structure):
+    """mxq_tensor_desc of include/mxq.h (one tensor of a multi-tensor launch)."""
+    _fields_ = [("x", ctypes.c_void_p), ("out_codes", ctypes.c_void_p), ("out_scales", ctypes.c_void_p),
+                ("out_block_sse", ctypes.c_void_p), ("n", ctypes.c_size_t)]
 
 
 _lib = None
@@ -50,6 +56,10 @@ def load_library() -> ctypes.CDLL:
     L.mxq_quantize.argtypes = [vp, sz, i32, i32, i32, f32, vp, vp, vp]
     L.mxq_quantize_ex.restype = i32
     L.mxq_quantize_ex.argtypes = [vp, i32, sz, i32, i32, i32, f32, vp, vp, vp, vp, vp]
+    L.mxq_quantize_mse.restype = i32
+    L.mxq_quantize_mse.argtypes = [vp, i32, sz, i32, i32, i32, f32, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.mxq_quantize_batch.restype = i32
+    L.mxq_quantize_batch.argtypes = [vp, vp, sz, i32, i32, i32, i32, f32, vp, vp]
     L.mxq_fake_quantize.restype = i32
     L.mxq_fake_quantize.argtypes = [vp, i32, sz, i32, i32, i32, f32, vp, vp, i32, vp]
     L.mxq_tensor_amax.restype = i32
@@ -142,6 +152,36 @@ def mxq_quantize_ex(x, n, block_size, scale_fmt, recipe, global_scale, d_global_
     _check(load_library().mxq_quantize_ex(_ptr(x), _dtype_id(x), n, block_size, scale_fmt, recipe, global_scale,
                                           _ptr(d_global_scale), _ptr(out_codes), _ptr(out_scales),
                                           _ptr(out_block_sse), _stream(stream, x)))
+
+
+def mxq_quantize_mse(x, n, block_size, scale_fmt, recipe, global_scale, d_global_scale, out_codes, out_scales,
+                     out_block_sse, d_out_mse, d_workspace, stream=None) -> None:
+    """Quantize and score in one call: the tensor MSE comes from partial sums formed inside the quantization kernel."""
+    ws_bytes = d_workspace.numel() * d_workspace.element_size() if d_workspace is not None else 0
+    _check(load_library().mxq_quantize_mse(_ptr(x), _dtype_id(x), n, block_size, scale_fmt, recipe, global_scale,
+                                           _ptr(d_global_scale), _ptr(out_codes), _ptr(out_scales), _ptr(out_block_sse),
+                                           _ptr(d_out_mse), _ptr(d_workspace), ws_bytes, _stream(stream, x)))
+
+
+def make_tensor_descs(items):
+    """Descriptor arrays for ``mxq_quantize_batch``: items = [(x, out_codes, out_scales, out_block_sse or None), ...]
+    (flat CUDA tensors of one dtype on one device).  Returns (host ctypes array, device uint8 tensor holding
+    the same bytes); both must be kept alive until the launch that uses them has run."""
+    if not items:
+        raise MxqError("empty tensor list")
+    arr = (TensorDesc * len(items))()
+    for d, (x, codes, scales, sse) in zip(arr, items):
+        d.x, d.out_codes, d.out_scales, d.out_block_sse, d.n = _ptr(x), _ptr(codes), _ptr(scales), _ptr(sse), x.numel()
+    host = torch.frombuffer(bytearray(bytes(arr)), dtype=torch.uint8)
+    return arr, host.to(items[0][0].device)
+
+
+def mxq_quantize_batch(h_descs, d_descs, n_tensors, dtype_id, block_size, scale_fmt, recipe, global_scale=1.0,
+                       d_global_scale=None, stream=None) -> None:
+    """One launch over a list of tensors; h_descs / d_descs from ``make_tensor_descs``."""
+    _check(load_library().mxq_quantize_batch(ctypes.addressof(h_descs), _ptr(d_descs), n_tensors, dtype_id, block_size,
+                                             scale_fmt, recipe, global_scale, _ptr(d_global_scale),
+                                             _stream(stream, d_descs)))
 
 
 def mxq_fake_quantize(x, n, block_size, scale_fmt, recipe, global_scale, d_global_scale, d_out, stream=None) -> None:

@@ -76,63 +76,84 @@ cudaError_t launch_block_clip_sse(const void* x, int dtype, size_t n, int B, int
 
 // ------------------------------------------------------------------------------------------------
 // Histograms: 16 bins of the 4-bit codes, 256 bins of the scale codes, ADDED to the caller's
-// 64-bit counters.  Per-CTA counts in shared memory (32-bit: a CTA sees fewer than 2^32 entries
-// per trip batch), flushed with 64-bit integer atomics -- integer sums are order-free, so the
-// result is deterministic.
+// 64-bit counters.  The pass is a byte histogram: a code byte holds two codes, so the kernel counts
+// the 256 byte values (one shared-memory integer atomic per TWO codes, one private copy of the
+// table per warp so that only lanes of one warp can collide) and folds them into the 16 code bins at
+// the end; scale bytes are counted the same way.  16-byte loads, no per-code compares.  Per-CTA
+// counts are 32-bit (a CTA sees far fewer than 2^32 bytes), flushed with 64-bit integer atomics --
+// integer sums are order-free, so the result is deterministic.
 // ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void count_bytes_of_word(unsigned int* tab, uint32_t w) {
+    atomicAdd(tab + (w & 0xFFu), 1u);
+    atomicAdd(tab + ((w >> 8) & 0xFFu), 1u);
+    atomicAdd(tab + ((w >> 16) & 0xFFu), 1u);
+    atomicAdd(tab + (w >> 24), 1u);
+}
+
+// Adds the byte histogram of p[0 .. n_bytes) to this warp's table: bytes up to the first 16-byte
+// boundary and past the last one singly (by the first threads of the grid), the rest as 16-byte loads.
+__device__ __forceinline__ void count_byte_range(unsigned int* tab, const uint8_t* p, size_t n_bytes, size_t tid, size_t stride) {
+    size_t head = (16u - (size_t)(reinterpret_cast<uintptr_t>(p) & 15u)) & 15u;
+    if (head > n_bytes) head = n_bytes;
+    const size_t n_vec = (n_bytes - head) / 16;
+    const size_t tail0 = head + n_vec * 16;
+    const uint4* v = reinterpret_cast<const uint4*>(p + head);
+    for (size_t i = tid; i < n_vec; i += stride) {
+        const uint4 w = __ldcs(v + i);
+        count_bytes_of_word(tab, w.x);
+        count_bytes_of_word(tab, w.y);
+        count_bytes_of_word(tab, w.z);
+        count_bytes_of_word(tab, w.w);
+    }
+    if (tid < head) atomicAdd(tab + p[tid], 1u);
+    if (tid < n_bytes - tail0) atomicAdd(tab + p[tail0 + tid], 1u);
+}
+
 __global__ void __launch_bounds__(kThreads) k_histograms(const uint8_t* codes, const uint8_t* scales, size_t n,
                                                          size_t n_blocks, unsigned long long* code_hist,
                                                          unsigned long long* scale_hist) {
-    __shared__ unsigned int sh_code[8][16];   // one copy per warp: fewer same-address collisions
-    __shared__ unsigned int sh_scale[256];
-    for (int i = threadIdx.x; i < 8 * 16; i += kThreads) (&sh_code[0][0])[i] = 0;
-    for (int i = threadIdx.x; i < 256; i += kThreads) sh_scale[i] = 0;
+    constexpr int kWarps = kThreads / 32;
+    __shared__ unsigned int sh_byte[kWarps][256];    // code bytes (two codes each), one table per warp
+    __shared__ unsigned int sh_scale[kWarps][256];
+    __shared__ unsigned long long sh_code[16];
+    for (int i = threadIdx.x; i < kWarps * 256; i += kThreads) {
+        (&sh_byte[0][0])[i] = 0;
+        (&sh_scale[0][0])[i] = 0;
+    }
+    if (threadIdx.x < 16) sh_code[threadIdx.x] = 0;
     __syncthreads();
     const size_t stride = (size_t)gridDim.x * kThreads;
     const size_t tid = (size_t)blockIdx.x * kThreads + threadIdx.x;
     const int w = threadIdx.x >> 5;
-    // codes: 32-bit words of eight codes; n is even, the last (n/2) % 4 bytes are handled bytewise
-    const size_t n_bytes = n / 2, n_words = n_bytes / 4;
-    unsigned int local[16];
-#pragma unroll
-    for (int k = 0; k < 16; ++k) local[k] = 0;
-    for (size_t i = tid; i < n_words; i += stride) {
-        const uint32_t word = reinterpret_cast<const uint32_t*>(codes)[i];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint32_t c = (word >> (4 * k)) & 15u;
-#pragma unroll
-            for (int b = 0; b < 16; ++b) local[b] += (c == (uint32_t)b) ? 1u : 0u;
-        }
-    }
-    if (tid < n_bytes - n_words * 4) {
-        const uint32_t byte = codes[n_words * 4 + tid];
-        atomicAdd(&sh_code[w][byte & 15u], 1u);
-        atomicAdd(&sh_code[w][byte >> 4], 1u);
-    }
-#pragma unroll
-    for (int b = 0; b < 16; ++b)
-        if (local[b]) atomicAdd(&sh_code[w][b], local[b]);
-    for (size_t i = tid; i < n_blocks; i += stride) atomicAdd(&sh_scale[scales[i]], 1u);
+    count_byte_range(sh_byte[w], codes, n / 2, tid, stride);
+    count_byte_range(sh_scale[w], scales, n_blocks, tid, stride);
     __syncthreads();
-    if (threadIdx.x < 16) {
-        unsigned long long t = 0;
-        for (int k = 0; k < 8; ++k) t += sh_code[k][threadIdx.x];
-        if (t) atomicAdd(&code_hist[threadIdx.x], t);
+    // thread t owns byte value t: fold the warps' tables, then the byte counts into the code bins
+    unsigned long long cb = 0, cs = 0;
+#pragma unroll
+    for (int k = 0; k < kWarps; ++k) {
+        cb += sh_byte[k][threadIdx.x];
+        cs += sh_scale[k][threadIdx.x];
     }
-    for (int i = threadIdx.x; i < 256; i += kThreads)
-        if (sh_scale[i]) atomicAdd(&scale_hist[i], (unsigned long long)sh_scale[i]);
+    if (cb) {
+        atomicAdd(&sh_code[threadIdx.x & 15], cb);    // element 2j sits in the low nibble
+        atomicAdd(&sh_code[threadIdx.x >> 4], cb);
+    }
+    if (cs) atomicAdd(&scale_hist[threadIdx.x], cs);
+    __syncthreads();
+    if (threadIdx.x < 16 && sh_code[threadIdx.x]) atomicAdd(&code_hist[threadIdx.x], sh_code[threadIdx.x]);
 }
 
 cudaError_t launch_histograms(const uint8_t* codes, const uint8_t* scales, size_t n, int B, unsigned long long* code_hist,
                               unsigned long long* scale_hist, cudaStream_t s) {
+    static_assert(kThreads == 256, "one thread per byte value in the fold");
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
-    size_t want = (n / 8 + kThreads - 1) / kThreads;
+    size_t want = (n / 32 + kThreads - 1) / kThreads;     // 32 codes per 16-byte load
     if (want == 0) want = 1;
-    // a thread must stay below 2^32 counts: n / (grid * 256) entries each -- true for any n < 2^40 here
-    const size_t cap = (size_t)sm_count(dev) * 8;
+    // a CTA must stay below 2^32 counts per table entry: n / 2 / grid bytes each -- true for any n < 2^40 here
+    const size_t cap = (size_t)sm_count(dev) * 4;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
     k_histograms<<<grid, kThreads, 0, s>>>(codes, scales, n, n / (size_t)B, code_hist, scale_hist);
     count_launch();

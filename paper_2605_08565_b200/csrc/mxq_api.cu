@@ -41,7 +41,8 @@ using namespace mxq;
 // Shared by mxq_quantize_ex (codes + scales, optional SSE) and mxq_fake_quantize (x_hat only).
 static int quantize_common(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe,
                            float global_scale, const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales,
-                           float* out_block_sse, void* out_xhat, int xhat_dtype, void* cuda_stream) {
+                           float* out_block_sse, void* out_xhat, int xhat_dtype, void* cuda_stream,
+                           double* d_mse_partials = nullptr, int* n_mse_partials = nullptr) {
     if (!x || (!out_xhat && (!out_codes || !out_scales))) return MXQ_ERR_NULL;
     if (dtype != MXQ_F32 && dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
     if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
@@ -69,6 +70,11 @@ static int quantize_common(const void* x, int dtype, size_t n, int block_size, i
     a.pow2_rule = (recipe == MXQ_ABSMAX_OCP) ? kPow2Ocp : (recipe == MXQ_ABSMAX_CLIP7) ? kPow2Clip7 : kPow2Eq1;
     a.xhat = out_xhat;
     a.xhat_dtype = xhat_dtype;
+    a.mse_partials = d_mse_partials;
+    a.mse_first = 0;
+    a.mse_n_partials = n_mse_partials;
+    a.batch = nullptr;
+    a.n_tensors = 0;
 
     cudaError_t err;
     if (brute) {
@@ -107,6 +113,70 @@ int mxq_fake_quantize(const void* x, int dtype, size_t n, int block_size, int sc
     if (!d_out) return MXQ_ERR_NULL;
     return quantize_common(x, dtype, n, block_size, scale_fmt, recipe, global_scale, d_global_scale, nullptr, nullptr,
                            nullptr, d_out, out_dtype, cuda_stream);
+}
+
+int mxq_quantize_mse(const void* x, int dtype, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,
+                     const float* d_global_scale, uint8_t* out_codes, uint8_t* out_scales, float* out_block_sse,
+                     double* d_out_mse, void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!out_codes || !out_scales || !d_out_mse) return MXQ_ERR_NULL;
+    if (!d_workspace || workspace_bytes < (size_t)kMsePartials * sizeof(double)) return MXQ_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(d_out_mse) & 7u) || (reinterpret_cast<uintptr_t>(d_workspace) & 7u)) return MXQ_ERR_ALIGN;
+    int n_partials = 0;
+    const int st = quantize_common(x, dtype, n, block_size, scale_fmt, recipe, global_scale, d_global_scale, out_codes,
+                                   out_scales, out_block_sse, nullptr, MXQ_F32, cuda_stream,
+                                   static_cast<double*>(d_workspace), &n_partials);
+    if (st != MXQ_OK) return st;
+    cudaError_t err = launch_mse_final(static_cast<const double*>(d_workspace), n_partials, n, d_out_mse,
+                                       static_cast<cudaStream_t>(cuda_stream));
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
+}
+
+int mxq_quantize_batch(const mxq_tensor_desc* h_descs, const mxq_tensor_desc* d_descs, size_t n_tensors, int dtype,
+                       int block_size, int scale_fmt, int recipe, float global_scale, const float* d_global_scale,
+                       void* cuda_stream) {
+    static_assert(sizeof(mxq_tensor_desc) == sizeof(BatchDesc), "public and internal descriptor layouts agree");
+    if (!h_descs || !d_descs) return MXQ_ERR_NULL;
+    if (n_tensors == 0 || n_tensors > (size_t)kMaxBatch) return MXQ_ERR_TOO_LARGE;
+    if (dtype != MXQ_F32 && dtype != MXQ_BF16) return MXQ_ERR_BAD_ENUM;
+    if (scale_fmt < MXQ_SF_UE8M0 || scale_fmt > MXQ_SF_UE5M3) return MXQ_ERR_BAD_ENUM;
+    if (recipe < MXQ_ABSMAX || recipe > MXQ_ABSMAX_CLIP7 || recipe == MXQ_BRUTE || recipe == MXQ_BRUTE_PZ) return MXQ_ERR_BAD_ENUM;
+    if ((recipe == MXQ_ABSMAX_OCP || recipe == MXQ_ABSMAX_CLIP7) && scale_fmt != MXQ_SF_UE8M0) return MXQ_ERR_BAD_ENUM;
+    if (!valid_block(block_size)) return MXQ_ERR_BAD_SHAPE;
+    if (!d_global_scale && !(global_scale > 0.0f && std::isfinite(global_scale))) return MXQ_ERR_BAD_SCALE;
+    if (!aligned16(d_descs) || (d_global_scale && (reinterpret_cast<uintptr_t>(d_global_scale) & 3u))) return MXQ_ERR_ALIGN;
+    const size_t chunk = (size_t)quantize_chunk_elems(dtype, block_size);
+    size_t rows = 0;
+    for (size_t t = 0; t < n_tensors; ++t) {
+        const mxq_tensor_desc& d = h_descs[t];
+        if (!d.x || !d.out_codes || !d.out_scales) return MXQ_ERR_NULL;
+        if (d.n == 0 || d.n % 64 != 0) return MXQ_ERR_BAD_SHAPE;
+        if (!aligned16(d.x) || !aligned16(d.out_codes) || !aligned16(d.out_scales) || !aligned16(d.out_block_sse)) return MXQ_ERR_ALIGN;
+        rows += (d.n / chunk + 31) / 32;
+    }
+    if (rows >= ((size_t)1 << 32)) return MXQ_ERR_TOO_LARGE;
+    QuantArgs a;
+    a.x = nullptr;
+    a.n_items = 0;
+    a.first_item = 0;
+    a.global_scale = d_global_scale ? 1.0f : global_scale;
+    a.d_global_scale = d_global_scale;
+    a.codes = nullptr;
+    a.scales = nullptr;
+    a.block_sse = nullptr;
+    a.prevent_zero = (recipe == MXQ_ABSMAX_PZ || recipe == MXQ_4O6_PZ) ? 1 : 0;
+    a.pow2_rule = (recipe == MXQ_ABSMAX_OCP) ? kPow2Ocp : (recipe == MXQ_ABSMAX_CLIP7) ? kPow2Clip7 : kPow2Eq1;
+    a.xhat = nullptr;
+    a.xhat_dtype = MXQ_F32;
+    a.mse_partials = nullptr;
+    a.mse_first = 0;
+    a.mse_n_partials = nullptr;
+    a.batch = reinterpret_cast<const BatchDesc*>(d_descs);
+    a.n_tensors = (int)n_tensors;
+    const bool dual = (recipe == MXQ_4O6 || recipe == MXQ_4O6_PZ);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t err = (dtype == MXQ_F32) ? launch_quantize_batch_f32(a, block_size, scale_fmt, dual, rows, s)
+                                         : launch_quantize_batch_bf16(a, block_size, scale_fmt, dual, rows, s);
+    return err == cudaSuccess ? MXQ_OK : cuda_fail(err);
 }
 
 int mxq_quantize(const float* x, size_t n, int block_size, int scale_fmt, int recipe, float global_scale,

@@ -31,6 +31,32 @@ __device__ __forceinline__ void release_dependents() {
 #endif
 }
 
+// Sum of one binary64 value per thread over a CTA of kThreads threads, in a fixed order (a shuffle
+// tree inside each warp, then the warps in order): the same inputs give the same bits.  Every
+// thread of the CTA must call it; the result is valid in thread 0.  scratch: kThreads / 32 doubles
+// of shared memory that nothing else uses until the next barrier.
+__device__ __forceinline__ double cta_sum_fixed_order(double v, double* scratch) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_down_sync(0xFFFFFFFFu, v, o));
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double t = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) t = __dadd_rn(t, scratch[w]);
+    }
+    return t;
+}
+
+// Tail kernels (one warp): the binary64 sum of one SSE per lane, shuffle tree in fixed order, stored
+// as the call's partial number p.mse_first.  Every lane of the warp calls it (0 for an idle lane).
+__device__ __forceinline__ void warp_sum_to_partial(const QuantArgs& p, float sse) {
+    double v = (double)sse;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_down_sync(0xFFFFFFFFu, v, o));
+    if ((threadIdx.x & 31) == 0) p.mse_partials[p.mse_first] = v;
+}
+
 __host__ __device__ constexpr int num_codes(int fmt) { return fmt == kUE4M3 ? 127 : 255; }
 __host__ __device__ constexpr int elem_bytes(int dt) { return dt == kF32 ? 4 : 2; }
 

@@ -14,6 +14,16 @@ constexpr int kMaxDevices = 64;
 // Power-of-two scale rules (UE8M0): Eq. 1 as printed; the OCP wording; the [3.5, 7) target.
 enum { kPow2Eq1 = 0, kPow2Ocp = 1, kPow2Clip7 = 2 };
 
+// One tensor of a multi-tensor launch (device-resident array; the public mxq_tensor_desc has this layout).
+struct BatchDesc {
+    const void* x;
+    uint8_t* codes;
+    uint8_t* scales;
+    float* block_sse;   // may be NULL
+    size_t n;           // elements
+};
+constexpr int kMaxBatch = 1024;   // tensors per multi-tensor launch
+
 struct QuantArgs {
     const void* x;
     size_t n_items;
@@ -27,6 +37,16 @@ struct QuantArgs {
     int pow2_rule;                // UE8M0 only: which power-of-two rule (kPow2Eq1, kPow2Ocp, kPow2Clip7)
     void* xhat;                   // fused fake-quantize output (codes / scales may then be NULL), or NULL
     int xhat_dtype;
+    // fused tensor-MSE partial sums (mxq_quantize_mse), or NULL: CTA i of the main kernel stores the
+    // binary64 sum of the block SSEs it produced in mse_partials[mse_first + i]; the tail kernel (one
+    // warp) stores its sum in mse_partials[mse_first]
+    double* mse_partials;
+    int mse_first;
+    int* mse_n_partials;          // host: receives how many partials the launches of this call write (or NULL)
+    // multi-tensor launch (mxq_quantize_batch): device array of n_tensors descriptors; x, codes, scales,
+    // block_sse and n_items above are then unused
+    const BatchDesc* batch;
+    int n_tensors;
 };
 
 int sm_count(int device);
@@ -54,6 +74,12 @@ void count_launch();
 
 cudaError_t launch_quantize_f32(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
 cudaError_t launch_quantize_bf16(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
+// Multi-tensor launch: a.batch / a.n_tensors set; total_rows = sum over tensors of ceil(chunks / 32),
+// chunks = n / quantize_chunk_elems(dtype, B).
+cudaError_t launch_quantize_batch_f32(const QuantArgs& a, int B, int fmt, bool dual, size_t total_rows, cudaStream_t s);
+cudaError_t launch_quantize_batch_bf16(const QuantArgs& a, int B, int fmt, bool dual, size_t total_rows, cudaStream_t s);
+// Elements one thread of the one-pass kernels handles per trip (at least 64 bytes and one block).
+__host__ __device__ constexpr int quantize_chunk_elems(int dtype, int B) { return dtype == 0 ? (B > 16 ? B : 16) : (B > 32 ? B : 32); }
 cudaError_t launch_fake_quantize_f32(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
 cudaError_t launch_fake_quantize_bf16(const QuantArgs& a, int B, int fmt, bool dual, cudaStream_t s);
 cudaError_t launch_brute_f32(const QuantArgs& a, int B, int fmt, cudaStream_t s);
@@ -81,5 +107,7 @@ cudaError_t launch_segment_mse(const float* sse, size_t n_segments, size_t block
 cudaError_t launch_mask_interval(const void* x, int dtype, size_t n, float lo, float hi, void* out, cudaStream_t s);
 
 constexpr int kMsePartials = 1024;  // fixed first-level width of the MSE tree
+// Second level of the tensor-MSE tree alone: out = (sum of n_partials <= kMsePartials partials) / n.
+cudaError_t launch_mse_final(const double* d_partials, int n_partials, size_t n, double* d_out, cudaStream_t s);
 
 }  // namespace mxq

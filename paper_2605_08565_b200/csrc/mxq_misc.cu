@@ -152,6 +152,12 @@ cudaError_t launch_tensor_mse(const float* d_sse, size_t n_blocks, size_t n, dou
     return err;
 }
 
+cudaError_t launch_mse_final(const double* d_partials, int n_partials, size_t n, double* d_out, cudaStream_t s) {
+    cudaError_t err = launch_pdl(k_mse_final, 1u, (unsigned)kMsePartials, 0, s, d_partials, n_partials, (double)n, d_out);
+    count_launch();
+    return err;
+}
+
 // ------------------------------------------------------------------------------------------------
 // De-quantization: x_hat = fl32(grid(code) * D), D = fl32(S * g).  One thread per 8 elements.
 // ------------------------------------------------------------------------------------------------
@@ -272,7 +278,8 @@ __device__ float tail_eval(const float* v, int B, int c, float g, uint8_t* codes
 template <int FMT>
 __global__ void k_quantize_tail(QuantArgs p, int dtype, int B, int dual) {
     const size_t b = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= p.n_items) return;
+    float my_sse = 0.0f;
+    if (b < p.n_items) {
     const size_t blk = p.first_item + b;
     const float g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
     float v[16];
@@ -310,6 +317,10 @@ __global__ void k_quantize_tail(QuantArgs p, int dtype, int B, int dual) {
             else static_cast<__nv_bfloat16*>(p.xhat)[blk * B + i] = __float2bfloat16_rn(xh);
         }
     }
+    my_sse = s;
+    }
+    // fused tensor-MSE partial sum: the kernel is one warp, every lane takes part (idle lanes add 0)
+    if (p.mse_partials != nullptr) warp_sum_to_partial(p, my_sse);
 }
 
 cudaError_t launch_quantize_tail(const QuantArgs& a, int dtype, int B, int fmt, bool dual, cudaStream_t s) {

@@ -378,7 +378,7 @@ __device__ __forceinline__ int target6_code(float u, int pow2_rule) {
 // (4 eps / 6 and 4 eps / 4 round to code 1; anything below rounds to 0 or 1, anything above to >= 1).
 template <int DT, int B, int FMT, bool DUAL, bool FAKE, bool LEAN>
 __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
-                                               size_t chunk, const uint32_t* raw) {
+                                               size_t chunk, const uint32_t* raw, double& sse_sum) {
     static_assert(!LEAN || (DT == kBF16 && FMT != kUE8M0), "lean path: bf16 input, FP8 scale formats");
     using S = QuantShape<DT, B>;
     constexpr int NBG = S::NBG;
@@ -519,6 +519,7 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             const int b = gi * NBG + j;
             sc[b / 4] |= (uint32_t)c6[j] << (8 * (b % 4));
             sw[b] = __float_as_uint(sse[j]);
+            if constexpr (!FAKE) sse_sum = __dadd_rn(sse_sum, (double)sse[j]);
         }
     }
     if constexpr (FAKE) return;
@@ -542,7 +543,7 @@ __device__ __forceinline__ int ring_index(int k, int lane) {
 // Only one part is live in registers at a time, which keeps as many CTAs resident as for B = 16.
 template <int DT, int B, int FMT, bool DUAL, bool FAKE>
 __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
-                                                    size_t chunk, const uint4* slot_warp, int lane) {
+                                                    size_t chunk, const uint4* slot_warp, int lane, double& sse_sum) {
     using S = QuantShape<DT, B>;
     static_assert(S::C == B && S::NBC == 1, "one block per chunk");
     constexpr int SG = 16;                        // elements per part
@@ -643,6 +644,7 @@ __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const Qu
     store_bytes<B / 2>(p.codes + chunk * (B / 2), pk);
     p.scales[chunk] = (uint8_t)c6;
     if (p.block_sse) p.block_sse[chunk] = sse;
+    sse_sum = __dadd_rn(sse_sum, (double)sse);
 }
 
 // Cooperative staging for chunks above 64 bytes.  With thread-private copies every 16-byte piece
@@ -684,13 +686,187 @@ __device__ __forceinline__ void stage_chunk(uint32_t slot_addr, const void* src,
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
-template <int DT, int B, int FMT, bool DUAL, bool FAKE>
+// Body of the multi-tensor kernel (see k_quantize, BATCH).
+template <int DT, int B, int FMT, bool DUAL>
+__device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTables& T, uint4* ring) {
+    using S = QuantShape<DT, B>;
+    __shared__ uint32_t row0[kMaxBatch + 1];   // row0[t] = first row of tensor t; row0[n_tensors] = all rows
+    __shared__ uint32_t warp_rows[kThreads / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nt = p.n_tensors;
+    // prefix sums of the tensors' row counts: four tensors per thread, a scan over the warps' totals
+    {
+        uint32_t r[4], mine = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int t = threadIdx.x * 4 + q;
+            r[q] = 0;
+            if (t < nt) r[q] = (uint32_t)((p.batch[t].n / S::C + 31) / 32);
+            mine += r[q];
+        }
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) warp_rows[warp] = incl;
+        __syncthreads();
+        uint32_t before = incl - mine;
+        for (int w = 0; w < warp; ++w) before += warp_rows[w];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int t = threadIdx.x * 4 + q;
+            if (t <= nt) row0[t] = before;     // t == nt: the total
+            before += r[q];
+        }
+        if (threadIdx.x == kThreads - 1) row0[nt] = before;   // (nt == 4 * kThreads has no owner above)
+    }
+    QuantConsts k;
+    k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
+    const bool all_short = build_quant_tables<FMT>(T, k.g);   // ends with a barrier: row0[] is complete too
+    k.unit_g = (k.g == 1.0f);
+    k.c_min = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
+    k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;
+    k.u_floor = k.c_min ? __fmul_rn(4.0f, scale_value(FMT, 1)) : 0.0f;
+    k.Rg = 1.0f;
+    k.need_lo = (FMT == kUE8M0) || !k.unit_g;
+    k.m_hi = kFastMax;
+    k.m_lo = 0.0f;
+    if (k.unit_g) {
+        if (FMT == kUE8M0) k.m_lo = 1.0e-30f;
+    } else if (k.g >= kFastMin && k.g <= kFastMax) {
+        k.Rg = __frcp_rn(k.g);
+        k.m_hi = fminf(kFastMax, __fmul_rn(k.g, 1.0e29f));
+        k.m_lo = fmaxf(1.084202172485504434e-19f /* 2^-63 */, (FMT == kUE8M0) ? __fmul_rn(k.g, 1.0e-29f) : 0.0f);
+    } else {
+        k.m_hi = -1.0f;
+        k.m_lo = 0.0f;
+    }
+
+    const uint32_t total_rows = row0[nt];
+    const uint32_t row_stride = gridDim.x * (kThreads / 32);
+    constexpr size_t kChunkBytes = (size_t)S::C * S::EB;
+    constexpr uint32_t kSlotBytes = S::PIECES * kThreads * 16;
+    constexpr int DIST = S::SLOTS - 1;
+    const uint32_t ring_warp = (uint32_t)__cvta_generic_to_shared(ring) + (threadIdx.x - lane) * 16;
+    const uint32_t ring_base = ring_warp + lane * 16;
+
+    // A cursor: the tensor that holds a given row (rows only move forward).  Warp-uniform.
+    struct Cursor {
+        int t;
+        uint32_t first, end;     // rows [first, end) belong to tensor t
+        size_t n_chunks;
+        const char* x;
+    };
+    auto seek = [&](Cursor& c, uint32_t row) {
+        while (row >= c.end && c.t + 1 < nt) {
+            ++c.t;
+            c.first = c.end;
+            c.end = row0[c.t + 1];
+            c.n_chunks = p.batch[c.t].n / S::C;
+            c.x = static_cast<const char*>(p.batch[c.t].x);
+        }
+    };
+    // request the chunks of row `row` into ring slot `fill` (an empty group when there is no such row)
+    auto request = [&](Cursor& c, uint32_t row, int fill) {
+        if (row < total_rows) {
+            seek(c, row);
+            const size_t wchunk = (size_t)(row - c.first) * 32;
+            if constexpr (S::COOP) {
+                stage_warp_chunks<S::PIECES>(ring_warp + fill * kSlotBytes, c.x, kChunkBytes, wchunk, c.n_chunks, lane);
+            } else {
+                stage_chunk<S::PIECES>(ring_base + fill * kSlotBytes, c.x + (wchunk + lane) * kChunkBytes, wchunk + lane < c.n_chunks);
+            }
+        } else {
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+    };
+
+    uint32_t row = blockIdx.x * (kThreads / 32) + warp;
+    if (row >= total_rows) return;    // whole warps leave; no barrier follows
+    Cursor ahead_c = {-1, 0u, 0u, 0, nullptr}, cur_c = {-1, 0u, 0u, 0, nullptr};
+    uint32_t ahead = row;
+#pragma unroll
+    for (int d = 0; d < DIST; ++d) {
+        request(ahead_c, ahead, d);
+        ahead += row_stride;
+    }
+    QuantArgs pl = p;                 // the current tensor's output pointers
+    pl.mse_partials = nullptr;
+    int cur_t = -1;
+    double unused_sum = 0.0;
+    auto row_loop = [&](auto lean_tag) {
+        constexpr bool LEAN = decltype(lean_tag)::value;
+        int slot = 0, fill = DIST % S::SLOTS;
+        for (; row < total_rows; row += row_stride) {
+            asm volatile("cp.async.wait_group %0;" ::"n"(DIST - 1) : "memory");
+            if constexpr (S::COOP) __syncwarp();
+            const uint4* slot_warp = ring + (size_t)slot * (S::PIECES * kThreads) + (threadIdx.x - lane);
+            request(ahead_c, ahead, fill);
+            ahead += row_stride;
+            slot = (slot + 1 == S::SLOTS) ? 0 : slot + 1;
+            fill = (fill + 1 == S::SLOTS) ? 0 : fill + 1;
+            seek(cur_c, row);
+            if (cur_c.t != cur_t) {
+                cur_t = cur_c.t;
+                pl.codes = p.batch[cur_t].codes;
+                pl.scales = p.batch[cur_t].scales;
+                pl.block_sse = p.batch[cur_t].block_sse;
+            }
+            const size_t chunk = (size_t)(row - cur_c.first) * 32 + lane;
+            if (chunk >= cur_c.n_chunks) continue;      // a lane past the end of the tensor's last row
+            if constexpr (B > 16 && !(DUAL && B == 32)) {
+                quantize_long_block<DT, B, FMT, DUAL, false>(pl, T, k, chunk, slot_warp, lane, unused_sum);
+            } else {
+                uint32_t raw[S::PIECES * 4];
+#pragma unroll
+                for (int q = 0; q < S::PIECES; ++q) {
+                    const uint4 w = slot_warp[ring_index<S::COOP>(q, lane)];
+                    raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
+                }
+                quantize_chunk<DT, B, FMT, DUAL, false, LEAN>(pl, T, k, chunk, raw, unused_sum);
+            }
+        }
+    };
+    constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
+    if constexpr (CAN_LEAN) {
+        if (all_short && k.unit_g) row_loop(std::true_type{});
+        else row_loop(std::false_type{});
+    } else {
+        row_loop(std::false_type{});
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+// BATCH: one launch over a list of tensors (same dtype, block size, format, recipe and tensor scale).
+// The unit of distribution is a ROW of 32 consecutive chunks of one tensor (what a warp handles in one
+// trip); tensor t owns ceil(chunks_t / 32) rows of a common index space whose prefix sums every CTA
+// forms in shared memory; a warp walks rows first, first + 8 * gridDim.x, ... and moves its tensor
+// cursor forward when a row passes the end of the current tensor.  Everything else (ring, staging,
+// per-chunk arithmetic) is as in the single-tensor kernel.
+template <int DT, int B, int FMT, bool DUAL, bool FAKE, bool BATCH = false>
 __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     using S = QuantShape<DT, B>;
+    static_assert(S::C == quantize_chunk_elems(DT, B), "host and kernel agree on the chunk size");
     extern __shared__ uint4 ring[];
     __shared__ QuantTables T;
+#ifndef MXQ_NO_L2_PREFETCH
+    if constexpr (!BATCH) {
+        // While the kernel before this one in the stream drains: ask L2 for this thread's first chunk.
+        // A prefetch changes no architectural state and L2 is the point of coherence, so this is safe
+        // even if that kernel is still writing x; the loads themselves come after the wait below.
+        const size_t first = (size_t)blockIdx.x * kThreads + threadIdx.x;
+        if (first < p.n_items)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const char*>(p.x) + first * ((size_t)S::C * S::EB)));
+    }
+#endif
     wait_for_prior_grid();
     release_dependents();
+    if constexpr (BATCH) {
+        quantize_batch_body<DT, B, FMT, DUAL>(p, T, ring);
+        return;
+    }
     // request the first chunks before anything else: their latency hides behind the table build
     const size_t stride = (size_t)gridDim.x * kThreads;
     const int lane = threadIdx.x & 31;
@@ -740,7 +916,10 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
 
     // Thread-private staging: a thread leaves when its chunks are done (no barrier follows).
     // Cooperative staging: the warp stays together, lanes past the end only take part in the copies.
-    if ((S::COOP ? wchunk0 : chunk) >= p.n_items) return;
+    // (with fused MSE partial sums every thread stays for the CTA-wide sum at the end)
+    const bool has_work = (S::COOP ? wchunk0 : chunk) < p.n_items;
+    if (!has_work && (FAKE || p.mse_partials == nullptr)) return;
+    double sse_sum = 0.0;   // binary64 sum of the SSEs of this thread's blocks, in the order it produced them
     // The chunk loop, instantiated with and without the lean per-block path (see quantize_chunk);
     // which one runs is the same for every thread of the launch.
     auto chunk_loop = [&](auto lean_tag) {
@@ -767,7 +946,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
             // blocks longer than 16 elements go part by part, except 4-over-6 at B = 32, which measured
             // slightly faster with the whole block in registers
             if constexpr (B > 16 && !(DUAL && B == 32)) {
-                quantize_long_block<DT, B, FMT, DUAL, FAKE>(p, T, k, chunk, slot_warp, lane);
+                quantize_long_block<DT, B, FMT, DUAL, FAKE>(p, T, k, chunk, slot_warp, lane, sse_sum);
             } else {
                 uint32_t raw[S::PIECES * 4];
 #pragma unroll
@@ -775,16 +954,26 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
                     const uint4 w = slot_warp[ring_index<S::COOP>(q, lane)];
                     raw[4 * q + 0] = w.x; raw[4 * q + 1] = w.y; raw[4 * q + 2] = w.z; raw[4 * q + 3] = w.w;
                 }
-                quantize_chunk<DT, B, FMT, DUAL, FAKE, LEAN>(p, T, k, chunk, raw);
+                quantize_chunk<DT, B, FMT, DUAL, FAKE, LEAN>(p, T, k, chunk, raw, sse_sum);
             }
         }
     };
     constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
-    if constexpr (CAN_LEAN) {
-        if (all_short && k.unit_g) chunk_loop(std::true_type{});
-        else chunk_loop(std::false_type{});
-    } else {
-        chunk_loop(std::false_type{});
+    if (has_work) {
+        if constexpr (CAN_LEAN) {
+            if (all_short && k.unit_g) chunk_loop(std::true_type{});
+            else chunk_loop(std::false_type{});
+        } else {
+            chunk_loop(std::false_type{});
+        }
+    }
+    if constexpr (!FAKE) {
+        if (p.mse_partials != nullptr) {   // launch-uniform: every thread of the CTA is here
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncthreads();               // the table is no longer read: its memory serves as scratch
+            const double total = cta_sum_fixed_order(sse_sum, reinterpret_cast<double*>(&T));
+            if (threadIdx.x == 0) p.mse_partials[p.mse_first + blockIdx.x] = total;
+        }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
@@ -812,23 +1001,37 @@ static cudaError_t launch_quantize_inst(const QuantArgs& a, cudaStream_t stream)
     }
     const size_t n_blocks = a.n_items;
     const size_t n_chunks = n_blocks / S::NBC;
+    const size_t done = n_chunks * S::NBC;
+    // The blocks past the last whole chunk go to the one-warp tail kernel.  With fused MSE partial sums it
+    // runs first and owns partial 0; the CTAs of the main kernel own the partials from 1 on.
+    auto launch_tail = [&]() -> cudaError_t {
+        if (done == n_blocks) return cudaSuccess;
+        QuantArgs t = a;
+        t.first_item = done;
+        t.n_items = n_blocks - done;
+        t.mse_first = 0;
+        return launch_quantize_tail(t, DT, B, FMT, DUAL, stream);
+    };
+    if (a.mse_partials) {
+        err = launch_tail();
+        if (err != cudaSuccess) return err;
+    }
     if (n_chunks > 0) {
         QuantArgs m = a;
         m.n_items = n_chunks;
+        m.mse_first = (done < n_blocks) ? 1 : 0;
         const size_t want = (n_chunks + kThreads - 1) / kThreads;
-        const size_t cap = (size_t)sm_count(dev) * (size_t)resident;
+        size_t cap = (size_t)sm_count(dev) * (size_t)resident;
+        if (a.mse_partials && cap > (size_t)kMsePartials - 1) cap = kMsePartials - 1;
         const unsigned grid = (unsigned)(want < cap ? want : cap);
         err = launch_pdl(k_quantize<DT, B, FMT, DUAL, FAKE>, grid, kThreads, S::RING_BYTES, stream, m);
         count_launch();
         if (err != cudaSuccess) return err;
+        if (a.mse_n_partials) *a.mse_n_partials = (int)grid + m.mse_first;
+    } else if (a.mse_n_partials) {
+        *a.mse_n_partials = (done < n_blocks) ? 1 : 0;
     }
-    const size_t done = n_chunks * S::NBC;
-    if (done < n_blocks) {
-        QuantArgs t = a;
-        t.first_item = done;
-        t.n_items = n_blocks - done;
-        err = launch_quantize_tail(t, DT, B, FMT, DUAL, stream);
-    }
+    if (!a.mse_partials) err = launch_tail();
     return err;
 }
 
@@ -856,6 +1059,55 @@ static cudaError_t launch_quantize_dt(const QuantArgs& a, int B, int fmt, bool d
     case 16: return launch_quantize_fmt<DT, 16, FAKE>(a, fmt, dual, s);
     case 32: return launch_quantize_fmt<DT, 32, FAKE>(a, fmt, dual, s);
     default: return launch_quantize_fmt<DT, 64, FAKE>(a, fmt, dual, s);
+    }
+}
+
+// Multi-tensor launch: one persistent grid over all rows of all tensors.
+template <int DT, int B, int FMT, bool DUAL>
+static cudaError_t launch_quantize_batch_inst(const QuantArgs& a, size_t total_rows, cudaStream_t stream) {
+    using S = QuantShape<DT, B>;
+    static std::atomic<int> ctas_per_sm[kMaxDevices];   // first-use cache; racing threads store the same value
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    int resident = ctas_per_sm[dev].load(std::memory_order_relaxed);
+    if (resident == 0) {
+        err = cudaFuncSetAttribute(k_quantize<DT, B, FMT, DUAL, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)S::RING_BYTES);
+        if (err != cudaSuccess) return err;
+        int n = 0;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_quantize<DT, B, FMT, DUAL, false, true>, kThreads, S::RING_BYTES);
+        if (err != cudaSuccess) return err;
+        resident = n > 0 ? n : 1;
+        ctas_per_sm[dev].store(resident, std::memory_order_relaxed);
+    }
+    const size_t want = (total_rows + kThreads / 32 - 1) / (kThreads / 32);
+    const size_t cap = (size_t)sm_count(dev) * (size_t)resident;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    err = launch_pdl(k_quantize<DT, B, FMT, DUAL, false, true>, grid, kThreads, S::RING_BYTES, stream, a);
+    count_launch();
+    return err;
+}
+
+template <int DT, int B>
+static cudaError_t launch_quantize_batch_fmt(const QuantArgs& a, int fmt, bool dual, size_t rows, cudaStream_t s) {
+    switch (fmt) {
+    case kUE8M0: return dual ? launch_quantize_batch_inst<DT, B, kUE8M0, true>(a, rows, s) : launch_quantize_batch_inst<DT, B, kUE8M0, false>(a, rows, s);
+    case kUE4M3: return dual ? launch_quantize_batch_inst<DT, B, kUE4M3, true>(a, rows, s) : launch_quantize_batch_inst<DT, B, kUE4M3, false>(a, rows, s);
+    default: return dual ? launch_quantize_batch_inst<DT, B, kUE5M3, true>(a, rows, s) : launch_quantize_batch_inst<DT, B, kUE5M3, false>(a, rows, s);
+    }
+}
+
+template <int DT>
+static cudaError_t launch_quantize_batch_dt(const QuantArgs& a, int B, int fmt, bool dual, size_t rows, cudaStream_t s) {
+    switch (B) {
+    case 2: return launch_quantize_batch_fmt<DT, 2>(a, fmt, dual, rows, s);
+    case 4: return launch_quantize_batch_fmt<DT, 4>(a, fmt, dual, rows, s);
+    case 8: return launch_quantize_batch_fmt<DT, 8>(a, fmt, dual, rows, s);
+    case 16: return launch_quantize_batch_fmt<DT, 16>(a, fmt, dual, rows, s);
+    case 32: return launch_quantize_batch_fmt<DT, 32>(a, fmt, dual, rows, s);
+    default: return launch_quantize_batch_fmt<DT, 64>(a, fmt, dual, rows, s);
     }
 }
 

@@ -67,6 +67,15 @@ def test_argument_errors_are_caught_on_the_host(lib):
     assert lib.mxq_dequantize(C, S, 64, 16, 1, 1.0, 0, 0, 0) == 1
     assert lib.mxq_dequantize(C, S, 64, 5, 1, 1.0, X, 0, 0) == 3
     assert lib.mxq_dequantize(C, S, 64, 16, 1, 0.0, X, 0, 0) == 5
+    assert lib.mxq_dequantize_ex(C, S, 64, 16, 1, 0.0, 0, X, 0, 0) == 5
+    assert lib.mxq_dequantize_ex(C, S, 64, 16, 1, 0.0, E + 2, X, 0, 0) == 4     # misaligned device scale
+    assert lib.mxq_dequantize_ex(C, S, 64, 16, 1, 0.0, E, 0, 0, 0) == 1
+    qm = lib.mxq_quantize_mse
+    assert qm(X, 0, 64, 16, 1, 0, 1.0, 0, C, S, E, 0, 0x60000, 8192, 0) == 1           # no MSE output
+    assert qm(X, 0, 64, 16, 1, 0, 1.0, 0, C, S, E, 0x50000, 0, 8192, 0) == 6           # no workspace
+    assert qm(X, 0, 64, 16, 1, 0, 1.0, 0, C, S, E, 0x50000, 0x60000, 4096, 0) == 6     # workspace too small
+    assert qm(X, 0, 60, 16, 1, 0, 1.0, 0, C, S, E, 0x50000, 0x60000, 8192, 0) == 3
+    assert qm(X, 0, 64, 16, 1, 0, 1.0, 0, C, S, E, 0x50004, 0x60000, 8192, 0) == 4
 
 
 def test_binding_refuses_cpu_tensors():

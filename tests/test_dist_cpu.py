@@ -56,3 +56,22 @@ def test_rank_seeds_never_collide_and_single_process_is_a_no_op():
         assert edges[0][0] == 0 and edges[-1][1] == rows
         assert all(a[1] == b[0] for a, b in zip(edges[:-1], edges[1:]))
     assert dist.global_mse(12.0, 48) == 0.25
+
+
+def test_bench_starts_its_own_ranks_when_not_under_torchrun(tmp_path):
+    """`bench.py --gpus N` outside a torchrun environment re-launches itself as N ranks; checked here with
+    a stand-in script that records the environment every rank was given."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "rank_probe.py"
+    script.write_text(
+        "import os, sys\n"
+        "open(os.path.join(sys.argv[1], 'rank' + os.environ['RANK']), 'w').write("
+        "' '.join([os.environ['WORLD_SIZE'], os.environ['LOCAL_RANK'], os.environ['MASTER_ADDR'], sys.argv[2]]))\n")
+    code = ("import sys; sys.path.insert(0, %r); import bench; "
+            "sys.exit(bench.spawn_ranks(2, %r, [%r, '--steps=7']))" % (root, str(script), str(tmp_path)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    assert subprocess.run([sys.executable, "-c", code], env=env, timeout=300).returncode == 0
+    for r in range(2):
+        assert (tmp_path / f"rank{r}").read_text() == f"2 {r} 127.0.0.1 --steps=7"

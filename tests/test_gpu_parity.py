@@ -351,3 +351,72 @@ def test_repeated_launches_give_the_same_bytes(dtype, B, recipe, sweep_mode):
             assert torch.equal(codes, ref[0]) and torch.equal(scales, ref[1])
             assert torch.equal(sse.view(torch.int32), ref[2].view(torch.int32))
     check_parity(x[: 4096 * B].cpu(), B, mxq.MXQ_SF_UE4M3, recipe)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", BLOCKS)
+def test_fused_quantize_mse_equals_quantize_then_tensor_mse(dtype, B, sweep_mode):
+    """``mxq_quantize_mse`` (tensor MSE from partial sums formed inside the quantization kernel) against the
+    two-call path and the oracle: same codes, scale bytes and block SSEs bit for bit; MSE within 1e-12 of
+    the two-call tree and within 1e-6 of the oracle; identical bits when repeated; block SSE output optional.
+    Sizes: only a ragged tail (less than one thread's chunk), whole chunks only, and several CTAs plus a tail."""
+    cases = [(mxq.MXQ_SF_UE4M3, mxq.MXQ_ABSMAX, 1.0), (mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6_PZ, 0.0131),
+             (mxq.MXQ_SF_UE8M0, mxq.MXQ_ABSMAX, 1.0), (mxq.MXQ_SF_UE5M3, mxq.MXQ_BRUTE, 1.0)]
+    chunk = max(B, 64)
+    for n in (B, 256 * chunk, 3 * 256 * chunk + 5 * 64 + (B if B < 8 else 0)):
+        x = _mixed(max(n, 64), 300 + B, dtype)[:n].contiguous()
+        xg = x.cuda()
+        for fmt, recipe, g in cases:
+            codes, scales, sse = mxq.quantize(xg, B, fmt, recipe, g)
+            mse2 = mxq.tensor_mse(sse, n)
+            c1, s1, e1 = mxq.alloc_outputs(n, B, xg.device)
+            ws = torch.full((mxq.mxq_tensor_mse_workspace_bytes(n // B) // 8,), float("nan"), dtype=torch.float64, device="cuda")
+            m1 = torch.empty(1, dtype=torch.float64, device="cuda")
+            mxq.mxq_quantize_mse(xg, n, B, fmt, recipe, g, None, c1, s1, e1, m1, ws)
+            m2 = torch.empty(1, dtype=torch.float64, device="cuda")
+            c2, s2, _ = mxq.alloc_outputs(n, B, xg.device, with_sse=False)
+            mxq.mxq_quantize_mse(xg, n, B, fmt, recipe, g, None, c2, s2, None, m2, ws)       # no SSE output
+            torch.cuda.synchronize()
+            assert torch.equal(codes, c1) and torch.equal(codes, c2)
+            assert torch.equal(scales, s1) and torch.equal(scales, s2)
+            assert torch.equal(sse.view(torch.int32), e1.view(torch.int32))
+            a, b, c = float(mse2.cpu()[0]), float(m1.cpu()[0]), float(m2.cpu()[0])
+            assert b == c                                            # deterministic
+            assert abs(a - b) <= 1e-12 * abs(a) + 1e-300, (n, fmt, recipe, a, b)
+            om = orc.tensor_mse(sse.cpu().numpy(), n)
+            assert abs(b - om) <= MSE_RTOL * abs(om) + 1e-300
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", BLOCKS)
+def test_multi_tensor_launch_equals_one_launch_per_tensor(dtype, B):
+    """``mxq_quantize_batch`` over tensors of very different sizes (one 64-element tensor, sizes that end in the
+    middle of a warp's row of chunks, one that spans many CTAs) against ``mxq_quantize_ex`` on each tensor and,
+    for the first recipe, against the oracle: every output byte identical, the optional SSE output included."""
+    sizes = [64, 64 * 37, 64 * 1024 + 64, 64, 64 * 5000, 64 * 33, 64 * 20000 + 64 * 7]
+    xs = [_mixed(n, 400 + i + B, dtype).cuda() for i, n in enumerate(sizes)]
+    dt = mxq.MXQ_F32 if dtype == torch.float32 else mxq.MXQ_BF16
+    cases = [(mxq.MXQ_SF_UE4M3, mxq.MXQ_ABSMAX, 1.0), (mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6_PZ, 1.0),
+             (mxq.MXQ_SF_UE5M3, mxq.MXQ_4O6, 0.0131), (mxq.MXQ_SF_UE8M0, mxq.MXQ_ABSMAX_OCP, 1.0)]
+    for ci, (fmt, recipe, g) in enumerate(cases):
+        outs = [mxq.alloc_outputs(x.numel(), B, x.device, with_sse=(i % 3 != 1)) for i, x in enumerate(xs)]
+        for c, s_, e in outs:
+            c.fill_(0xAA); s_.fill_(0xAA)
+        h, d = mxq.make_tensor_descs([(x, c, s_, e) for x, (c, s_, e) in zip(xs, outs)])
+        mxq.mxq_quantize_batch(h, d, len(xs), dt, B, fmt, recipe, g)
+        torch.cuda.synchronize()
+        for i, (x, (c, s_, e)) in enumerate(zip(xs, outs)):
+            c1, s1, e1 = mxq.quantize(x, B, fmt, recipe, g)
+            assert torch.equal(c, c1) and torch.equal(s_, s1), (i, fmt, recipe)
+            if e is not None:
+                assert torch.equal(e.view(torch.int32), e1.view(torch.int32)), (i, fmt, recipe)
+            if ci == 0:
+                oc, os_, oe = orc.quantize(inputs.to_numpy_bits(x), B, fmt, recipe, g)
+                assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_)
+    # argument checks happen on the host, before any launch
+    with pytest.raises(mxq.MxqError):
+        mxq.mxq_quantize_batch(h, d, len(xs), dt, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_BRUTE)
+    bad = mxq.alloc_outputs(96, B, xs[0].device)
+    hb, db = mxq.make_tensor_descs([(xs[2][:96], *bad)])
+    with pytest.raises(mxq.MxqError):
+        mxq.mxq_quantize_batch(hb, db, 1, dt, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_ABSMAX)      # 96 is not a multiple of 64
