@@ -75,7 +75,6 @@ struct BruteTables {
     // pruned sweep only
     uint8_t below[kLists - 1][256];  // below[list][E]: members of the paired list whose D has a biased exponent < E
     int flat_zero_min;               // smallest code of the flat list that has the multiplier 0; 256 if none
-    int total;                       // candidates in all lists together
 };
 
 template <int FMT>
@@ -158,11 +157,6 @@ __device__ __forceinline__ void build_brute_tables(BruteTables& T, float g, int 
         T.member[last + 1] = T.member[last];
     }
     if constexpr (PRUNE) {
-        if (c == 0) {
-            int t = 0;
-            for (int l = 0; l < kLists; ++l) t += T.cnt[l];
-            T.total = t;
-        }
         // Exponents rise strictly along a paired list (one member per binade of its class), so
         // member `rank` owns the exponents above its predecessor's up to its own, and the last
         // member also those above.
@@ -473,15 +467,6 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
     // and store nothing), so that the warp can agree on the candidates it leaves out.
     const size_t stride = (size_t)gridDim.x * kThreads;
     const int lane = PRUNE ? (threadIdx.x & 31) : 0;
-    // PRUNE: a warp whose bounds left out less than 1/16 of the candidates over kProbeTrips trips in a
-    // row takes the next kFullTrips trips without forming any bound (limits that cut nothing, the very
-    // same code), then tries the bounds again.  All of it is warp-uniform.
-    constexpr int kProbeTrips = 4, kFullTrips = 28;
-#if defined(MXQ_PRUNE_ALWAYS_FULL)
-    [[maybe_unused]] int full_trips = 1 << 30, probe_left = kProbeTrips, probe_evaluated = 0;
-#else
-    [[maybe_unused]] int full_trips = 0, probe_left = kProbeTrips, probe_evaluated = 0;
-#endif
     double sse_sum = 0.0;                  // binary64 sum of the SSEs of this thread's blocks, in the order it stored them
     for (size_t wbase = (size_t)blockIdx.x * kThreads + threadIdx.x - lane; wbase < p.n_items; wbase += stride) {
         const bool active = wbase + lane < p.n_items;
@@ -493,7 +478,7 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
         {
             float v[G];
             load_elems<DT, G>(p.x, grp * G, v);
-            if (PRUNE && !ONEBLK && full_trips == 0) {   // per-block maxima: only the bounds need them
+            if constexpr (PRUNE && !ONEBLK) {
                 float2 bmax[NBL];
 #pragma unroll
                 for (int k = 0; k < NBL; ++k) bmax[k] = make_float2(0.0f, 0.0f);
@@ -540,46 +525,25 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
                 tb[i] = quotient_pair(v2[i], nDr2, Rr2);
         };
 
-        // every candidate of every list
-        auto full_sweep = [&]() {
-            if (!fast_ok) return;
-            for (int cls = 0; cls < NCLS; ++cls) {
-                const int n0 = T.cnt[2 * cls], n1 = T.cnt[2 * cls + 1];
-                if (n0 + n1 == 0) continue;
-                float2 tb[NP];
-                class_quotients(cls, tb);
-                search_list<B, FMT, false>(T, 2 * cls, 0, n0, v2, tb, best);
-                search_list<B, FMT, true>(T, 2 * cls + 1, 0, n1, v2, tb, best);
-            }
-            // Dref = 1: the elements are their own quotients
-            search_list<B, FMT, false>(T, kFlatList, 0, T.cnt[kFlatList], v2, v2, best);
-        };
         if constexpr (!PRUNE) {
-            full_sweep();
+            if (fast_ok) {
+                for (int cls = 0; cls < NCLS; ++cls) {
+                    const int n0 = T.cnt[2 * cls], n1 = T.cnt[2 * cls + 1];
+                    if (n0 + n1 == 0) continue;
+                    float2 tb[NP];
+                    class_quotients(cls, tb);
+                    search_list<B, FMT, false>(T, 2 * cls, 0, n0, v2, tb, best);
+                    search_list<B, FMT, true>(T, 2 * cls + 1, 0, n1, v2, tb, best);
+                }
+                // Dref = 1: the elements are their own quotients
+                search_list<B, FMT, false>(T, kFlatList, 0, T.cnt[kFlatList], v2, v2, best);
+            }
         } else {
-            // The trip is ONE loop over work items -- (list, first member, count) -- with one call site of
-            // the search per residual kind, so that the kernel's code is no larger than the plain sweep's
-            // (seven inlined copies of the search made every trip miss the instruction cache):
-            //   items 0, 1        class 0, members within nine binades below the zero rule's limit (the
-            //                     optimum of nearly every block lies there, which makes the bounds tight)
-            //   before item 2     the bounds are formed from what has been found so far
-            //   items 2, 3        class 0, the members below that range that the low rule keeps
-            //   items 4 ...       the other classes inside [low, high)
-            //   last item         the flat list
-            // use_bounds false: the bounds cut too little on this warp's recent trips; the same loop runs
-            // with limits that cut nothing (zero and high limit +inf, low limit 0) and forms no bound.
-            const bool use_bounds = (full_trips == 0);
-            if (!use_bounds) --full_trips;
-            int evaluated = 0;         // candidates this trip evaluates (warp-uniform, like every range)
             // Warp-wide steps are taken by every lane; lanes on the general path contribute neutral
             // values and evaluate nothing here.
             constexpr uint32_t kFull = 0xFFFFFFFFu, kInfBits = 0x7F800000u;
-            float wmax = 0.0f;
-            uint32_t zero_limit = kInfBits;
-            if (use_bounds) {
-                wmax = __uint_as_float(__reduce_max_sync(kFull, fast_ok ? __float_as_uint(amax) : 0u));
-                zero_limit = __float_as_uint(__fmul_rn(4.0f, wmax));   // exact: wmax <= 2^60
-            }
+            const float wmax = __uint_as_float(__reduce_max_sync(kFull, fast_ok ? __float_as_uint(amax) : 0u));
+            const uint32_t zero_limit = __float_as_uint(__fmul_rn(4.0f, wmax));   // exact: wmax <= 2^60
             int skipped_min = 256;     // smallest code left out under the zero rule
             uint32_t high_limit = zero_limit, low_limit = 0u;
 
@@ -598,8 +562,26 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
                 }
             };
 
-            // Bounds from what has been found so far: sets low_limit and high_limit.
-            auto form_bounds = [&]() {
+            // First the members of class 0 within nine binades below the zero rule's limit: the
+            // optimum of nearly every block lies there, which makes the bounds below tight.
+            int lo0[2] = {0, 0}, hi0[2] = {0, 0}, probe[2] = {0, 0};
+            const bool have0 = T.cnt[0] + T.cnt[1] > 0;
+            if (have0) {
+                class_ranges(0, lo0, hi0);
+                const uint32_t mant = __float_as_uint(T.clsD[0]) & 0x007FFFFFu;
+                const uint32_t cut_probe = exponent_cut(mant, limit_shifted_down(zero_limit, 9));
+                probe[0] = min(hi0[0], (int)T.below[0][cut_probe]);
+                probe[1] = min(hi0[1], (int)T.below[1][cut_probe]);
+                if (fast_ok) {
+                    float2 tb[NP];
+                    class_quotients(0, tb);
+                    search_list<B, FMT, false>(T, 0, probe[0], hi0[0] - probe[0], v2, tb, best);
+                    search_list<B, FMT, true>(T, 1, probe[1], hi0[1] - probe[1], v2, tb, best);
+                }
+            }
+
+            // Bounds from what has been found so far.
+            {
                 uint32_t ubits = 0u;       // largest best SSE of the thread's blocks
 #pragma unroll
                 for (int k = 0; k < NBT; ++k) ubits = max(ubits, (uint32_t)(best[k] >> 32));
@@ -658,82 +640,36 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
                 const int jw = (int)__reduce_min_sync(kFull, (unsigned)jt);
                 high_limit = limit_shifted_down(zero_limit, jw);
                 if (high_limit == 0u) high_limit = zero_limit;
-            };
+            }
 
-            int lo0[2] = {0, 0}, hi0[2] = {0, 0}, probe[2] = {0, 0};
-            const bool have0 = T.cnt[0] + T.cnt[1] > 0;
+            // the members of class 0 below the first range that the low rule keeps
             if (have0) {
-                class_ranges(0, lo0, hi0);
-                const uint32_t mant = __float_as_uint(T.clsD[0]) & 0x007FFFFFu;
-                const uint32_t cut_probe = exponent_cut(mant, limit_shifted_down(zero_limit, 9));
-                probe[0] = min(hi0[0], (int)T.below[0][cut_probe]);
-                probe[1] = min(hi0[1], (int)T.below[1][cut_probe]);
-            }
-            constexpr int kItems = 2 * NCLS + 3;
-            constexpr int kIdentity = NCLS;     // "class" of the flat list: the elements are their own quotients
-            int lo[2] = {0, 0}, hi[2] = {0, 0};
-            int cur_cls = -1;
-            float2 tb[NP];
-#pragma unroll 1
-            for (int it = 0; it < kItems; ++it) {
-                int list, first, cnt, cls;
-                if (it < 2) {
-                    cls = 0; list = it;
-                    first = it ? probe[1] : probe[0];
-                    cnt = (it ? hi0[1] : hi0[0]) - first;
-                } else if (it < 4) {
-                    if (it == 2) {
-                        if (use_bounds) form_bounds();
-                        if (have0) {
-                            const uint32_t cut_low = exponent_cut(__float_as_uint(T.clsD[0]) & 0x007FFFFFu, low_limit);
+                const uint32_t cut_low = exponent_cut(__float_as_uint(T.clsD[0]) & 0x007FFFFFu, low_limit);
 #pragma unroll
-                            for (int kind = 0; kind < 2; ++kind) lo0[kind] = min(probe[kind], (int)T.below[kind][cut_low]);
-                        }
-                        cur_cls = -1;   // the quotients are formed again rather than kept across the bounds: fewer live registers
-                    }
-                    cls = 0; list = it - 2;
-                    first = (it & 1) ? lo0[1] : lo0[0];
-                    cnt = ((it & 1) ? probe[1] : probe[0]) - first;
-                } else if (it < 2 + 2 * NCLS) {
-                    cls = (it - 2) >> 1;
-                    const int kind = it & 1;
-                    if (kind == 0) {
-                        lo[0] = lo[1] = hi[0] = hi[1] = 0;
-                        if (T.cnt[2 * cls] + T.cnt[2 * cls + 1] > 0) class_ranges(cls, lo, hi);
-                    }
-                    list = 2 * cls + kind;
-                    first = kind ? lo[1] : lo[0];
-                    cnt = (kind ? hi[1] : hi[0]) - first;
-                } else {
-                    // Flat list.  Its members with a subnormal D lie below every normal low limit; the ones
-                    // with the multiplier 0 fall under the zero rule.
-                    cls = kIdentity; list = kFlatList; first = 0; cnt = T.cnt[kFlatList];
-                    if (low_limit >= 0x00800000u) {
-                        skipped_min = min(skipped_min, T.flat_zero_min);
-                        cnt = 0;
-                    }
+                for (int kind = 0; kind < 2; ++kind) lo0[kind] = min(probe[kind], (int)T.below[kind][cut_low]);
+                if (fast_ok && probe[0] - lo0[0] + probe[1] - lo0[1] > 0) {
+                    float2 tb[NP];
+                    class_quotients(0, tb);    // formed again rather than kept: fewer live registers
+                    search_list<B, FMT, false>(T, 0, lo0[0], probe[0] - lo0[0], v2, tb, best);
+                    search_list<B, FMT, true>(T, 1, lo0[1], probe[1] - lo0[1], v2, tb, best);
                 }
-                evaluated += cnt;
-                if (cnt <= 0 || !fast_ok) continue;
-                if (cls != cur_cls) {
-                    if (cls == kIdentity) {
-#pragma unroll
-                        for (int i = 0; i < NP; ++i) tb[i] = v2[i];
-                    } else {
-                        class_quotients(cls, tb);
-                    }
-                    cur_cls = cls;
-                }
-                if (list & 1) search_list<B, FMT, true>(T, list, first, cnt, v2, tb, best);
-                else search_list<B, FMT, false>(T, list, first, cnt, v2, tb, best);
             }
-            if (use_bounds) {
-                probe_evaluated += evaluated;
-                if (--probe_left == 0) {
-                    if (probe_evaluated * 16 > T.total * kProbeTrips * 15) full_trips = kFullTrips;
-                    probe_left = kProbeTrips;
-                    probe_evaluated = 0;
-                }
+            for (int cls = 1; cls < NCLS; ++cls) {
+                if (T.cnt[2 * cls] + T.cnt[2 * cls + 1] == 0) continue;
+                int lo[2], hi[2];
+                class_ranges(cls, lo, hi);
+                if (hi[0] - lo[0] + hi[1] - lo[1] == 0 || !fast_ok) continue;
+                float2 tb[NP];
+                class_quotients(cls, tb);
+                search_list<B, FMT, false>(T, 2 * cls, lo[0], hi[0] - lo[0], v2, tb, best);
+                search_list<B, FMT, true>(T, 2 * cls + 1, lo[1], hi[1] - lo[1], v2, tb, best);
+            }
+            // Flat list.  Its members with a subnormal D lie below every normal low limit; the ones
+            // with the multiplier 0 fall under the zero rule.
+            if (low_limit >= 0x00800000u) {
+                skipped_min = min(skipped_min, T.flat_zero_min);
+            } else if (fast_ok) {
+                search_list<B, FMT, false>(T, kFlatList, 0, T.cnt[kFlatList], v2, v2, best);
             }
             if (fast_ok && skipped_min < 256) {
                 // all-zero quantization: e = v, summed in element order like every other candidate
