@@ -72,8 +72,9 @@ ACT_ROWS, ACT_COLS, ACT_ROTATE = 8192, 4096, 3
 ACT_N = ACT_ROWS * ACT_COLS
 ACT_PASSES = ((UE4M3, True, ABSMAX), (UE5M3, False, ABSMAX), (UE4M3, True, R4O6), (UE5M3, False, R4O6))
 
-CPU_SAMPLE_ELEMS = 1 << 20        # per tensor, cpu_baseline leg
+CPU_SAMPLE_ELEMS = 1 << 22        # per tensor, cpu_baseline leg (about 15 s on 16 host cores)
 REFERENCE_BUDGET_S = 40.0         # wall-clock target of a whole --impl reference run
+REF_SAMPLE_ELEMS = 1 << 18        # longest prefix per tensor the reference arm may take per step
 STREAM_ELEMS = 1 << 27            # tensor size of the streaming (HBM-bound) kernel measurements
 
 
@@ -263,15 +264,15 @@ def run_reference(args) -> None:
     from paper_2605_08565_b200 import inputs
     orc.build()
     threads = host_threads()
-    full = {k: inputs.to_numpy_bits(v) for k, v in make_inputs(0, "cpu", CPU_SAMPLE_ELEMS // 4).items()}
+    full = {k: inputs.to_numpy_bits(v) for k, v in make_inputs(0, "cpu", REF_SAMPLE_ELEMS).items()}
     # Size the per-step sample so that the whole run (warm-up + steps) stays near REFERENCE_BUDGET_S:
     # probe the oracle's rate on a short prefix, then give every step the same prefix of every tensor.
-    probe_frac = 4096.0 / (CPU_SAMPLE_ELEMS // 4)
+    probe_frac = 4096.0 / REF_SAMPLE_ELEMS
     pe, ps = oracle_step(full, threads, probe_frac)
     rate = pe / max(ps, 1e-6)                                    # elements of the pass mix per second
     trips = max(1, args.steps + args.warmup)
     per_step_elems = REFERENCE_BUDGET_S * rate / trips
-    frac = min(1.0, max(probe_frac / 8, per_step_elems / (len(pass_table()) * (CPU_SAMPLE_ELEMS // 4))))
+    frac = min(1.0, max(probe_frac / 8, per_step_elems / (len(pass_table()) * REF_SAMPLE_ELEMS)))
     for _ in range(args.warmup):
         oracle_step(full, threads, frac)
     elems, secs = 0.0, 0.0
@@ -280,7 +281,7 @@ def run_reference(args) -> None:
         elems += e
         secs += s
     value = elems / secs / 1e9
-    n_prefix = max(64, int((CPU_SAMPLE_ELEMS // 4) * frac) // 64 * 64)
+    n_prefix = max(64, int(REF_SAMPLE_ELEMS * frac) // 64 * 64)
     sample_desc = (f"first {n_prefix} elements of every tensor of the step, every pass of the step "
                    f"({len(pass_table())} quantize passes + MSE each, dequantize)")
     print(json.dumps({
@@ -906,20 +907,48 @@ def run_configs(configs, hash_inputs=False):
         rows += acc.rows("C3 8192x4096 bf16 outlier columns", 2, hbm, alu_peak)
         del xs
 
-    if 4 in configs:   # Llama-3-8B-shaped weight set, 224 matrices, one at a time
+    if 4 in configs:   # Llama-3-8B-shaped weight set, 224 matrices: one launch per matrix, then one launch for all
         acc = _Acc(torch, mxq)
         digests["C4"] = _InputDigest(hash_inputs)
+        xs = []
         for layer in range(inputs.LLAMA8B_LAYERS):
             for idx, (name, rows_, cols) in enumerate(inputs.LLAMA8B_LAYER_SHAPES):
                 x = inputs.student_t(rows_ * cols, 4, 1.0 / math.sqrt(cols), 4 + layer * 7 + idx, torch.bfloat16, dev)
                 digests["C4"].add(x)
+                xs.append(x)
                 for B in (8, 16):
                     b = bufs(x.numel(), B)
                     for fmt in (UE4M3, UE5M3):
                         for r in (A, P, R4, R4P, BR, BRP):
                             acc.run((B, fmt, r, "none"), [x], B, fmt, r, 1.0, None, b)
-                del x
-        rows += acc.rows("C4 Llama-3-8B-shaped set (224 matrices, 6.98 G elements)", 2, hbm, alu_peak)
+        name = "C4 Llama-3-8B-shaped set (224 matrices, 6.98 G elements)"
+        rows += acc.rows(name, 2, hbm, alu_peak)
+        # the same set through the multi-tensor entry point: ONE launch per (block size, format, recipe)
+        n_total = sum(x.numel() for x in xs)
+        for B in (8, 16):
+            outs = [mxq.alloc_outputs(x.numel(), B, dev) for x in xs]
+            h, d = mxq.make_tensor_descs([(x, c, s_, e) for x, (c, s_, e) in zip(xs, outs)])
+            mse_out = torch.empty(1, dtype=torch.float64, device=dev)
+            ws = torch.empty(1024, dtype=torch.float64, device=dev)
+            for fmt in (UE4M3, UE5M3):
+                for r in (A, P, R4, R4P):
+                    mxq.mxq_quantize_batch(h, d, len(xs), mxq.MXQ_BF16, B, fmt, r, 1.0)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    mxq.mxq_quantize_batch(h, d, len(xs), mxq.MXQ_BF16, B, fmt, r, 1.0)
+                    e1.record()
+                    tot = 0.0
+                    for x, (c, s_, e) in zip(xs, outs):
+                        mxq.mxq_tensor_mse(e, x.numel() // B, x.numel(), mse_out, ws)
+                        tot += float(mse_out.cpu()[0]) * x.numel()
+                    ms = e0.elapsed_time(e1)
+                    ach = n_total * (2 + 0.5 + 5.0 / B) / ms / 1e6
+                    rows.append({"config": name, "block": B, "scale_fmt": FMT_NAME[fmt], "recipe": RECIPE_NAME[r] + " (one batch launch)",
+                                 "tensor_scale": "none", "elements": n_total, "ms": ms, "gelem_s": n_total / ms / 1e6,
+                                 "mse": tot / n_total, "bound": "hbm", "achieved_gb_s": ach, "frac": ach / hbm,
+                                 "frac_of_8tbs": ach / NOMINAL_HBM_GBS})
+            del outs
+        del xs
 
     if 5 in configs:   # 16384 x 16384 fp32 Laplace, brute force, tensor scale
         x = inputs.laplace(16384 * 16384, 5, torch.float32, dev)
@@ -940,7 +969,7 @@ def run_config_mode(args) -> None:
     configs = (1, 2, 3, 4, 5) if args.config == "all" else tuple(int(c) for c in args.config.split(","))
     res = run_configs(configs, hash_inputs=args.hash_inputs)
     for r in res["rows"]:
-        head = (f'{r["config"][:28]:28s} B={r["block"]:<2d} {r["scale_fmt"]:5s} {r["recipe"]:14s} g={r["tensor_scale"]:9s} '
+        head = (f'{r["config"][:28]:28s} B={r["block"]:<2d} {r["scale_fmt"]:5s} {r["recipe"]:28s} g={r["tensor_scale"]:9s} '
                 f'{r["gelem_s"]:9.1f} GElem/s  ')
         if r["frac"] is None:
             print(head + f'{r["speedup_over_full_sweep"]:8.2f} x the full sweep{"":14s}  mse={r["mse"]:.4e}', file=sys.stderr)

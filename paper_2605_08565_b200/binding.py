@@ -12,7 +12,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# MXQ_LIB: load another build of the library (kernel experiments); the default is the in-tree build
+# MXQ_LIB: path of another build of the library; the default is the in-tree build
 LIB_PATH = os.environ.get("MXQ_LIB") or os.path.join(_HERE, "libmxq.so")
 
 MXQ_F32, MXQ_BF16 = 0, 1

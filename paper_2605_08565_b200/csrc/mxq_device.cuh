@@ -25,11 +25,7 @@ __device__ __forceinline__ void wait_for_prior_grid() { asm volatile("griddepcon
 // completed and flushed its writes, so the ordering of a plain stream is kept.  The dependent grid
 // is released only after EVERY CTA of this grid has executed this instruction (or exited), i.e.
 // when all of them are resident or done: the staged CTAs can never keep this grid off the SMs.
-__device__ __forceinline__ void release_dependents() {
-#ifndef MXQ_NO_EARLY_RELEASE
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-#endif
-}
+__device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Sum of one binary64 value per thread over a CTA of kThreads threads, in a fixed order (a shuffle
 // tree inside each warp, then the warps in order): the same inputs give the same bits.  Every

@@ -29,6 +29,12 @@
 // scale), else an f16->f32 convert plus an FFMA; the square-accumulate FMA, for 4-over-6 one
 // fma.rn.f32x2 serving both candidates.  Blocks whose numbers fall outside the ranges these
 // shortcuts need are redone with IEEE divisions (general path).
+//
+// Variants of the chunk loop inside one kernel, chosen once per launch after the table is built: the
+// lean loop (see quantize_chunk) when no block can leave the shortcuts, the general loop otherwise.
+// Every thread also adds the SSEs of its blocks in binary64; a launch that was given a partial-sum
+// array (mxq_quantize_mse) ends with a fixed-order sum over the CTA.  The BATCH instantiation walks a
+// list of tensors in one launch (quantize_batch_body()).
 #pragma once
 
 #include <cuda_bf16.h>
@@ -54,29 +60,36 @@ struct QuantTables {
     float4 E[256];
 };
 
-// Returns whether EVERY code of the format got class 3 (CTA-uniform).
+// Returns the smallest code of the format whose class is below 3, or num_codes(FMT) if every code
+// has class 3 (CTA-uniform).
 template <int FMT>
-__device__ __forceinline__ bool build_quant_tables(QuantTables& T, float g) {
+__device__ __forceinline__ int build_quant_tables(QuantTables& T, float g) {
     static_assert(kThreads == 256, "one thread per table entry");
-    bool all_short = true;
-    for (int c = threadIdx.x; c < 256; c += blockDim.x) {
-        float D = __uint_as_float(0x7FC00000u), R = 0.0f, w = 0.0f;
-        uint32_t h16 = 0;
-        if (c < num_codes(FMT)) {
-            D = __fmul_rn(scale_value(FMT, c), g);
-            const bool in_range = (D >= kFastMin && D <= kFastMax);
-            if (in_range || D == 0.0f) {
-                if (in_range) R = __frcp_rn(D);
-                const __half hD = __float2half_rn(-D);
-                h16 = (uint32_t)__half_as_ushort(hD);
-                w = (__half2float(hD) == -D) ? 2.0f : 1.0f;
-                if (w == 2.0f && (__float_as_uint(D) & 0x000FFFFFu) == 0u) w = 3.0f;
-            }
+    __shared__ int leading_good[kThreads / 32];   // per warp: how many of its 32 codes, from the first on, have class 3
+    const int c = threadIdx.x;
+    float D = __uint_as_float(0x7FC00000u), R = 0.0f, w = 0.0f;
+    uint32_t h16 = 0;
+    if (c < num_codes(FMT)) {
+        D = __fmul_rn(scale_value(FMT, c), g);
+        const bool in_range = (D >= kFastMin && D <= kFastMax);
+        if (in_range || D == 0.0f) {
+            if (in_range) R = __frcp_rn(D);
+            const __half hD = __float2half_rn(-D);
+            h16 = (uint32_t)__half_as_ushort(hD);
+            w = (__half2float(hD) == -D) ? 2.0f : 1.0f;
+            if (w == 2.0f && (__float_as_uint(D) & 0x000FFFFFu) == 0u) w = 3.0f;
         }
-        T.E[c] = make_float4(D, R, __uint_as_float(h16), w);
-        all_short = all_short && (c >= num_codes(FMT) || w == 3.0f);
     }
-    return __syncthreads_and(all_short) != 0;
+    T.E[c] = make_float4(D, R, __uint_as_float(h16), w);
+    const uint32_t good = __ballot_sync(0xFFFFFFFFu, w == 3.0f);
+    if ((c & 31) == 0) leading_good[c >> 5] = (good == 0xFFFFFFFFu) ? 32 : (__ffs(~good) - 1);
+    __syncthreads();
+    int first_bad = 0;
+#pragma unroll
+    for (int wp = 0; wp < kThreads / 32; ++wp) {
+        if (first_bad == 32 * wp) first_bad += leading_good[wp];
+    }
+    return min(first_bad, num_codes(FMT));
 }
 
 // fl32(v / D) by a reciprocal multiply and ONE residual correction, R = RN(1 / D) correctly rounded,
@@ -346,7 +359,16 @@ struct QuantConsts {
     int c_min;          // smallest admissible code: 1 under prevent-zero (FP8 formats), else 0
     int pow2_rule;      // kPow2Eq1 unless the format is UE8M0 and another rule was asked for
     float u_floor;      // lean path: prevent-zero as a floor on amax / g, 4 * value(code 1), else 0
+    int lean_cmax;      // lean path: every code up to this one has class 3 (UE5M3: the codes above it take the general path)
 };
+
+// The lean path runs when there is no tensor scale and every code of the table has class 3 (UE4M3), or
+// every code but the last few (UE5M3: the scales from 2^16 on are not f16 values; a block that lands on
+// one of them is redone on the general path).
+template <int FMT>
+__device__ __forceinline__ bool lean_allowed(int first_bad, bool unit_g) {
+    return unit_g && first_bad >= (FMT == kUE5M3 ? num_codes(FMT) - 16 : num_codes(FMT));
+}
 
 // Both 4-over-6 scale codes of a block from one conversion (UE4M3): the code for w6 in bits 0..7,
 // the code for w4 in bits 8..15.
@@ -367,8 +389,9 @@ __device__ __forceinline__ int target6_code(float u, int pow2_rule) {
 }
 
 // LEAN (launch-uniform; bf16 input, FP8 scale format, no tensor scale, every decode scale of the
-// table of class 3): nothing of a block can leave the shortcuts, so the per-block class and range
-// tests, the tensor-scale quotient and the general path are left out.  Why no magnitude test is
+// table of class 3 -- for UE5M3 all but its last few codes, whose scales from 2^16 on are not f16
+// values: a group whose code lands there is redone on the general path): nothing of a block can leave
+// the shortcuts, so the per-block class and range tests and the tensor-scale quotient are left out.  Why no magnitude test is
 // needed: the one-multiply quotient neither forms a residual nor divides (a product that
 // overflows or underflows still rounds to the FP4 code of the true quotient, 6 or 0 with the sign
 // of the element); amax / 6 by multiply-and-correct is exact from 1e-30 to 1e30, below that every
@@ -402,6 +425,7 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
 #pragma unroll
             for (int i = 0; i < B; ++i) a = fmaxf(a, fabsf(v[j * B + i]));
             if constexpr (LEAN) {
+                m[j] = a;
                 const float uf = fmaxf(a, k.u_floor);
                 const float w6 = div6_fast(uf);
                 if constexpr (DUAL && FMT == kUE4M3) {
@@ -433,10 +457,17 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
         float sse[NBG], sse4[NBG];
 #pragma unroll
         for (int j = 0; j < NBG; ++j) sse[j] = sse4[j] = 0.0f;
-        if constexpr (LEAN) {
+        bool lean_group = LEAN;
+        if constexpr (LEAN && FMT == kUE5M3) {   // a code above the class-3 range: this group takes the general path
+            int cmx = 0;
+#pragma unroll
+            for (int j = 0; j < NBG; ++j) cmx = max(cmx, DUAL ? max(c6[j], c4[j]) : c6[j]);
+            lean_group = cmx <= k.lean_cmax;
+        }
+        if (LEAN && lean_group) {
             if constexpr (DUAL) encode_group_fast_dual<B, true, true>(v, E6, E4, pk, pk4, sse, sse4);
             else encode_group_fast<B, true, true>(v, E6, pk, sse);
-        } else if (wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
+        } else if (!LEAN && wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
             // one decision for both candidates.  bf16 input: the one-multiply quotient with the f16
             // residual when every decode scale of the group is short, else the general shortcuts.
             constexpr bool SH = (DT == kBF16);
@@ -724,11 +755,12 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
     }
     QuantConsts k;
     k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    const bool all_short = build_quant_tables<FMT>(T, k.g);   // ends with a barrier: row0[] is complete too
+    const int first_bad = build_quant_tables<FMT>(T, k.g);   // contains a barrier: row0[] is complete too
     k.unit_g = (k.g == 1.0f);
     k.c_min = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;
     k.u_floor = k.c_min ? __fmul_rn(4.0f, scale_value(FMT, 1)) : 0.0f;
+    k.lean_cmax = first_bad - 1;
     k.Rg = 1.0f;
     k.need_lo = (FMT == kUE8M0) || !k.unit_g;
     k.m_hi = kFastMax;
@@ -831,7 +863,7 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
     };
     constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
     if constexpr (CAN_LEAN) {
-        if (all_short && k.unit_g) row_loop(std::true_type{});
+        if (lean_allowed<FMT>(first_bad, k.unit_g)) row_loop(std::true_type{});
         else row_loop(std::false_type{});
     } else {
         row_loop(std::false_type{});
@@ -851,7 +883,6 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     static_assert(S::C == quantize_chunk_elems(DT, B), "host and kernel agree on the chunk size");
     extern __shared__ uint4 ring[];
     __shared__ QuantTables T;
-#ifndef MXQ_NO_L2_PREFETCH
     if constexpr (!BATCH) {
         // While the kernel before this one in the stream drains: ask L2 for this thread's first chunk.
         // A prefetch changes no architectural state and L2 is the point of coherence, so this is safe
@@ -860,7 +891,6 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
         if (first < p.n_items)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const char*>(p.x) + first * ((size_t)S::C * S::EB)));
     }
-#endif
     wait_for_prior_grid();
     release_dependents();
     if constexpr (BATCH) {
@@ -890,11 +920,12 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     }
     QuantConsts k;
     k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    const bool all_short = build_quant_tables<FMT>(T, k.g);
+    const int first_bad = build_quant_tables<FMT>(T, k.g);
     k.unit_g = (k.g == 1.0f);
     k.c_min = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;
     k.u_floor = k.c_min ? __fmul_rn(4.0f, scale_value(FMT, 1)) : 0.0f;
+    k.lean_cmax = first_bad - 1;
     k.Rg = 1.0f;
     // Ranges of a block maximum m for which u = fl(m / g) and fl(u / 6) come out exact from the
     // multiply-and-correct forms.  The FP8 formats round every u below 2^-20 to code 0, so an
@@ -961,7 +992,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
     if (has_work) {
         if constexpr (CAN_LEAN) {
-            if (all_short && k.unit_g) chunk_loop(std::true_type{});
+            if (lean_allowed<FMT>(first_bad, k.unit_g)) chunk_loop(std::true_type{});
             else chunk_loop(std::false_type{});
         } else {
             chunk_loop(std::false_type{});

@@ -420,3 +420,34 @@ def test_multi_tensor_launch_equals_one_launch_per_tensor(dtype, B):
     hb, db = mxq.make_tensor_descs([(xs[2][:96], *bad)])
     with pytest.raises(mxq.MxqError):
         mxq.mxq_quantize_batch(hb, db, 1, dt, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_ABSMAX)      # 96 is not a multiple of 64
+
+
+def test_multi_tensor_launch_with_hundreds_of_small_tensors():
+    """777 tensors of 256 to 2560 elements in one launch (the prefix sums over the tensor list span several
+    warps of the scan; most tensors end inside a warp's row), and the largest list the entry point takes.
+    Lengths are multiples of 256 so that every slice of the shared output buffers is 16-byte aligned."""
+    gen = torch.Generator().manual_seed(5)
+    B = 16
+    for count in (777, 1024):
+        sizes = (256 * torch.randint(1, 11, (count,), generator=gen)).tolist()
+        big = _mixed(sum(sizes), 600 + count, torch.bfloat16).cuda()
+        xs, o = [], 0
+        for n in sizes:
+            xs.append(big[o:o + n])
+            o += n
+        codes = torch.zeros(sum(sizes) // 2, dtype=torch.uint8, device="cuda")
+        scales = torch.zeros(sum(sizes) // B, dtype=torch.uint8, device="cuda")
+        sse = torch.zeros(sum(sizes) // B, dtype=torch.float32, device="cuda")
+        items, o = [], 0
+        for n, x in zip(sizes, xs):
+            items.append((x, codes[o // 2:(o + n) // 2], scales[o // B:(o + n) // B], sse[o // B:(o + n) // B]))
+            o += n
+        h, d = mxq.make_tensor_descs(items)
+        mxq.mxq_quantize_batch(h, d, count, mxq.MXQ_BF16, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6)
+        # blocks never straddle tensors here (every length is a multiple of 64), so the whole buffer quantized as
+        # one tensor must give the same bytes
+        c1, s1, e1 = mxq.quantize(big, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6)
+        torch.cuda.synchronize()
+        assert torch.equal(codes, c1) and torch.equal(scales, s1) and torch.equal(sse.view(torch.int32), e1.view(torch.int32))
+    with pytest.raises(mxq.MxqError):
+        mxq.mxq_quantize_batch(h, d, 1025, mxq.MXQ_BF16, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6)

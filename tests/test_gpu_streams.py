@@ -127,3 +127,56 @@ def test_row_sharded_hierarchical_quantize_as_two_ranks(tmp_path, recipe):
     # the sharded MSE is exactly (sum of the two ranks' binary64 tree sums) / n
     s = [float(p["local_sum"]) for p in parts]
     assert float(parts[0]["mse"]) == (s[0] + s[1]) / (rows * cols)
+
+
+def test_entry_points_called_from_four_host_threads_at_once():
+    """Four host threads, each with its own stream and tensors, run abs-max -> quantize + MSE -> de-quantize
+    sixteen times over while a fifth flips the process-wide brute-force option: every thread must get the
+    bytes that a quiet single-threaded run gets (the header's statement on threads)."""
+    import threading
+    n, B = 1 << 18, 16
+    xs = [inputs.student_t(n, 5, 0.02, 50 + i, torch.bfloat16).cuda() for i in range(4)]
+    recipes = [mxq.MXQ_ABSMAX, mxq.MXQ_4O6, mxq.MXQ_BRUTE, mxq.MXQ_ABSMAX_PZ]
+    want = []
+    for x, r in zip(xs, recipes):
+        c, s_, e = mxq.quantize(x, B, mxq.MXQ_SF_UE4M3, r)
+        want.append((c.clone(), s_.clone(), e.clone(), mxq.tensor_mse(e, n).clone()))
+    torch.cuda.synchronize()
+    errors = []
+    stop = threading.Event()
+
+    def worker(i):
+        try:
+            torch.cuda.set_device(0)
+            st = torch.cuda.Stream()
+            c, s_, e = mxq.alloc_outputs(n, B, xs[i].device)
+            m = torch.empty(1, dtype=torch.float64, device="cuda")
+            ws = torch.empty(1024, dtype=torch.float64, device="cuda")
+            for _ in range(16):
+                mxq.mxq_quantize_mse(xs[i], n, B, mxq.MXQ_SF_UE4M3, recipes[i], 1.0, None, c, s_, e, m, ws, stream=st)
+                st.synchronize()
+                ok = (torch.equal(c, want[i][0]) and torch.equal(s_, want[i][1])
+                      and torch.equal(e.view(torch.int32), want[i][2].view(torch.int32))
+                      and abs(float(m.cpu()[0]) - float(want[i][3].cpu()[0])) <= 1e-12 * float(want[i][3].cpu()[0]))
+                if not ok:
+                    errors.append(i)
+        except Exception as ex:      # noqa: BLE001
+            errors.append((i, repr(ex)))
+
+    def flipper():
+        v = 0
+        while not stop.is_set():
+            v ^= 1
+            mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, v)
+
+    ths = [threading.Thread(target=worker, args=(i,)) for i in range(4)]
+    fl = threading.Thread(target=flipper)
+    fl.start()
+    for t in ths:
+        t.start()
+    for t in ths:
+        t.join()
+    stop.set()
+    fl.join()
+    mxq.mxq_set_option(mxq.MXQ_OPT_BRUTE_PRUNE, 0)
+    assert not errors, errors
