@@ -20,36 +20,56 @@ __device__ __forceinline__ float warp_max(float m) {
     return m;
 }
 
+// Zeroes the running maximum and, when a tensor scale is wanted, the word that first counts the CTAs
+// that have finished and then receives the scale.
+__global__ void k_amax_init(uint32_t* amax_bits, uint32_t* g_word) {
+    wait_for_prior_grid();
+    release_dependents();
+    *amax_bits = 0u;
+    if (g_word) *g_word = 0u;
+}
+
+// One CTA reads tiles of U x 256 sixteen-byte vectors (U independent loads per thread in flight).  The
+// last CTA to finish (a count in g_word) turns the maximum into g = amax / (6 * 448), the tensor
+// maximum mapped to the top of FP4 times the top of E4M3, and stores it over the count.  Loads are
+// streaming (evict-first): reading with the default policy, so that the quantize pass that follows finds
+// the tensor in L2, was measured on 33 to 117 MB tensors and gains nothing (that pass is not DRAM-bound
+// enough at those sizes), while it slows this kernel by 5 %.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) k_tensor_amax(const void* x, size_t n, uint32_t* out_bits) {
+__global__ void __launch_bounds__(kThreads) k_tensor_amax(const void* x, size_t n, uint32_t* out_bits, uint32_t* g_word) {
     constexpr int VEC = 16 / elem_bytes(DT);
+    constexpr int U = 4;
     const size_t n_vec = n / VEC;
-    const size_t stride = (size_t)gridDim.x * kThreads;
+    const size_t tile = (size_t)U * kThreads;
     const uint4* p = static_cast<const uint4*>(x);
-    float m = 0.0f;
-    if constexpr (DT == kF32) {
-        float m0 = 0.f, m1 = 0.f, m2 = 0.f, m3 = 0.f;
-        for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec; i += stride) {
-            const uint4 w = __ldcs(p + i);
-            m0 = fmaxf(m0, fabsf(__uint_as_float(w.x)));
-            m1 = fmaxf(m1, fabsf(__uint_as_float(w.y)));
-            m2 = fmaxf(m2, fabsf(__uint_as_float(w.z)));
-            m3 = fmaxf(m3, fabsf(__uint_as_float(w.w)));
-        }
-        m = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-    } else {
-        // magnitudes of bf16 order like their 15-bit patterns: packed unsigned 16-bit max
-        uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
-        for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec; i += stride) {
-            const uint4 w = __ldcs(p + i);
-            a0 = __vmaxu2(a0, w.x & 0x7FFF7FFFu);
-            a1 = __vmaxu2(a1, w.y & 0x7FFF7FFFu);
-            a2 = __vmaxu2(a2, w.z & 0x7FFF7FFFu);
-            a3 = __vmaxu2(a3, w.w & 0x7FFF7FFFu);
-        }
-        const uint32_t a = __vmaxu2(__vmaxu2(a0, a1), __vmaxu2(a2, a3));
-        m = fmaxf(__uint_as_float(a << 16), __uint_as_float(a & 0xFFFF0000u));
+    {   // while the kernel before this one drains: ask L2 for this thread's first vector (no architectural effect)
+        const size_t first = (size_t)blockIdx.x * tile + threadIdx.x;
+        if (first < n_vec) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + first));
     }
+    wait_for_prior_grid();
+    release_dependents();
+    float m = 0.0f;
+    uint32_t a16 = 0;   // bf16: magnitudes order like their 15-bit patterns, packed unsigned 16-bit max
+    for (size_t base = (size_t)blockIdx.x * tile; base < n_vec; base += (size_t)gridDim.x * tile) {
+        uint4 w[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t i = base + (size_t)u * kThreads + threadIdx.x;
+            w[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (i < n_vec) w[u] = __ldcs(p + i);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if constexpr (DT == kF32) {
+                m = fmaxf(fmaxf(m, fabsf(__uint_as_float(w[u].x))), fabsf(__uint_as_float(w[u].y)));
+                m = fmaxf(fmaxf(m, fabsf(__uint_as_float(w[u].z))), fabsf(__uint_as_float(w[u].w)));
+            } else {
+                a16 = __vmaxu2(a16, __vmaxu2(w[u].x & 0x7FFF7FFFu, w[u].y & 0x7FFF7FFFu));
+                a16 = __vmaxu2(a16, __vmaxu2(w[u].z & 0x7FFF7FFFu, w[u].w & 0x7FFF7FFFu));
+            }
+        }
+    }
+    if constexpr (DT == kBF16) m = fmaxf(__uint_as_float(a16 << 16), __uint_as_float(a16 & 0xFFFF0000u));
     if (blockIdx.x == 0 && threadIdx.x < (unsigned)(n - n_vec * VEC)) {  // ragged end, scalar
         const size_t i = n_vec * VEC + threadIdx.x;
         float v;
@@ -64,38 +84,37 @@ __global__ void __launch_bounds__(kThreads) k_tensor_amax(const void* x, size_t 
     if (threadIdx.x < 32) {
         m = threadIdx.x < kThreads / 32 ? warp_m[threadIdx.x] : 0.0f;
         m = warp_max(m);
-        if (threadIdx.x == 0) atomicMax(out_bits, __float_as_uint(m));
+        if (threadIdx.x == 0) {
+            atomicMax(out_bits, __float_as_uint(m));
+            if (g_word) {
+                __threadfence();
+                if (atomicAdd(g_word, 1u) == gridDim.x - 1) {   // every CTA's maximum is in: this one writes the scale
+                    __threadfence();
+                    const float a = __uint_as_float(atomicMax(out_bits, 0u));
+                    *reinterpret_cast<float*>(g_word) = (a > 0.0f && a <= 3.402823466e38f) ? __fdiv_rn(a, 2688.0f) : 1.0f;
+                }
+            }
+        }
     }
 }
 
-// g = amax / (6 * 448): the tensor maximum maps to the top of FP4 times the top of E4M3.
-__global__ void k_global_scale(const float* amax, float* g) {
-    wait_for_prior_grid();
-    release_dependents();
-    const float a = *amax;
-    *g = (a > 0.0f && a <= 3.402823466e38f) ? __fdiv_rn(a, 2688.0f) : 1.0f;
-}
-
 cudaError_t launch_tensor_amax(const void* x, int dtype, size_t n, float* d_amax, float* d_g, cudaStream_t s) {
-    cudaError_t err = cudaMemsetAsync(d_amax, 0, sizeof(float), s);
+    uint32_t* amax_bits = reinterpret_cast<uint32_t*>(d_amax);
+    uint32_t* g_word = reinterpret_cast<uint32_t*>(d_g);
+    cudaError_t err = launch_pdl(k_amax_init, 1u, 1u, 0, s, amax_bits, g_word);
+    count_launch();
     if (err != cudaSuccess) return err;
     int dev = 0;
     err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     const size_t n_vec = n / (16 / elem_bytes(dtype));
-    size_t want = (n_vec + kThreads - 1) / kThreads;
+    size_t want = (n_vec + 4 * kThreads - 1) / (4 * kThreads);
     if (want == 0) want = 1;
     const size_t cap = (size_t)sm_count(dev) * 8;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
-    if (dtype == kF32) k_tensor_amax<kF32><<<grid, kThreads, 0, s>>>(x, n, reinterpret_cast<uint32_t*>(d_amax));
-    else k_tensor_amax<kBF16><<<grid, kThreads, 0, s>>>(x, n, reinterpret_cast<uint32_t*>(d_amax));
+    if (dtype == kF32) err = launch_pdl(k_tensor_amax<kF32>, grid, (unsigned)kThreads, 0, s, x, n, amax_bits, g_word);
+    else err = launch_pdl(k_tensor_amax<kBF16>, grid, (unsigned)kThreads, 0, s, x, n, amax_bits, g_word);
     count_launch();
-    err = cudaGetLastError();
-    if (err != cudaSuccess) return err;
-    if (d_g) {
-        err = launch_pdl(k_global_scale, 1u, 1u, 0, s, (const float*)d_amax, d_g);
-        count_launch();
-    }
     return err;
 }
 

@@ -23,7 +23,8 @@
 // Arithmetic per element (kernel time follows the number of warp instructions): bf16 -> binary32
 // by a mixed-precision add of -0 (FMA pipe); the exact quotient by the decode scale, two elements
 // per instruction (reciprocal multiply + one residual correction; for bf16 input and decode scales
-// of at most four significant bits a single multiply rounded toward zero); half an FP4 pack, half an FP4
+// of at most four significant bits, or long ones whose reciprocal passed the per-launch check, a single
+// multiply rounded toward zero); half an FP4 pack, half an FP4
 // unpack; the residual as fma.rn.f32.f16 straight from the unpacked f16 grid value whenever the
 // decode scales of the group are exactly representable in f16 (always, for UE4M3 without a tensor
 // scale), else an f16->f32 convert plus an FFMA; the square-accumulate FMA, for 4-over-6 one
@@ -51,45 +52,118 @@ namespace mxq {
 // Per-code table entry, one 128-bit shared-memory read per block and candidate:
 //   x  D = fl32(value(c) * g); NaN for codes that do not exist
 //   y  R = RN(1 / D) when 2^-60 <= D <= 2^60, else 0
-//   z  bits: f16(-D) in the low half
+//   z  bits: f16(-D) in the low half; in a bf16 kernel under a tensor scale that is not a power of two,
+//      the reciprocal for the one-multiply quotient instead (R or a neighbour of it, see
+//      build_quant_tables())
 //   w  0: general path only; 1: shortcuts valid; 2: shortcuts valid and -D exact in f16; 3: as 2,
 //      and D has at most four significant bits (every decode scale of the FP8 and power-of-two
-//      formats when the tensor scale is a power of two).
+//      formats when the tensor scale is a power of two).  Where z holds a reciprocal, w is 0 or 1.
 //      D = 0 counts as valid with R = 0: every quotient comes out as a zero with the sign of v.
 struct QuantTables {
     float4 E[256];
 };
 
-// Returns the smallest code of the format whose class is below 3, or num_codes(FMT) if every code
-// has class 3 (CTA-uniform).
-template <int FMT>
-__device__ __forceinline__ int build_quant_tables(QuantTables& T, float g) {
+// Does the FP4 code of RZ(v * R) equal the FP4 code of fl32(v / D) for EVERY bf16 value v?  (D a
+// normal binary32 number, R within a few units in the last place of 1 / D.)  Both codes are
+// non-decreasing step functions of v >= 0 (and odd in v), so they agree everywhere iff they agree where
+// either of them steps.  The steps are next to the seven points M * D, M a rounding midpoint of the FP4
+// grid: the product and the true quotient differ by less than 2^-21 relative, bf16 values are at least
+// 2^-8 apart, so at the second bf16 value above M * D both are safely above M and at the first one
+// below floor_bf16(M * D) both safely below.  That leaves v0 = floor_bf16(M * D) and the bf16 value
+// after it: two values per midpoint, tried here with the very instructions the hot loop uses (this
+// function does one midpoint).
+__device__ __forceinline__ bool one_multiply_codes_agree_at(float D, float R, float M) {
+    const uint32_t b0 = __float_as_uint(__fmul_rz(M, D)) & 0xFFFF0000u;   // floor to 8 significant bits
+    const float v0 = __uint_as_float(b0), v1 = __uint_as_float(b0 + 0x10000u);
+    uint32_t codes;   // byte 0: {fl(v0 / D), RZ(v0 R)}, byte 1: the same for v1, FP4 codes in the two nibbles
+    asm("{\n"
+        " .reg .b8 b0, b1;\n"
+        " cvt.rn.satfinite.e2m1x2.f32 b0, %1, %2;\n"
+        " cvt.rn.satfinite.e2m1x2.f32 b1, %3, %4;\n"
+        " mov.b32 %0, {b0, b1, b0, b1};\n"
+        "}"
+        : "=r"(codes)
+        : "f"(__fdiv_rn(v0, D)), "f"(__fmul_rz(v0, R)), "f"(__fdiv_rn(v1, D)), "f"(__fmul_rz(v1, R)));
+    return (((codes >> 4) ^ codes) & 0x0F0Fu) == 0u;
+}
+
+// Builds the table.  first_bad: the smallest code of the format whose class is below 3, or
+// num_codes(FMT) if every code has class 3.  Returns (CTA-uniform) whether the one-multiply quotient
+// with the reciprocals in E[].z may be used for every entry of class 1 (BF16_IN kernels under a tensor
+// scale that is not a power of two; false otherwise).
+//
+// The one-multiply quotient under such a tensor scale.  Decode scales then have 24 significant bits, and
+// whether RZ(v * R) has the FP4 code of fl(v / D) for every bf16 v depends on how the roundings fall
+// where a bf16 value lies within 2^-23 or so of M * D.  With g = amax / 2688 from a bf16 amax that
+// happens for most significands (v / D is then a ratio of small integers and hits midpoints exactly in
+// real arithmetic; RN(1 / D) alone passes for 40 of the 128 amax significands).  It depends on the
+// significand of D only (v, D and the quotient all scale by powers of two), and the scales of a table
+// have at most eight significands: those of fl((1 + m / 8) * g).  So the check runs per significand
+// class, for three candidate reciprocals (RN(1 / D), the float above it, the float below it) and the
+// seven midpoints, on 168 threads, with the tensor scale's significand moved to [1, 2).  Each class
+// takes the first candidate that passes at all seven midpoints (126 of those 128 significands then
+// pass in every class); an entry records it only if its own significand bits are those of its class
+// (always, unless g is denormal).  If some class has no passing candidate the launch keeps the
+// corrected quotient throughout.
+template <int FMT, bool BF16_IN>
+__device__ __forceinline__ bool build_quant_tables(QuantTables& T, float g, int& first_bad) {
     static_assert(kThreads == 256, "one thread per table entry");
     __shared__ int leading_good[kThreads / 32];   // per warp: how many of its 32 codes, from the first on, have class 3
+    __shared__ uint32_t class_sig[8];             // significand bits of fl((1 + m / 8) * g)
+    __shared__ __align__(8) uint8_t cand_ok[8][3][8];   // [m][candidate][j]: midpoint j agrees ([..][7] = 1)
     const int c = threadIdx.x;
+    const bool check = BF16_IN && (__float_as_uint(g) & 0x007FFFFFu) != 0u;   // a power of two keeps every scale short
+    if (check) {                                  // CTA-uniform
+        if (c < 8 * 21) {
+            const int m = c / 21, r = c - 21 * m, cand = r / 7, j = r - 7 * cand;
+            const float gn = __uint_as_float((__float_as_uint(g) & 0x007FFFFFu) | 0x3F800000u);
+            const float Dr = __fmul_rn(1.0f + 0.125f * (float)m, gn);
+            const float Rc = __uint_as_float(__float_as_uint(__frcp_rn(Dr)) + (cand == 0 ? 0u : (cand == 1 ? 1u : 0xFFFFFFFFu)));
+            const float M = (j < 4) ? 0.25f + 0.5f * (float)j : (j == 4 ? 2.5f : (j == 5 ? 3.5f : 5.0f));
+            cand_ok[m][cand][j] = one_multiply_codes_agree_at(Dr, Rc, M) ? 1 : 0;
+            if (j == 0) cand_ok[m][cand][7] = 1;
+            if (r == 0) class_sig[m] = __float_as_uint(Dr) & 0x007FFFFFu;
+        }
+        __syncthreads();
+    }
     float D = __uint_as_float(0x7FC00000u), R = 0.0f, w = 0.0f;
-    uint32_t h16 = 0;
+    uint32_t z = 0;
+    bool vote = true;
     if (c < num_codes(FMT)) {
-        D = __fmul_rn(scale_value(FMT, c), g);
+        const float S = scale_value(FMT, c);
+        D = __fmul_rn(S, g);
         const bool in_range = (D >= kFastMin && D <= kFastMax);
         if (in_range || D == 0.0f) {
             if (in_range) R = __frcp_rn(D);
-            const __half hD = __float2half_rn(-D);
-            h16 = (uint32_t)__half_as_ushort(hD);
-            w = (__half2float(hD) == -D) ? 2.0f : 1.0f;
-            if (w == 2.0f && (__float_as_uint(D) & 0x000FFFFFu) == 0u) w = 3.0f;
+            if (check) {
+                w = 1.0f;
+                if (in_range) {
+                    const int m = (__float_as_uint(S) >> 20) & 7;
+                    constexpr unsigned long long kAll = 0x0101010101010101ull;
+                    const unsigned long long* ok = reinterpret_cast<const unsigned long long*>(cand_ok[m]);
+                    const int cand = ok[0] == kAll ? 0 : (ok[1] == kAll ? 1 : (ok[2] == kAll ? 2 : 3));
+                    vote = cand < 3 && (__float_as_uint(D) & 0x007FFFFFu) == class_sig[m];
+                    z = __float_as_uint(R) + (cand == 1 ? 1u : (cand == 2 ? 0xFFFFFFFFu : 0u));
+                }
+            } else {
+                const __half hD = __float2half_rn(-D);
+                z = (uint32_t)__half_as_ushort(hD);
+                w = (__half2float(hD) == -D) ? 2.0f : 1.0f;
+                if (w == 2.0f && (__float_as_uint(D) & 0x000FFFFFu) == 0u) w = 3.0f;
+            }
         }
     }
-    T.E[c] = make_float4(D, R, __uint_as_float(h16), w);
+    T.E[c] = make_float4(D, R, __uint_as_float(z), w);
     const uint32_t good = __ballot_sync(0xFFFFFFFFu, w == 3.0f);
     if ((c & 31) == 0) leading_good[c >> 5] = (good == 0xFFFFFFFFu) ? 32 : (__ffs(~good) - 1);
-    __syncthreads();
-    int first_bad = 0;
+    const bool all_voted = __syncthreads_and(vote) != 0;
+    int fb = 0;
 #pragma unroll
     for (int wp = 0; wp < kThreads / 32; ++wp) {
-        if (first_bad == 32 * wp) first_bad += leading_good[wp];
+        if (fb == 32 * wp) fb += leading_good[wp];
     }
-    return min(first_bad, num_codes(FMT));
+    first_bad = min(fb, num_codes(FMT));
+    return check && all_voted;
 }
 
 // fl32(v / D) by a reciprocal multiply and ONE residual correction, R = RN(1 / D) correctly rounded,
@@ -253,6 +327,9 @@ __device__ __forceinline__ void pack_and_score(const float* v, const float* t, c
 // truncation returns M itself, which the FP4 rounding then sends to the even neighbour exactly as it
 // does for the true quotient.  Checked on the host for every bf16 value and
 // every significand (tests/test_quotient_hard_cases.py).  The sign of a zero product is that of v.
+// Under a tensor scale that is not a power of two D is long; the same multiply is then used with a
+// reciprocal that build_quant_tables() has checked for the launch's eight scale significands (R is that
+// reciprocal here, taken from the table's z field).
 template <int B, bool SHORT>
 __device__ __forceinline__ void block_quotients(const float* v, float D, float R, float* t) {
     if constexpr (SHORT) {
@@ -284,7 +361,7 @@ __device__ __forceinline__ void encode_group_fast(const float* v, const float4* 
     constexpr int NBG = GE / B;
     float t[GE];
 #pragma unroll
-    for (int j = 0; j < NBG; ++j) block_quotients<B, SHORT>(&v[j * B], E[j].x, E[j].y, &t[j * B]);
+    for (int j = 0; j < NBG; ++j) block_quotients<B, SHORT>(&v[j * B], E[j].x, (SHORT && !HALF) ? E[j].z : E[j].y, &t[j * B]);
     pack_and_score<B, HALF>(v, t, E, packed, sse);
 }
 
@@ -300,8 +377,8 @@ __device__ __forceinline__ void encode_group_fast_dual(const float* v, const flo
     float t6[GE], t4[GE];
 #pragma unroll
     for (int j = 0; j < NBG; ++j) {
-        block_quotients<B, SHORT>(&v[j * B], E6[j].x, E6[j].y, &t6[j * B]);
-        block_quotients<B, SHORT>(&v[j * B], E4[j].x, E4[j].y, &t4[j * B]);
+        block_quotients<B, SHORT>(&v[j * B], E6[j].x, (SHORT && !HALF) ? E6[j].z : E6[j].y, &t6[j * B]);
+        block_quotients<B, SHORT>(&v[j * B], E4[j].x, (SHORT && !HALF) ? E4[j].z : E4[j].y, &t4[j * B]);
     }
     uint32_t h6[GE / 2], h4[GE / 2];
 #pragma unroll
@@ -360,6 +437,7 @@ struct QuantConsts {
     int pow2_rule;      // kPow2Eq1 unless the format is UE8M0 and another rule was asked for
     float u_floor;      // lean path: prevent-zero as a floor on amax / g, 4 * value(code 1), else 0
     int lean_cmax;      // lean path: every code up to this one has class 3 (UE5M3: the codes above it take the general path)
+    bool onemul;        // bf16 input under a tensor scale: the one-multiply quotient with the reciprocals in E[].z holds for the whole table
 };
 
 // The lean path runs when there is no tensor scale and every code of the table has class 3 (UE4M3), or
@@ -474,6 +552,9 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             if (wmin >= (SH ? 3.0f : 2.0f)) {
                 if constexpr (DUAL) encode_group_fast_dual<B, true, SH>(v, E6, E4, pk, pk4, sse, sse4);
                 else encode_group_fast<B, true, SH>(v, E6, pk, sse);
+            } else if (SH && k.onemul) {   // one-multiply quotient with the checked reciprocals, binary32 residual
+                if constexpr (DUAL) encode_group_fast_dual<B, false, SH>(v, E6, E4, pk, pk4, sse, sse4);
+                else encode_group_fast<B, false, SH>(v, E6, pk, sse);
             } else {
                 if constexpr (DUAL) encode_group_fast_dual<B, false, false>(v, E6, E4, pk, pk4, sse, sse4);
                 else encode_group_fast<B, false, false>(v, E6, pk, sse);
@@ -631,6 +712,9 @@ __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const Qu
             if (wmin >= (SH ? 3.0f : 2.0f)) {
                 if constexpr (DUAL) encode_group_fast_dual<SG, true, SH>(v, &E6, &E4, o6, o4, &sse, &sse4);
                 else encode_group_fast<SG, true, SH>(v, &E6, o6, &sse);
+            } else if (SH && k.onemul) {
+                if constexpr (DUAL) encode_group_fast_dual<SG, false, SH>(v, &E6, &E4, o6, o4, &sse, &sse4);
+                else encode_group_fast<SG, false, SH>(v, &E6, o6, &sse);
             } else {
                 if constexpr (DUAL) encode_group_fast_dual<SG, false, false>(v, &E6, &E4, o6, o4, &sse, &sse4);
                 else encode_group_fast<SG, false, false>(v, &E6, o6, &sse);
@@ -755,7 +839,8 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
     }
     QuantConsts k;
     k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    const int first_bad = build_quant_tables<FMT>(T, k.g);   // contains a barrier: row0[] is complete too
+    int first_bad;
+    k.onemul = build_quant_tables<FMT, DT == kBF16>(T, k.g, first_bad);   // contains a barrier: row0[] is complete too
     k.unit_g = (k.g == 1.0f);
     k.c_min = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;
@@ -920,7 +1005,8 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     }
     QuantConsts k;
     k.g = p.d_global_scale ? *p.d_global_scale : p.global_scale;
-    const int first_bad = build_quant_tables<FMT>(T, k.g);
+    int first_bad;
+    k.onemul = build_quant_tables<FMT, DT == kBF16>(T, k.g, first_bad);
     k.unit_g = (k.g == 1.0f);
     k.c_min = (p.prevent_zero && FMT != kUE8M0) ? 1 : 0;
     k.pow2_rule = (FMT == kUE8M0) ? p.pow2_rule : kPow2Eq1;

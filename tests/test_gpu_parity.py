@@ -199,6 +199,127 @@ def test_elements_and_maxima_next_to_rounding_midpoints(fmt, g):
     check_parity(x[: 64 * B], B, fmt, mxq.MXQ_BRUTE, g)
 
 
+def _to_bf16_floor(p64):
+    """Largest bf16 value not above the positive binary64 number p64, as float32."""
+    f = np.float32(p64)
+    if np.float64(f) > p64:
+        f = np.nextafter(f, np.float32(0), dtype=np.float32)
+    return (np.array([f], dtype=np.float32).view(np.uint32) & np.uint32(0xFFFF0000)).view(np.float32)[0]
+
+
+def _bf16_step(v, k):
+    """The bf16 value k steps above (k < 0: below) the bf16 value v."""
+    return (np.array([v], dtype=np.float32).view(np.uint32).astype(np.int64) + (k << 16)).astype(np.uint32).view(np.float32)[0]
+
+
+def _one_multiply_code_differs(v, D):
+    """True if rounding RZ(v * RN(1 / D)) to the FP4 grid gives another magnitude than rounding fl32(v / D)
+    (a single multiply by the reciprocal, rounded toward zero, against the correctly rounded quotient)."""
+    R = np.float32(np.float32(1) / D)
+    p = np.float64(v) * np.float64(R)                 # exact: 8 x 24 significant bits
+    h = np.float32(p)
+    if np.float64(h) > p:
+        h = np.nextafter(h, np.float32(0), dtype=np.float32)
+    f = np.float32(v / D)
+    return orc.e2m1_index(float(h)) != orc.e2m1_index(float(f))
+
+
+def test_bf16_elements_next_to_midpoints_of_long_decode_scales():
+    """bf16 input under tensor scales g chosen so that, for the decode scale D = fl(1.0 * g) of code 0x38,
+    M * D lies within a few 2^-24 of a bf16 value for one FP4 midpoint M: there a single multiply by 1 / D
+    can round to the other side of M although bf16 values are 2^-8 apart.  Each block holds a maximum
+    that selects code 0x38 and, for all seven midpoints, the bf16 values just below and above M * D.  The
+    test first shows (on the host) that for several of these scales the one-multiply quotient is wrong
+    for an element of the block, so a kernel that took that shortcut unchecked fails here."""
+    B, fmt = 16, mxq.MXQ_SF_UE4M3
+    mids = [0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0]
+    rng = np.random.default_rng(77)
+    wrong_somewhere = 0
+    cases = []
+    for _ in range(400):
+        vb = _bf16_step(np.float32(2.0 ** int(rng.integers(-12, 3))), int(rng.integers(0, 128)))
+        m = mids[int(rng.integers(0, 7))]
+        D = np.float32(np.float64(vb) / m)
+        for _k in range(int(rng.integers(0, 4))):
+            D = np.nextafter(D, np.float32(np.inf if rng.integers(0, 2) else 0), dtype=np.float32)
+        g = D                                          # code 0x38 has scale value 1.0: D = fl(1.0 * g) = g
+        near = []
+        for mm in mids:
+            v0 = _to_bf16_floor(np.float64(mm) * np.float64(D))
+            near += [v0, _bf16_step(v0, 1)]
+        a = None                                       # a bf16 maximum above every other element that selects code 0x38
+        for cand in (_to_bf16_floor(6.0 * np.float64(D)), _bf16_step(_to_bf16_floor(6.0 * np.float64(D)), 1),
+                     _bf16_step(_to_bf16_floor(6.0 * np.float64(D)), -1)):
+            head = np.zeros(B, dtype=np.float32)
+            head[0] = cand
+            if cand > max(near) and orc.quantize(head, B, fmt, orc.ABSMAX, float(g))[1][0] == 0x38:
+                a = cand
+                break
+        if a is None:
+            continue
+        wrong = any(_one_multiply_code_differs(v, D) for v in near)
+        wrong_somewhere += int(wrong)
+        if wrong or len(cases) < 12:
+            blk = np.zeros(B, dtype=np.float32)
+            blk[0] = a
+            blk[1:15] = near
+            blk[2::2] *= -1
+            cases.append((float(g), blk))
+        if wrong_somewhere >= 12 and len(cases) >= 24:
+            break
+    assert wrong_somewhere >= 5, "the generator no longer produces scales that defeat the one-multiply quotient"
+    filler = inputs.normal(64 * B, 3, 1.0, torch.float32).numpy()
+    for g, blk in cases:
+        x = torch.from_numpy(np.concatenate([blk, filler * np.float32(g), blk[::-1].copy()])).to(torch.bfloat16)
+        for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_4O6_PZ):
+            check_parity(x, B, fmt, recipe, g, device_g=True)
+    # the same blocks walked as parts of longer blocks and as small ones
+    g, blk = cases[0]
+    x = torch.from_numpy(np.concatenate([blk] * 8 + [filler * np.float32(g)])).to(torch.bfloat16)
+    for Bx in (4, 8, 32, 64):
+        check_parity(x, Bx, fmt, mxq.MXQ_4O6, g)
+        check_parity(x, Bx, mxq.MXQ_SF_UE5M3, mxq.MXQ_ABSMAX, g)
+
+
+def test_bf16_under_the_tensor_scale_of_every_bf16_amax_significand():
+    """Hierarchical scaling of a bf16 tensor: g = amax / 2688 with amax a bf16 value.  Quotients v / D are
+    then ratios of small integers and hit FP4 rounding midpoints exactly in real arithmetic, for every
+    amax, while the binary32 g and D carry rounding errors: the inputs on which a reciprocal multiply is
+    most likely to round to the wrong side.  One launch per amax significand (128 of them), the tensor
+    scale taken on the device from the tensor itself, data drawn as bf16 values over four binades below
+    the maximum so that every (significand, midpoint) meeting occurs thousands of times."""
+    B, n = 16, 64 * 1024
+    gen = torch.Generator().manual_seed(2688)
+    for s in range(128, 256):
+        amax = np.float32(s / 128.0 * 2.0 ** ((s % 7) - 3))
+        sig = torch.randint(128, 256, (n,), generator=gen).float() / 128.0
+        ex = torch.randint(-6, 0, (n,), generator=gen).float()
+        sign = torch.randint(0, 2, (n,), generator=gen).float() * 2 - 1
+        x = (sig * torch.exp2(ex) * sign * float(amax)).to(torch.bfloat16)
+        x[int(s) * 17] = float(amax)
+        xg = x.cuda()
+        a = torch.empty(1, dtype=torch.float32, device="cuda")
+        dg = torch.empty(1, dtype=torch.float32, device="cuda")
+        mxq.mxq_tensor_amax(xg, n, a, dg)
+        g = float(dg.cpu()[0])
+        assert float(a.cpu()[0]) == float(amax) and g == float(orc.global_scale_from_amax(amax))
+        fmt = mxq.MXQ_SF_UE4M3 if s % 2 == 0 else mxq.MXQ_SF_UE5M3
+        check_parity(x, B, fmt, mxq.MXQ_4O6 if s % 4 < 2 else mxq.MXQ_ABSMAX, g, device_g=True)
+
+
+@pytest.mark.parametrize("B", [4, 16, 32])
+def test_bf16_under_many_tensor_scales(B):
+    """The per-launch check of the decode-scale table runs for every tensor scale that is not a power of
+    two: many scales, both FP8 formats, bf16 data at the magnitudes the scales imply."""
+    rng = np.random.default_rng(5 + B)
+    base = _mixed(4 * 256 * max(B, 8) + 3 * 64, 90 + B, torch.float32)
+    for i in range(24):
+        g = float(np.float32(np.exp(rng.uniform(np.log(1e-6), np.log(30.0)))))
+        x = (base * np.float32(g * 300.0)).to(torch.bfloat16)
+        fmt = mxq.MXQ_SF_UE4M3 if i % 2 == 0 else mxq.MXQ_SF_UE5M3
+        check_parity(x, B, fmt, mxq.MXQ_4O6 if i % 3 else mxq.MXQ_ABSMAX_PZ, g, device_g=bool(i % 2))
+
+
 def test_device_resident_global_scale_matches_host_scale():
     x = _mixed(8192, 5, torch.bfloat16)
     for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_4O6, mxq.MXQ_BRUTE):
