@@ -448,6 +448,16 @@ __device__ __forceinline__ bool lean_allowed(int first_bad, bool unit_g) {
     return unit_g && first_bad >= (FMT == kUE5M3 ? num_codes(FMT) - 16 : num_codes(FMT));
 }
 
+// The lean path under a tensor scale (LEAN == 2; bf16 input, FP8 scale formats): the launch's table passed
+// the one-multiply check and g lies in [2^-40, 2^20].  Then every decode scale of both formats is within
+// [2^-60, 2^60] (or zero), so every entry carries a checked reciprocal; a block maximum above m_hi may be
+// clamped to it (m_hi / g is at least 2^40: the scale code is the top one either way); a maximum below
+// 2^-63, where the quotient by g is no longer exact, gives a / g < 2^-23 and code 0 (or the prevent-zero
+// floor) whatever its last bits are.
+__device__ __forceinline__ bool lean_scaled_allowed(const QuantConsts& k) {
+    return k.onemul && k.g >= 9.094947017729282379e-13f /* 2^-40 */ && k.g <= 1048576.0f;
+}
+
 // Both 4-over-6 scale codes of a block from one conversion (UE4M3): the code for w6 in bits 0..7,
 // the code for w4 in bits 8..15.
 __device__ __forceinline__ uint32_t round_scale_pair_ue4m3(float w4, float w6) {
@@ -466,7 +476,9 @@ __device__ __forceinline__ int target6_code(float u, int pow2_rule) {
     return round_scale<FMT>(EXACT ? __fdiv_rn(u, 6.0f) : div6_fast(u));
 }
 
-// LEAN (launch-uniform; bf16 input, FP8 scale format, no tensor scale, every decode scale of the
+// LEAN == 2: the same loop under a tensor scale, see lean_scaled_allowed(): the block maximum is divided by g
+// first (corrected quotient), the residual is formed in binary32.
+// LEAN == 1 (launch-uniform; bf16 input, FP8 scale format, no tensor scale, every decode scale of the
 // table of class 3 -- for UE5M3 all but its last few codes, whose scales from 2^16 on are not f16
 // values: a group whose code lands there is redone on the general path): nothing of a block can leave
 // the shortcuts, so the per-block class and range tests and the tensor-scale quotient are left out.  Why no magnitude test is
@@ -477,7 +489,7 @@ __device__ __forceinline__ int target6_code(float u, int pow2_rule) {
 // above it both formats saturate.  Prevent-zero is a floor on the block maximum: for both
 // formats max(code_M(u), 1) = code_M(max(u, 4 eps)) for M = 6 and M = 4, eps = value(code 1)
 // (4 eps / 6 and 4 eps / 4 round to code 1; anything below rounds to 0 or 1, anything above to >= 1).
-template <int DT, int B, int FMT, bool DUAL, bool FAKE, bool LEAN>
+template <int DT, int B, int FMT, bool DUAL, bool FAKE, int LEAN>
 __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTables& T, const QuantConsts& k,
                                                size_t chunk, const uint32_t* raw, double& sse_sum) {
     static_assert(!LEAN || (DT == kBF16 && FMT != kUE8M0), "lean path: bf16 input, FP8 scale formats");
@@ -504,7 +516,9 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
             for (int i = 0; i < B; ++i) a = fmaxf(a, fabsf(v[j * B + i]));
             if constexpr (LEAN) {
                 m[j] = a;
-                const float uf = fmaxf(a, k.u_floor);
+                float ua = a;
+                if constexpr (LEAN == 2) ua = quotient_corrected(fminf(a, k.m_hi), k.g, k.Rg);
+                const float uf = fmaxf(ua, k.u_floor);
                 const float w6 = div6_fast(uf);
                 if constexpr (DUAL && FMT == kUE4M3) {
                     const uint32_t r = round_scale_pair_ue4m3(__fmul_rn(uf, 0.25f), w6);
@@ -535,16 +549,17 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
         float sse[NBG], sse4[NBG];
 #pragma unroll
         for (int j = 0; j < NBG; ++j) sse[j] = sse4[j] = 0.0f;
-        bool lean_group = LEAN;
-        if constexpr (LEAN && FMT == kUE5M3) {   // a code above the class-3 range: this group takes the general path
+        bool lean_group = LEAN != 0;
+        if constexpr (LEAN == 1 && FMT == kUE5M3) {   // a code above the class-3 range: this group takes the general path
             int cmx = 0;
 #pragma unroll
             for (int j = 0; j < NBG; ++j) cmx = max(cmx, DUAL ? max(c6[j], c4[j]) : c6[j]);
             lean_group = cmx <= k.lean_cmax;
         }
         if (LEAN && lean_group) {
-            if constexpr (DUAL) encode_group_fast_dual<B, true, true>(v, E6, E4, pk, pk4, sse, sse4);
-            else encode_group_fast<B, true, true>(v, E6, pk, sse);
+            constexpr bool HALF = (LEAN == 1);   // under a tensor scale the residual is formed in binary32
+            if constexpr (DUAL) encode_group_fast_dual<B, HALF, true>(v, E6, E4, pk, pk4, sse, sse4);
+            else encode_group_fast<B, HALF, true>(v, E6, pk, sse);
         } else if (!LEAN && wmin >= 1.0f && mmax <= k.m_hi && mmin >= k.m_lo) {
             // one decision for both candidates.  bf16 input: the one-multiply quotient with the f16
             // residual when every decode scale of the group is short, else the general shortcuts.
@@ -914,7 +929,7 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
     int cur_t = -1;
     double unused_sum = 0.0;
     auto row_loop = [&](auto lean_tag) {
-        constexpr bool LEAN = decltype(lean_tag)::value;
+        constexpr int LEAN = decltype(lean_tag)::value;
         int slot = 0, fill = DIST % S::SLOTS;
         for (; row < total_rows; row += row_stride) {
             asm volatile("cp.async.wait_group %0;" ::"n"(DIST - 1) : "memory");
@@ -948,10 +963,11 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
     };
     constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
     if constexpr (CAN_LEAN) {
-        if (lean_allowed<FMT>(first_bad, k.unit_g)) row_loop(std::true_type{});
-        else row_loop(std::false_type{});
+        if (lean_allowed<FMT>(first_bad, k.unit_g)) row_loop(std::integral_constant<int, 1>{});
+        else if (lean_scaled_allowed(k)) row_loop(std::integral_constant<int, 2>{});
+        else row_loop(std::integral_constant<int, 0>{});
     } else {
-        row_loop(std::false_type{});
+        row_loop(std::integral_constant<int, 0>{});
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
@@ -1040,7 +1056,7 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     // The chunk loop, instantiated with and without the lean per-block path (see quantize_chunk);
     // which one runs is the same for every thread of the launch.
     auto chunk_loop = [&](auto lean_tag) {
-        constexpr bool LEAN = decltype(lean_tag)::value;
+        constexpr int LEAN = decltype(lean_tag)::value;
         int slot = 0;                      // slot holding `chunk`
         int fill = DIST % S::SLOTS;        // slot that the next request goes to
         size_t ahead = (S::COOP ? wchunk0 : chunk) + (size_t)DIST * stride;
@@ -1078,10 +1094,11 @@ __global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
     constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
     if (has_work) {
         if constexpr (CAN_LEAN) {
-            if (lean_allowed<FMT>(first_bad, k.unit_g)) chunk_loop(std::true_type{});
-            else chunk_loop(std::false_type{});
+            if (lean_allowed<FMT>(first_bad, k.unit_g)) chunk_loop(std::integral_constant<int, 1>{});
+            else if (lean_scaled_allowed(k)) chunk_loop(std::integral_constant<int, 2>{});
+            else chunk_loop(std::integral_constant<int, 0>{});
         } else {
-            chunk_loop(std::false_type{});
+            chunk_loop(std::integral_constant<int, 0>{});
         }
     }
     if constexpr (!FAKE) {

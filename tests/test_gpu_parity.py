@@ -307,6 +307,30 @@ def test_bf16_under_the_tensor_scale_of_every_bf16_amax_significand():
         check_parity(x, B, fmt, mxq.MXQ_4O6 if s % 4 < 2 else mxq.MXQ_ABSMAX, g, device_g=True)
 
 
+@pytest.mark.parametrize("g", [1.3 * 2.0 ** -40, 0.0131, 1.7 * 2.0 ** 19, 1.1 * 2.0 ** -41, 1.2 * 2.0 ** 20])
+def test_bf16_block_maxima_over_the_whole_exponent_range_under_tensor_scales(g):
+    """bf16 blocks whose maxima run through the binades from the bf16 denormals up to 2^60 under
+    tensor scales at and just outside the range for which the kernels use their lean loop: maxima far above
+    the saturation point of the scale format, maxima so small that the quotient by g underflows, zero
+    blocks, and everything in between, for both FP8 formats and every one-pass recipe."""
+    B = 8
+    gen = torch.Generator().manual_seed(41)
+    blocks = []
+    for e in range(-133, 61):                      # block SSEs stay finite in binary32
+        blk = (torch.rand(4, B, generator=gen) * 2 - 1) * 2.0 ** e
+        blk[:, e % B] = 2.0 ** e * (1.0 + (e % 7) / 8.0)
+        blocks.append(blk.reshape(-1))
+    blocks.append(torch.zeros(4 * B))
+    x = torch.cat(blocks).to(torch.bfloat16)
+    x = torch.cat([x, x.flip(0)])
+    for fmt in (mxq.MXQ_SF_UE4M3, mxq.MXQ_SF_UE5M3):
+        for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_ABSMAX_PZ, mxq.MXQ_4O6, mxq.MXQ_4O6_PZ):
+            check_parity(x, B, fmt, recipe, g)
+    check_parity(x, 16, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6_PZ, g, device_g=True)
+    check_parity(x, 32, mxq.MXQ_SF_UE5M3, mxq.MXQ_4O6, g)
+    check_parity(x, 2, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6_PZ, g)
+
+
 @pytest.mark.parametrize("B", [4, 16, 32])
 def test_bf16_under_many_tensor_scales(B):
     """The per-launch check of the decode-scale table runs for every tensor scale that is not a power of
