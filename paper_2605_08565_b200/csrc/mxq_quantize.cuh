@@ -664,6 +664,13 @@ __device__ __forceinline__ int ring_index(int k, int lane) {
     return k * kThreads + (COOP ? (lane ^ k) : lane);
 }
 
+// Larger magnitude of two bf16 pairs, half by half (the sign bits of the result carry no meaning).
+__device__ __forceinline__ uint32_t absmax_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
 // Blocks of 32 and 64 elements (chunk = one block).  The block is walked twice in parts of 16
 // elements read from the thread's ring slot, which stays valid until the next trip's request:
 // once for the block maximum, once for the encode with the SSE chains carried from part to part.
@@ -687,12 +694,26 @@ __device__ __forceinline__ void quantize_long_block(const QuantArgs& p, const Qu
     };
 
     float a = 0.0f;
+    if constexpr (DT == kBF16) {
+        // the maximum pass on the packed words: magnitudes of bf16 values order like the values, and one
+        // max.xorsign.abs.bf16x2 takes the larger magnitude in either half (the sign it leaves is dropped below)
+        uint32_t m0 = 0, m1 = 0;
 #pragma unroll
-    for (int sg = 0; sg < NSG; ++sg) {
-        float v[SG];
-        load_part(sg, v);
+        for (int q = 0; q < S::PIECES; ++q) {
+            const uint4 x = slot_warp[ring_index<S::COOP>(q, lane)];
+            m0 = absmax_bf16x2(absmax_bf16x2(m0, x.x), x.z);
+            m1 = absmax_bf16x2(absmax_bf16x2(m1, x.y), x.w);
+        }
+        const uint32_t mm = absmax_bf16x2(m0, m1) & 0x7FFF7FFFu;
+        a = fmaxf(__uint_as_float(mm << 16), __uint_as_float(mm & 0xFFFF0000u));
+    } else {
 #pragma unroll
-        for (int i = 0; i < SG; ++i) a = fmaxf(a, fabsf(v[i]));
+        for (int sg = 0; sg < NSG; ++sg) {
+            float v[SG];
+            load_part(sg, v);
+#pragma unroll
+            for (int i = 0; i < SG; ++i) a = fmaxf(a, fabsf(v[i]));
+        }
     }
     float u = k.unit_g ? a : quotient_corrected(a, k.g, k.Rg);
     int c6 = max(target6_code<FMT, false>(u, k.pow2_rule), k.c_min), c4 = 0;
@@ -978,8 +999,13 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
 // forms in shared memory; a warp walks rows first, first + 8 * gridDim.x, ... and moves its tensor
 // cursor forward when a row passes the end of the current tensor.  Everything else (ring, staging,
 // per-chunk arithmetic) is as in the single-tensor kernel.
+// Resident CTAs the register allocation has to allow.  The multi-tensor instantiations carry a cursor and
+// a row loop on top of the chunk arithmetic; without a bound some of them (B = 16) land a few registers
+// above the 85 that three CTAs per SM allow and lose a third of their loads in flight.
+__host__ __device__ constexpr int quantize_min_ctas(int B, bool batch) { return (batch && B >= 4 && B <= 16) ? 3 : 1; }
+
 template <int DT, int B, int FMT, bool DUAL, bool FAKE, bool BATCH = false>
-__global__ void __launch_bounds__(kThreads) k_quantize(QuantArgs p) {
+__global__ void __launch_bounds__(kThreads, quantize_min_ctas(B, BATCH)) k_quantize(QuantArgs p) {
     using S = QuantShape<DT, B>;
     static_assert(S::C == quantize_chunk_elems(DT, B), "host and kernel agree on the chunk size");
     extern __shared__ uint4 ring[];
