@@ -855,8 +855,10 @@ class _InputDigest:
 
 def run_configs(configs, hash_inputs=False):
     """Times every (configuration, block size, scale format, recipe) of the five benchmark configurations
-    at full size: the quantize pass with CUDA events as it is called from Python (launches back to back;
-    tensors larger than L2 or rotated so that inputs come from HBM), the tensor MSE afterwards."""
+    at full size with CUDA events: the quantize launches of a row back to back (tensors larger than L2 or
+    rotated so that inputs come from HBM), replayed from a CUDA graph where a launch lasts microseconds
+    (the one-pass recipes) and called from Python where it lasts milliseconds (brute force); the tensor MSE
+    afterwards, untimed."""
     import torch
     from paper_2605_08565_b200 import binding as mxq
     from paper_2605_08565_b200 import inputs

@@ -837,6 +837,10 @@ __device__ __forceinline__ void stage_chunk(uint32_t slot_addr, const void* src,
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
+// Blocks longer than 16 elements go part by part (quantize_long_block()), except 4-over-6 at B = 32, which
+// is faster with the whole block in registers (33.5 M bf16 elements: 0.775 against 0.711 of the copy bandwidth).
+__host__ __device__ constexpr bool long_block_path(int B, bool dual) { return B > 16 && !(dual && B == 32); }
+
 // Body of the multi-tensor kernel (see k_quantize, BATCH).
 template <int DT, int B, int FMT, bool DUAL>
 __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTables& T, uint4* ring) {
@@ -969,7 +973,7 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
             }
             const size_t chunk = (size_t)(row - cur_c.first) * 32 + lane;
             if (chunk >= cur_c.n_chunks) continue;      // a lane past the end of the tensor's last row
-            if constexpr (B > 16 && !(DUAL && B == 32)) {
+            if constexpr (long_block_path(B, DUAL)) {
                 quantize_long_block<DT, B, FMT, DUAL, false>(pl, T, k, chunk, slot_warp, lane, unused_sum);
             } else {
                 uint32_t raw[S::PIECES * 4];
@@ -982,7 +986,7 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
             }
         }
     };
-    constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
+    constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(long_block_path(B, DUAL));
     if constexpr (CAN_LEAN) {
         if (lean_allowed<FMT>(first_bad, k.unit_g)) row_loop(std::integral_constant<int, 1>{});
         else if (lean_scaled_allowed(k)) row_loop(std::integral_constant<int, 2>{});
@@ -999,10 +1003,12 @@ __device__ __forceinline__ void quantize_batch_body(const QuantArgs& p, QuantTab
 // forms in shared memory; a warp walks rows first, first + 8 * gridDim.x, ... and moves its tensor
 // cursor forward when a row passes the end of the current tensor.  Everything else (ring, staging,
 // per-chunk arithmetic) is as in the single-tensor kernel.
-// Resident CTAs the register allocation has to allow.  The multi-tensor instantiations carry a cursor and
-// a row loop on top of the chunk arithmetic; without a bound some of them (B = 16) land a few registers
-// above the 85 that three CTAs per SM allow and lose a third of their loads in flight.
-__host__ __device__ constexpr int quantize_min_ctas(int B, bool batch) { return (batch && B >= 4 && B <= 16) ? 3 : 1; }
+// Resident CTAs the register allocation has to allow (0: no bound, the allocator's own choice; an explicit 1
+// is NOT the same: it lets the allocator spend up to 255 registers and measured far slower).  The
+// multi-tensor instantiations carry a cursor and a row loop on top of the chunk arithmetic; without a bound
+// some of them (B = 16) land a few registers above the 85 that three CTAs per SM allow and lose a third of
+// their loads in flight.
+__host__ __device__ constexpr int quantize_min_ctas(int B, bool batch) { return (batch && B >= 4 && B <= 16) ? 3 : 0; }
 
 template <int DT, int B, int FMT, bool DUAL, bool FAKE, bool BATCH = false>
 __global__ void __launch_bounds__(kThreads, quantize_min_ctas(B, BATCH)) k_quantize(QuantArgs p) {
@@ -1104,7 +1110,7 @@ __global__ void __launch_bounds__(kThreads, quantize_min_ctas(B, BATCH)) k_quant
             if (S::COOP && chunk >= p.n_items) continue;   // a lane past the end (the warp's last trip)
             // blocks longer than 16 elements go part by part, except 4-over-6 at B = 32, which measured
             // slightly faster with the whole block in registers
-            if constexpr (B > 16 && !(DUAL && B == 32)) {
+            if constexpr (long_block_path(B, DUAL)) {
                 quantize_long_block<DT, B, FMT, DUAL, FAKE>(p, T, k, chunk, slot_warp, lane, sse_sum);
             } else {
                 uint32_t raw[S::PIECES * 4];
@@ -1117,7 +1123,7 @@ __global__ void __launch_bounds__(kThreads, quantize_min_ctas(B, BATCH)) k_quant
             }
         }
     };
-    constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(B > 16 && !(DUAL && B == 32));
+    constexpr bool CAN_LEAN = (DT == kBF16) && (FMT != kUE8M0) && !(long_block_path(B, DUAL));
     if (has_work) {
         if constexpr (CAN_LEAN) {
             if (lean_allowed<FMT>(first_bad, k.unit_g)) chunk_loop(std::integral_constant<int, 1>{});

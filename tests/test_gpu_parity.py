@@ -432,6 +432,25 @@ def test_tensor_amax(dtype):
         mxq.mxq_tensor_amax(xg, n, out)
         torch.cuda.synchronize()
         assert float(out.cpu()[0]) == float(orc.tensor_amax(inputs.to_numpy_bits(x)))
+    # with the tensor scale: the last CTA to finish writes it, whatever the grid size (one CTA to the
+    # full persistent grid), and buffers that held something else before are overwritten
+    for n in (5, 4096, 1024 * 1024 + 16, 24 * 1024 * 1024 + 5):
+        x = (inputs.normal(n, 7 + n, 3.0, torch.float32) * (1.0 + (n % 5))).clamp(-50.0, 50.0).to(dtype).contiguous()
+        x[n // 3] = -77.5
+        xg = x.cuda()
+        out = torch.full((1,), 1.0e30, dtype=torch.float32, device="cuda")
+        dg = torch.full((1,), -3.0, dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            mxq.mxq_tensor_amax(xg, n, out, dg)
+        torch.cuda.synchronize()
+        want = orc.tensor_amax(inputs.to_numpy_bits(x))
+        assert float(out.cpu()[0]) == float(want) == 77.5
+        assert float(dg.cpu()[0]) == float(orc.global_scale_from_amax(want))
+    z = torch.zeros(4096, dtype=dtype, device="cuda")
+    out = torch.full((1,), 5.0, dtype=torch.float32, device="cuda")
+    dg = torch.full((1,), 5.0, dtype=torch.float32, device="cuda")
+    mxq.mxq_tensor_amax(z, 4096, out, dg)
+    assert float(out.cpu()[0]) == 0.0 and float(dg.cpu()[0]) == 1.0      # an all-zero tensor: scale 1
 
 
 def test_tensor_mse_is_deterministic_and_accurate():
