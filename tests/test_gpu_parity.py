@@ -344,6 +344,39 @@ def test_bf16_under_many_tensor_scales(B):
         check_parity(x, B, fmt, mxq.MXQ_4O6 if i % 3 else mxq.MXQ_ABSMAX_PZ, g, device_g=bool(i % 2))
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B", [2, 16, 32])
+def test_non_finite_elements_stay_inside_their_own_blocks(dtype, B, sweep_mode):
+    """NaN and infinite elements are outside the contract: the outputs of a block that holds one are
+    unspecified.  What the library does promise is that nothing else suffers: the call returns normally,
+    every block WITHOUT such an element still comes out bit for bit as the oracle has it (the oracle sees a
+    copy with the offending blocks zeroed), and the next call on the same context is exact again."""
+    n = 2 * 256 * 64 + 7 * 64
+    x = _mixed(n, 400 + B, torch.float32)
+    x = torch.nan_to_num(x, nan=0.0, posinf=0.0, neginf=0.0)
+    gen = torch.Generator().manual_seed(9 + B)
+    where = torch.randperm(n, generator=gen)[:60]
+    x[where[:20]] = float("nan")
+    x[where[20:40]] = float("inf")
+    x[where[40:]] = float("-inf")
+    x = x.to(dtype)
+    bad_block = (~torch.isfinite(x.float())).reshape(-1, B).any(dim=1).numpy()
+    clean = x.clone().reshape(-1, B)
+    clean[torch.from_numpy(bad_block)] = 0
+    clean = clean.reshape(-1).contiguous()
+    good = ~bad_block
+    for fmt in FMTS:
+        for recipe in (mxq.MXQ_ABSMAX_PZ, mxq.MXQ_4O6, mxq.MXQ_BRUTE):
+            if recipe == mxq.MXQ_BRUTE and fmt == mxq.MXQ_SF_UE5M3 and B == 32:
+                continue                                  # the same kernels as UE4M3; keeps the oracle time down
+            gc, gs, ge, _ = gpu_quantize(x, B, fmt, recipe, 1.0)
+            oc, os_, oe = orc.quantize(inputs.to_numpy_bits(clean), B, fmt, recipe, 1.0, threads=8)
+            assert np.array_equal(gs[good], os_[good]), (fmt, recipe)
+            assert np.array_equal(gc.reshape(-1, B // 2)[good], oc.reshape(-1, B // 2)[good]), (fmt, recipe)
+            assert np.array_equal(ge.view(np.uint32)[good], oe.view(np.uint32)[good]), (fmt, recipe)
+    check_parity(clean, B, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6_PZ, 1.0)
+
+
 def test_device_resident_global_scale_matches_host_scale():
     x = _mixed(8192, 5, torch.bfloat16)
     for recipe in (mxq.MXQ_ABSMAX, mxq.MXQ_4O6, mxq.MXQ_BRUTE):
