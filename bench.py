@@ -437,7 +437,7 @@ def streaming_rooflines(torch, mxq, device, peaks):
     out = {}
     n = STREAM_ELEMS
     prof = {("bf16", ABSMAX): "k_quantize_absmax_bf16_B16_128Mi.txt", ("bf16", R4O6): "k_quantize_4o6_bf16_B16_128Mi.txt",
-            ("f32", ABSMAX): "k_quantize_absmax_f32_B16_128Mi.txt"}
+            ("f32", ABSMAX): "k_quantize_absmax_f32_B16_128Mi.txt", ("f32", R4O6): "k_quantize_4o6_f32_B16_128Mi.txt"}
     for name, dt, recipe, B in (
             ("absmax_bf16_B16", torch.bfloat16, ABSMAX, 16), ("4o6_bf16_B16", torch.bfloat16, R4O6, 16),
             ("absmax_f32_B16", torch.float32, ABSMAX, 16), ("4o6_f32_B16", torch.float32, R4O6, 16),
