@@ -466,6 +466,23 @@ __device__ __forceinline__ uint32_t round_scale_pair_ue4m3(float w4, float w6) {
     return r;
 }
 
+// The same for UE5M3, whose values are the UE4M3 values times 2^-8 (codes 0..0x7E), times 1 (the UE4M3
+// normals, codes + 0x40) and times 2^8 (codes + 0x80): rounding to nearest even commutes with an exact
+// scaling by a power of two, so the pair is scaled into the stretch of UE4M3 that matches its magnitude,
+// converted, and the code offset added to both bytes.  The stretch is chosen by w4; w6 must lie within
+// [w4 / 2, w4] (it is w4 / 1.5 here), which keeps it among the UE4M3 normals wherever w4 is: w4 < 1 uses
+// the whole of UE4M3 including its subnormals (256 w <= 448: no saturation), 1 <= w4 < 256 the normals
+// from 0.5 up, w4 >= 256 the same after a division by 256, where saturation at 448 is the saturation of
+// UE5M3 at 114688.  Either stretch gives the same code where two of them overlap.
+__device__ __forceinline__ uint32_t round_scale_pair_ue5m3(float w4, float w6) {
+    const bool low = w4 < 1.0f, high = w4 >= 256.0f;
+    const float s = low ? 256.0f : (high ? 0.00390625f : 1.0f);
+    const uint32_t offset = low ? 0u : (high ? 0x8080u : 0x4040u);
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(__fmul_rn(w4, s)), "f"(__fmul_rn(w6, s)));
+    return (uint32_t)r + offset;
+}
+
 // Scale code for the M = 6 target from u = amax / g: Eq. 2 (Eq. 1 for UE8M0), or one of the
 // alternative power-of-two rules.
 template <int FMT, bool EXACT>
@@ -520,7 +537,11 @@ __device__ __forceinline__ void quantize_chunk(const QuantArgs& p, const QuantTa
                 if constexpr (LEAN == 2) ua = quotient_corrected(fminf(a, k.m_hi), k.g, k.Rg);
                 const float uf = fmaxf(ua, k.u_floor);
                 const float w6 = div6_fast(uf);
-                if constexpr (DUAL && FMT == kUE4M3) {
+                if constexpr (DUAL && FMT == kUE5M3) {
+                    const uint32_t r = round_scale_pair_ue5m3(__fmul_rn(uf, 0.25f), w6);
+                    c6[j] = (int)(r & 0xFFu);
+                    c4[j] = (int)(r >> 8);
+                } else if constexpr (DUAL && FMT == kUE4M3) {
                     const uint32_t r = round_scale_pair_ue4m3(__fmul_rn(uf, 0.25f), w6);
                     c6[j] = (int)(r & 0xFFu);
                     c4[j] = (int)(r >> 8);

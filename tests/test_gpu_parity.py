@@ -331,6 +331,37 @@ def test_bf16_block_maxima_over_the_whole_exponent_range_under_tensor_scales(g):
     check_parity(x, 2, mxq.MXQ_SF_UE4M3, mxq.MXQ_4O6_PZ, g)
 
 
+@pytest.mark.parametrize("g", [1.0, 0.0131, 0.75])
+def test_bf16_block_maxima_next_to_every_ue5m3_scale_midpoint(g):
+    """4-over-6 on bf16 with UE5M3 scales: block maxima placed at the bf16 values around M * g * (midpoint of
+    two neighbouring scale values) for every pair of neighbouring codes and both targets M = 4 and 6, i.e.
+    where the rounding of either candidate's scale is decided, across the whole code range (the kernels
+    round both candidates with one UE4M3 conversion of a scaled pair; see the oracle-side test of that
+    identity).  UE4M3 runs on the same data for comparison."""
+    B = 8
+    blocks = []
+    for fmt in (mxq.MXQ_SF_UE5M3,):
+        for c in range(0, orc.num_codes(fmt) - 1):
+            mid = (orc.scale_value(fmt, c) + orc.scale_value(fmt, c + 1)) / 2
+            for M in (4.0, 6.0):
+                a0 = _to_bf16_floor(np.float64(mid) * M * g)
+                if not (0 < a0 < 1e30):
+                    continue
+                for k in (-1, 0, 1, 2):
+                    a = _bf16_step(a0, k)
+                    blk = np.zeros(B, dtype=np.float32)
+                    blk[(c + k) % B] = a if c % 2 else -a
+                    blk[(c + k + 3) % B] = a * np.float32(0.4375)
+                    blocks.append(blk)
+    x = torch.from_numpy(np.concatenate(blocks)).to(torch.bfloat16)
+    for fmt in (mxq.MXQ_SF_UE5M3, mxq.MXQ_SF_UE4M3):
+        for recipe in (mxq.MXQ_4O6, mxq.MXQ_4O6_PZ, mxq.MXQ_ABSMAX):
+            check_parity(x, B, fmt, recipe, g)
+    check_parity(x, 16, mxq.MXQ_SF_UE5M3, mxq.MXQ_4O6, g, device_g=True)
+    check_parity(x, 2, mxq.MXQ_SF_UE5M3, mxq.MXQ_4O6_PZ, g)
+    check_parity(x, 32, mxq.MXQ_SF_UE5M3, mxq.MXQ_4O6, g)
+
+
 @pytest.mark.parametrize("B", [4, 16, 32])
 def test_bf16_under_many_tensor_scales(B):
     """The per-launch check of the decode-scale table runs for every tensor scale that is not a power of

@@ -134,3 +134,38 @@ def test_mx_scale_is_largest_power_with_6S_le_amax():
     assert orc.round_scale(orc.UE8M0, 2.0 ** 127) == 254
     assert orc.round_scale(orc.UE8M0, np.nextafter(f32(1.0), f32(0))) == 126
     assert orc.round_scale(orc.UE8M0, 1.0) == 127
+
+
+def test_ue5m3_rounding_equals_a_scaled_ue4m3_rounding():
+    """The UE5M3 value set is the UE4M3 value set times 2^-8 (codes 0..0x7E), the UE4M3 normals themselves
+    (codes + 0x40) and the UE4M3 normals times 2^8 (codes + 0x80), so rounding onto UE5M3 is rounding a
+    scaled number onto UE4M3 plus a code offset: below 1 scale by 256, from 1 to 256 by 1, above by 1/256,
+    with saturation at 448 standing for saturation at 114688.  The lean kernels round both 4-over-6 targets
+    this way with one hardware E4M3 conversion, choosing the stretch by the larger target.  Checked against
+    the oracle's UE5M3 rounding on every mantissa pattern near the stretch boundaries, on a sample of all
+    other binades, and for the smaller target w / 1.5 rounded in the stretch that w selects."""
+    import ml_dtypes
+
+    rng = np.random.default_rng(53)
+    ws = [np.float32(0.0)]
+    for e in (-19, -18, -17, -15, -14, -9, -1, 0, 7, 8, 15, 16, 17):          # whole binades, every 64th mantissa
+        ws += list((np.arange(0, 1 << 23, 64, dtype=np.uint32) | np.uint32((e + 127) << 23)).view(np.float32))
+    for e in range(-30, 30):
+        ws += list((rng.integers(0, 1 << 23, 600).astype(np.uint32) | np.uint32((e + 127) << 23)).view(np.float32))
+    for c in range(0, 254):                                                   # the midpoints between codes, and their neighbours
+        mid = np.float32((orc.scale_value(orc.UE5M3, c) + orc.scale_value(orc.UE5M3, c + 1)) / 2)
+        ws += [mid, np.nextafter(mid, np.float32(0)), np.nextafter(mid, np.float32(np.inf))]
+    ws = np.array(ws, dtype=np.float32)
+
+    def via_e4m3(w, chooser):
+        low, high = chooser < 1.0, chooser >= 256.0
+        s = np.where(low, 256.0, np.where(high, 1.0 / 256.0, 1.0)).astype(np.float32)
+        off = np.where(low, 0, np.where(high, 0x80, 0x40))
+        t = np.minimum((w * s).astype(np.float32), np.float32(448.0))         # the conversion saturates
+        return t.astype(ml_dtypes.float8_e4m3fn).view(np.uint8).astype(np.int64) + off
+
+    want = np.array([orc.round_scale(orc.UE5M3, float(w)) for w in ws])
+    assert np.array_equal(via_e4m3(ws, ws), want)
+    w6 = (ws / np.float32(1.5)).astype(np.float32)
+    want6 = np.array([orc.round_scale(orc.UE5M3, float(w)) for w in w6])
+    assert np.array_equal(via_e4m3(w6, ws), want6)
