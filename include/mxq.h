@@ -307,9 +307,9 @@ int mxq_mask_interval(const void* x, int dtype, size_t n, float lo, float hi, vo
  *     the best SSE found so far, in every block.
  * The bounds are evaluated in the kernel's own binary32 arithmetic and compared strictly, so the
  * outputs (codes, scale bytes, block SSE; ties to the smaller code) are bit-identical to the full
- * sweep; only the time differs, by an amount that depends on the data.  Where the bounds are known
- * not to pay (UE4M3 under a tensor scale with block sizes up to 8) the call runs the full sweep
- * whatever the option says.  The paper states no such shortcut.
+ * sweep; only the time differs, by an amount that depends on the data.  For block sizes up to 16
+ * the kernel first sorts the blocks of each CTA by magnitude (in shared memory), so that a warp holds
+ * blocks of like size and its bounds are tight.  The paper states no such shortcut.
  *
  * mxq_set_option: MXQ_ERR_BAD_ENUM for an unknown option or a value outside {0, 1}.
  * mxq_get_option: MXQ_ERR_NULL for a NULL out_value (host pointer). */

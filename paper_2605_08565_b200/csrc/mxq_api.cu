@@ -79,15 +79,8 @@ static int quantize_common(const void* x, int dtype, size_t n, int block_size, i
     cudaError_t err;
     if (brute) {
         a.n_items = n / (size_t)block_size;
-        // The pruned sweep is a speed option only (same outputs), so where it is known to lose the plain
-        // sweep is launched instead: UE4M3 under a tensor scale with blocks of at most 8 elements.  A
-        // tensor scale derived from the tensor maximum puts every UE4M3 decode scale below amax_t / 6, so
-        // the rule that leaves out all-zero candidates cannot fire unless a warp's largest element is 24
-        // times below the tensor's, and with 128 or more blocks per warp some block defeats the other two
-        // bounds: measured 0.90 to 0.97 of the plain sweep's speed.
-        const bool has_tensor_scale = d_global_scale != nullptr || global_scale != 1.0f;
-        const bool prune_pays = !(scale_fmt == MXQ_SF_UE4M3 && has_tensor_scale && block_size <= 8);
-        if (g_brute_prune.load(std::memory_order_relaxed) && prune_pays)
+        // the pruned sweep is a speed option only: same outputs, bit for bit
+        if (g_brute_prune.load(std::memory_order_relaxed))
             err = (dtype == MXQ_F32) ? launch_brute_pruned_f32(a, block_size, scale_fmt, s)
                                      : launch_brute_pruned_bf16(a, block_size, scale_fmt, s);
         else

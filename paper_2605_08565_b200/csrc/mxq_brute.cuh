@@ -444,6 +444,30 @@ __host__ __device__ constexpr int brute_group_elems(int B) { return B >= 32 ? B 
 
 constexpr int brute_min_ctas(int B, bool prune) { (void)prune; return B <= 32 ? 2 : 1; }
 
+// The pruned sweep sorts the blocks of a CTA's 256 groups by magnitude when a thread holds several blocks.
+__host__ __device__ constexpr bool brute_sorted(int B, bool prune) { return prune && B < 32; }
+
+// Dynamic shared memory of the sorted mode.  The tile holds the CTA's 256 groups as binary32, one padded row
+// per group (so that both a thread's own row and rows gathered at random spread over the banks); once
+// every thread has taken its blocks the same memory receives the results (code bytes, scale bytes, block
+// SSEs, each at the block's original position).  Bins and permutation have memory of their own.
+template <int B>
+struct BruteTile {
+    static constexpr int G = brute_group_elems(B);
+    static constexpr int NBT = G / B;                       // blocks per thread (only used for B < 32)
+    static constexpr int ROW = G + 1;
+    static constexpr int BINS = 1024;                       // exponent and two significand bits of the block maximum
+    static constexpr size_t TILE_BYTES = (size_t)kThreads * ROW * 4;
+    static constexpr size_t OUT_SCALES = (size_t)kThreads * G / 2;            // after the code bytes
+    static constexpr size_t OUT_SSE = OUT_SCALES + (size_t)kThreads * NBT;    // a multiple of 256
+    static constexpr size_t OUT_BYTES = OUT_SSE + (size_t)kThreads * NBT * 4;
+    static constexpr size_t HIST_OFF = (TILE_BYTES + 15) / 16 * 16;
+    static constexpr size_t PERM_OFF = HIST_OFF + (size_t)BINS * 4;
+    static constexpr size_t BYTES = PERM_OFF + (size_t)kThreads * NBT * 2;
+    static_assert(OUT_BYTES <= TILE_BYTES, "the results fit into the tile's memory");
+    static_assert(kThreads * NBT <= 65536 && BINS == 4 * kThreads, "16-bit block indices; four bins per thread");
+};
+
 template <int DT, int B, int FMT, bool PRUNE>
 __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(QuantArgs p) {
     constexpr bool ONEBLK = (B >= 32);        // the thread owns exactly one block
@@ -465,19 +489,89 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
 
     // With PRUNE the loop is uniform per warp (lanes past the end repeat the warp's first group
     // and store nothing), so that the warp can agree on the candidates it leaves out.
+    //
+    // SORTED (PRUNE with several blocks per thread, B <= 16): what a warp may leave out is decided by the
+    // smallest and the largest block maximum it holds, and with a handful of small blocks per lane a warp
+    // of unsorted blocks holds nearly the whole range of the tensor.  So the CTA first sorts the blocks of
+    // its 256 groups by magnitude (a counting sort on the exponent and two significand bits of the block
+    // maximum, in shared memory), every thread takes NBT neighbours of the sorted order, and the results
+    // travel back through shared memory to the thread that owns the group they belong to, which stores them
+    // and adds their SSEs in the original order.  Which thread evaluates a block changes nothing in its
+    // result, so the outputs do not depend on the (unordered) ranks inside a bin.  The loop is uniform per
+    // CTA in this mode (every barrier below is reached by all 256 threads the same number of times);
+    // groups past the end are filled with zeros and store nothing.
+    constexpr bool SORTED = brute_sorted(B, PRUNE);
+    using Tile = BruteTile<B>;
+    extern __shared__ uint4 brute_dyn[];
+    [[maybe_unused]] unsigned char* const dyn = reinterpret_cast<unsigned char*>(brute_dyn);
+    [[maybe_unused]] float* const tile = reinterpret_cast<float*>(dyn);
+    [[maybe_unused]] uint32_t* const hist = reinterpret_cast<uint32_t*>(dyn + Tile::HIST_OFF);
+    [[maybe_unused]] uint16_t* const perm = reinterpret_cast<uint16_t*>(dyn + Tile::PERM_OFF);
+    __shared__ uint32_t warp_total[kThreads / 32];
     const size_t stride = (size_t)gridDim.x * kThreads;
-    const int lane = PRUNE ? (threadIdx.x & 31) : 0;
+    const int lane = (PRUNE && !SORTED) ? (threadIdx.x & 31) : 0;
     double sse_sum = 0.0;                  // binary64 sum of the SSEs of this thread's blocks, in the order it stored them
-    for (size_t wbase = (size_t)blockIdx.x * kThreads + threadIdx.x - lane; wbase < p.n_items; wbase += stride) {
-        const bool active = wbase + lane < p.n_items;
-        const size_t grp = active ? wbase + lane : wbase;
+    for (size_t wbase = (size_t)blockIdx.x * kThreads + (SORTED ? 0 : threadIdx.x - lane); wbase < p.n_items; wbase += stride) {
+        const bool active = wbase + (SORTED ? threadIdx.x : lane) < p.n_items;
+        const size_t grp = SORTED ? wbase + threadIdx.x : (active ? wbase + lane : wbase);
         float2 v2[NP];
         float amax = 0.0f;
         [[maybe_unused]] float amin = 0.0f;   // PRUNE: smallest block maximum of the thread
         bool tiny = false;   // a nonzero magnitude below 2^-62: its quotient by Dref may be inexact
         {
             float v[G];
-            load_elems<DT, G>(p.x, grp * G, v);
+            if constexpr (SORTED) {
+                // own group -> own (padded) row of the tile; bins cleared
+                if (active) {
+                    load_elems<DT, G>(p.x, grp * G, v);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < G; ++i) v[i] = 0.0f;
+                }
+#pragma unroll
+                for (int i = 0; i < G; ++i) tile[threadIdx.x * Tile::ROW + i] = v[i];
+                reinterpret_cast<uint4*>(hist)[threadIdx.x] = make_uint4(0u, 0u, 0u, 0u);
+                __syncthreads();
+                uint32_t key[NBT], rank[NBT];
+#pragma unroll
+                for (int kb = 0; kb < NBT; ++kb) {
+                    float a = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < B; ++i) a = fmaxf(a, fabsf(v[kb * B + i]));
+                    key[kb] = min(__float_as_uint(a) >> 21, (uint32_t)Tile::BINS - 1u);
+                    rank[kb] = atomicAdd(&hist[key[kb]], 1u);
+                }
+                __syncthreads();
+                {   // exclusive prefix sums over the bins: four bins per thread, a scan over the warps' totals
+                    const uint4 h = reinterpret_cast<const uint4*>(hist)[threadIdx.x];
+                    const uint32_t mine = h.x + h.y + h.z + h.w;
+                    uint32_t incl = mine;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                        if ((threadIdx.x & 31) >= o) incl += up;
+                    }
+                    if ((threadIdx.x & 31) == 31) warp_total[threadIdx.x >> 5] = incl;
+                    __syncthreads();
+                    uint32_t before = incl - mine;
+                    for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) before += warp_total[w];
+                    reinterpret_cast<uint4*>(hist)[threadIdx.x] = make_uint4(before, before + h.x, before + h.x + h.y, before + h.x + h.y + h.z);
+                }
+                __syncthreads();
+#pragma unroll
+                for (int kb = 0; kb < NBT; ++kb) perm[hist[key[kb]] + rank[kb]] = (uint16_t)(threadIdx.x * NBT + kb);
+                __syncthreads();
+#pragma unroll
+                for (int kb = 0; kb < NBT; ++kb) {
+                    const int ob = perm[threadIdx.x * NBT + kb];
+                    const float* src = tile + (ob / NBT) * Tile::ROW + (ob % NBT) * B;
+#pragma unroll
+                    for (int i = 0; i < B; ++i) v[kb * B + i] = src[i];
+                }
+                __syncthreads();   // the tile has been read: its memory takes the results below
+            } else {
+                load_elems<DT, G>(p.x, grp * G, v);
+            }
             if constexpr (PRUNE && !ONEBLK) {
                 float2 bmax[NBL];
 #pragma unroll
@@ -777,6 +871,33 @@ __global__ void __launch_bounds__(kThreads, brute_min_ctas(B, PRUNE)) k_brute(Qu
                                                            t[8 * k + 5], t[8 * k + 6], t[8 * k + 7]);
             }
         }
+        if constexpr (SORTED) {
+            // results to the blocks' original positions, then every thread fetches those of its own group
+            unsigned char* const oc = dyn;
+            unsigned char* const os = dyn + Tile::OUT_SCALES;
+            uint32_t* const oe = reinterpret_cast<uint32_t*>(dyn + Tile::OUT_SSE);
+#pragma unroll
+            for (int kb = 0; kb < NBT; ++kb) {
+                const int ob = perm[threadIdx.x * NBT + kb];
+                if constexpr (B == 2) oc[ob] = (unsigned char)(packed[kb / 4] >> (8 * (kb % 4)));
+                else if constexpr (B == 4) reinterpret_cast<uint16_t*>(oc)[ob] = (uint16_t)(packed[kb / 2] >> (16 * (kb % 2)));
+                else if constexpr (B == 8) reinterpret_cast<uint32_t*>(oc)[ob] = packed[kb];
+                else reinterpret_cast<uint2*>(oc)[ob] = make_uint2(packed[2 * kb], packed[2 * kb + 1]);
+                os[ob] = (unsigned char)(sc[kb / 4] >> (8 * (kb % 4)));
+                oe[ob] = sw[kb];
+            }
+            __syncthreads();
+#pragma unroll
+            for (int k = 0; k < G / 8; ++k) packed[k] = reinterpret_cast<const uint32_t*>(oc)[threadIdx.x * (G / 8) + k];
+#pragma unroll
+            for (int k = 0; k < (NBT + 3) / 4; ++k) sc[k] = 0;
+#pragma unroll
+            for (int kb = 0; kb < NBT; ++kb) {
+                sc[kb / 4] |= (uint32_t)os[threadIdx.x * NBT + kb] << (8 * (kb % 4));
+                sw[kb] = oe[threadIdx.x * NBT + kb];
+            }
+            __syncthreads();   // before the next trip writes the tile
+        }
         if (!PRUNE || active) {
             store_bytes<G / 2>(p.codes + grp * (G / 2), packed);
             store_bytes<NBT>(p.scales + grp * NBT, sc);
@@ -846,10 +967,15 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    constexpr size_t kDynBytes = brute_sorted(B, PRUNE) ? BruteTile<B>::BYTES : 0;   // the sorted mode's tile, bins, permutation
     int resident = ctas_per_sm[dev].load(std::memory_order_relaxed);
     if (resident == 0) {
+        if (kDynBytes > 0) {
+            err = cudaFuncSetAttribute(k_brute<DT, B, FMT, PRUNE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynBytes);
+            if (err != cudaSuccess) return err;
+        }
         int n = 0;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_brute<DT, B, FMT, PRUNE>, kThreads, 0);
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_brute<DT, B, FMT, PRUNE>, kThreads, kDynBytes);
         if (err != cudaSuccess) return err;
         resident = n > 0 ? n : 1;
         ctas_per_sm[dev].store(resident, std::memory_order_relaxed);
@@ -886,7 +1012,7 @@ static cudaError_t launch_brute_inst(const QuantArgs& a, cudaStream_t stream) {
         size_t cap = (size_t)sm_count(dev) * (size_t)resident;
         if (a.mse_partials && cap > (size_t)kMsePartials - 1) cap = kMsePartials - 1;
         const unsigned grid = (unsigned)(want < cap ? want : cap);
-        err = launch_pdl(k_brute<DT, B, FMT, PRUNE>, grid, kThreads, 0, stream, m);
+        err = launch_pdl(k_brute<DT, B, FMT, PRUNE>, grid, kThreads, kDynBytes, stream, m);
         count_launch();
         if (err != cudaSuccess) return err;
         if (a.mse_n_partials) *a.mse_n_partials = (int)grid + m.mse_first;
